@@ -1,0 +1,185 @@
+/*
+ * rkv.h - C ABI of the RefreshKV decode-attention library (CUDA, sm_100a).
+ *
+ * The library implements the per-layer attention work of RefreshKV
+ * (arXiv 2411.05787, Sec. 2.2): the periodic FULL step (attention over the
+ * whole KV cache C_f, attention scores a_L aggregated over the query heads of
+ * each grouped-query group, top-K positions, rebuild of the small cache C_p)
+ * and the cheap PARTIAL steps (attention over C_p), plus the cache append and
+ * the query-similarity refresh trigger.
+ *
+ * General conventions
+ *  - Every pointer is a DEVICE pointer unless its comment says "host".
+ *  - Every call except create/destroy/get_device_status only enqueues work on
+ *    the given stream (a cudaStream_t passed as void*; NULL = default stream)
+ *    and returns; nothing synchronises, nothing is copied to the host.
+ *  - The caller owns all tensors and the stream.  The context owns only its
+ *    scratch workspace (split partials, per-head logits, tickets, a status
+ *    word), sized once in rkv_create.  Calls on one context must not overlap
+ *    on the GPU (they share that workspace): issue them on one stream.
+ *  - bf16 tensors are plain arrays of 16-bit brain floats.  head_dim is 128.
+ *  - Query head h reads KV head h / G, G = n_q_heads / n_kv_heads (1..8).
+ *  - Errors: every call returns an rkv_status.  Bad arguments are detected on
+ *    the host before anything is launched.  Conditions only the device can
+ *    see (append past capacity, a length above the configured maximum,
+ *    a non-finite score) set bits in a sticky device status word and the
+ *    offending access is skipped or clamped; nothing traps.
+ *
+ * Cache layout (rkv_cache).  K and V are each ONE buffer of n_rows rows of 128
+ * bf16 channels (256 bytes per row, base 16-byte aligned).  Sequence b,
+ * KV head g, position p is row  row_offset[b] + g * cap[b] + p.
+ * Ragged batches are packed by choosing row_offset/cap per sequence.
+ */
+#ifndef RKV_H_
+#define RKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RKV_HEAD_DIM 128
+#define RKV_MAX_GROUP 8
+
+typedef struct rkv_ctx rkv_ctx; /* opaque */
+
+typedef enum {
+  RKV_OK = 0,
+  RKV_ERR_INVALID_ARG = 1, /* null pointer, size out of the configured range        */
+  RKV_ERR_UNSUPPORTED = 2, /* head_dim != 128, G > 8, mode not built                */
+  RKV_ERR_WORKSPACE = 3,   /* workspace allocation failed                           */
+  RKV_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (rkv_last_cuda_error)*/
+  RKV_ERR_DEVICE_CHECK = 5 /* rkv_get_device_status found device-side flags set     */
+} rkv_status;
+
+/* bits of the device status word */
+#define RKV_DEV_APPEND_OVERFLOW 1 /* rkv_append: len == cap, row not written            */
+#define RKV_DEV_LEN_CLAMPED 2     /* a seq_len exceeded cap or max_len and was clamped   */
+#define RKV_DEV_NONFINITE 4       /* a NaN/Inf attention logit was seen                  */
+#define RKV_DEV_BAD_INDEX 8       /* rkv_gather_small: index outside [0, len), row skipped*/
+
+/* score aggregation over the query heads of a group (Sec. 2.2 footnote; App. A.3, Table 6) */
+typedef enum { RKV_AGG_MAX = 0, RKV_AGG_MEAN = 1, RKV_AGG_FIRST = 2 } rkv_agg;
+
+typedef struct {
+  int32_t n_seq;         /* B                                                          */
+  int32_t n_q_heads;     /* Hq                                                         */
+  int32_t n_kv_heads;    /* Hkv; Hq % Hkv == 0, Hq / Hkv <= 8                          */
+  int32_t head_dim;      /* must be 128                                                */
+  int32_t max_len;       /* largest full-cache length any call will see                */
+  int32_t max_small;     /* largest small-cache length any call will see               */
+  int32_t agg;           /* rkv_agg; RKV_AGG_MAX is the paper's rule                   */
+  int32_t pool_kernel;   /* 1 = no pooling; odd w > 1 = max-pool of width w (App. A.1) */
+  float softmax_scale;   /* 0 -> 1/sqrt(head_dim)                                      */
+} rkv_config;
+
+typedef struct {
+  void* k;                   /* bf16 [n_rows][128]                                     */
+  void* v;                   /* bf16 [n_rows][128]                                     */
+  int64_t n_rows;            /* host value: rows in each buffer (< 2^31)               */
+  const int64_t* row_offset; /* [B] first row of sequence b                            */
+  const int32_t* cap;        /* [B] capacity of sequence b in positions                */
+  int32_t* len;              /* [B] current length; append / gather_small update it    */
+} rkv_cache;
+
+/* Host.  Creates a context on the current device and allocates its workspace
+ * (cudaMalloc).  *out is NULL on failure. */
+rkv_status rkv_create(const rkv_config* cfg /*host*/, rkv_ctx** out /*host*/);
+/* Host.  Frees the workspace.  The caller must have synchronised its streams. */
+rkv_status rkv_destroy(rkv_ctx* ctx);
+/* Host.  Bytes of device workspace rkv_create allocates for this config (0 if cfg is invalid). */
+size_t rkv_workspace_bytes(const rkv_config* cfg /*host*/);
+
+/*
+ * FULL step (Sec. 2.2 "Decoding with full cache"; App. A.1 on obtaining the
+ * scores; Sec. 2.2 footnote on the group aggregation).  For every sequence b
+ * with active[b] != 0 (active == NULL: all) and n = full->len[b]:
+ *   s[h][j]   = scale * <q[b][h], K[b][h/G][j]>               j < n
+ *   p[h][j]   = softmax_j(s[h][:])
+ *   out[b][h] = sum_j p[h][j] V[b][h/G][j]                     (bf16)
+ *   score[b][g][j] = agg_{h in group g} p[h][j]                (fp32, optional output)
+ *   topk_idx[b][g][0..m) = the m = min(k_small[b], n) positions of largest
+ *       score, ties to the lower position, listed in ASCENDING position
+ *       order; entries m..k_max-1 are -1.
+ * If q_last_full != NULL, q[b] is copied there for the active sequences (the
+ * reference query of the refresh trigger).  Inactive sequences: nothing is
+ * read or written.
+ *   q            bf16 [B][Hq][128]
+ *   k_small      int32 [B]  small-cache size per sequence, 0 <= k_small[b] <= k_max
+ *   k_max        host value, 1..max_small
+ *   out          bf16 [B][Hq][128]
+ *   scores       fp32 [B][Hkv][score_stride] or NULL; positions >= n are not written
+ *   score_stride host value >= max length in this call (ignored if scores == NULL)
+ *   topk_idx     int32 [B][Hkv][k_max]
+ *   max_len_hint host value: upper bound of full->len[b] over active b in this
+ *                call (0 = cfg.max_len).  Only launch geometry depends on it;
+ *                a longer sequence is clamped and flagged RKV_DEV_LEN_CLAMPED.
+ */
+rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
+                         const int32_t* k_small, int32_t k_max, const int32_t* active,
+                         void* out, float* scores, int64_t score_stride, int32_t* topk_idx,
+                         void* q_last_full, int32_t max_len_hint, void* stream);
+
+/*
+ * Rebuild C_p from the selected positions (Sec. 2.2 "refresh the partial
+ * cache").  For active b, KV head g, r < m = min(k_small[b], full->len[b]):
+ *   small.K[b][g][r] = full.K[b][g][topk_idx[b][g][r]]   (same for V; bit copy)
+ * and small->len[b] = m.  Entries of topk_idx that are -1 are skipped; an
+ * index outside [0, full->len[b]) is skipped and flagged RKV_DEV_BAD_INDEX.
+ * Requires m <= small->cap[b].
+ */
+rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t* k_small,
+                            int32_t k_max, const rkv_cache* full /*host struct*/,
+                            const rkv_cache* small_cache /*host struct*/, const int32_t* active,
+                            void* stream);
+
+/*
+ * PARTIAL step (Sec. 2.2 "Decoding with partial cache"): softmax attention of
+ * q over the first small->len[b] rows of the small cache, for sequences with
+ * active[b] != 0 (NULL: all).  out as in rkv_full_step.  max_len_hint: upper
+ * bound of small->len[b] (0 = cfg.max_small).
+ */
+rkv_status rkv_small_step(rkv_ctx* ctx, const void* q, const rkv_cache* small_cache /*host struct*/,
+                          const int32_t* active, void* out, int32_t max_len_hint, void* stream);
+
+/*
+ * Append the current token's key/value (Sec. 2.1: the cache is updated with
+ * the current token's pair; Sec. 2.2: both C_p and C_f receive it).  For each
+ * non-NULL cache c and every b: row len[b] of every KV head receives
+ * k_new[b][g] / v_new[b][g], then c->len[b] += 1.  If len[b] == cap[b] nothing
+ * is written for that sequence and RKV_DEV_APPEND_OVERFLOW is set.
+ *   k_new, v_new  bf16 [B][Hkv][128]
+ */
+rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new,
+                      const rkv_cache* full /*host struct or NULL*/,
+                      const rkv_cache* small_cache /*host struct or NULL*/, void* stream);
+
+/*
+ * Refresh trigger (Sec. 2.2 "Deciding when to decode with full cache").
+ *   qbar  = mean over the Hq heads of q_now[b];  qbar' likewise from q_last_full[b]
+ *   sim   = <qbar, qbar'> / (|qbar| |qbar'|)          (fp32)
+ *   flag[b] = 0 (partial step) if sim > threshold, else 1 (full step);
+ *   equality and NaN (a zero mean vector) give 1.
+ *   q_now, q_last_full  bf16 [B][Hq][128];  flag int32 [B];  sim fp32 [B] or NULL
+ */
+rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_last_full,
+                              float threshold, int32_t* flag, float* sim, void* stream);
+
+/* Host.  Synchronises the stream, copies the sticky device status word to
+ * *host_bits, clears it, and returns RKV_ERR_DEVICE_CHECK if it was non-zero. */
+rkv_status rkv_get_device_status(rkv_ctx* ctx, int32_t* host_bits /*host*/, void* stream);
+
+/* Host.  Static strings; never NULL. */
+const char* rkv_status_string(rkv_status s);
+const char* rkv_last_cuda_error(const rkv_ctx* ctx);
+
+/* Host.  Number of kernels this context has launched since creation (each call
+ * above launches a fixed, documented number; used by benchmarks to report it). */
+int64_t rkv_launch_count(const rkv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RKV_H_ */

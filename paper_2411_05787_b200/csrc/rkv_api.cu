@@ -1,0 +1,323 @@
+// C ABI of librkv: argument validation, workspace, tensor maps, launches.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "rkv_internal.h"
+
+namespace {
+
+using rkv::AttnParams;
+using rkv::CacheDev;
+using rkv::SelectParams;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn g_encode = nullptr;
+bool g_prepared = false;
+
+bool config_ok(const rkv_config* c, rkv_status* why) {
+  if (c == nullptr) { *why = RKV_ERR_INVALID_ARG; return false; }
+  if (c->n_seq < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_len < 1 || c->max_small < 1 ||
+      c->n_q_heads % c->n_kv_heads != 0) { *why = RKV_ERR_INVALID_ARG; return false; }
+  if (c->head_dim != rkv::kHeadDim || c->n_q_heads / c->n_kv_heads > rkv::kMaxGroup ||
+      c->agg < RKV_AGG_MAX || c->agg > RKV_AGG_FIRST || c->pool_kernel != 1 ||
+      (int64_t)c->max_len > (int64_t)rkv::kSelectCluster * rkv::kSelectMaxKeysPerCta ||
+      (int64_t)c->n_seq * c->n_kv_heads > 65535 * 8) { *why = RKV_ERR_UNSUPPORTED; return false; }
+  if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) { *why = RKV_ERR_INVALID_ARG; return false; }
+  return true;
+}
+
+int splits_for(const rkv_config* c) {
+  int s = (c->max_len + rkv::kTile - 1) / rkv::kTile;
+  return s < rkv::kMaxSplits ? (s < 1 ? 1 : s) : rkv::kMaxSplits;
+}
+
+struct WsLayout { size_t partials, tickets, lse, logits, status, total; int64_t logit_stride; };
+
+WsLayout ws_layout(const rkv_config* c) {
+  WsLayout w;
+  const size_t bg = (size_t)c->n_seq * c->n_kv_heads;
+  const int group = c->n_q_heads / c->n_kv_heads;
+  auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+  w.logit_stride = ((int64_t)c->max_len + 63) & ~int64_t(63);
+  size_t off = 0;
+  w.partials = off; off = up(off + bg * splits_for(c) * rkv::PartialLayout::kFloats * sizeof(float));
+  w.tickets = off;  off = up(off + bg * sizeof(int32_t));
+  w.lse = off;      off = up(off + (size_t)c->n_seq * c->n_q_heads * sizeof(double));
+  w.logits = off;   off = up(off + bg * group * (size_t)w.logit_stride * sizeof(float));
+  w.status = off;   off = up(off + sizeof(int32_t));
+  w.total = off;
+  return w;
+}
+
+rkv_status cuda_fail(rkv_ctx* ctx, cudaError_t e, const char* where) {
+  if (ctx) ctx->last_error = std::string(where) + ": " + cudaGetErrorString(e);
+  return RKV_ERR_CUDA;
+}
+
+bool cache_ok(const rkv_cache* c) {
+  return c && c->k && c->v && c->row_offset && c->cap && c->len && c->n_rows > 0 && c->n_rows < (int64_t(1) << 31) &&
+         (reinterpret_cast<uintptr_t>(c->k) & 15) == 0 && (reinterpret_cast<uintptr_t>(c->v) & 15) == 0;
+}
+
+CacheDev dev_of(const rkv_cache* c) { return CacheDev{c->k, c->v, c->row_offset, c->cap, c->len}; }
+
+// 2-D view [n_rows][128] bf16, box = 64 rows x 64 channels (128 bytes), 128-byte swizzle
+rkv_status tensor_map(rkv_ctx* ctx, void* base, int64_t n_rows, CUtensorMap* out) {
+  const uint64_t key = reinterpret_cast<uint64_t>(base) ^ ((uint64_t)n_rows * 0x9E3779B97F4A7C15ull);
+  auto it = ctx->tmaps.find(key);
+  if (it != ctx->tmaps.end()) { *out = it->second; return RKV_OK; }
+  if (g_encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess)
+      return cuda_fail(ctx, e == cudaSuccess ? cudaErrorUnknown : e, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)");
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  cuuint64_t dims[2] = {(cuuint64_t)rkv::kHeadDim, (cuuint64_t)n_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)rkv::kHeadDim * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)rkv::kTile};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap tm;
+  CUresult r = g_encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    ctx->last_error = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string((int)r);
+    return RKV_ERR_CUDA;
+  }
+  if (ctx->tmaps.size() > 8192) ctx->tmaps.clear();
+  ctx->tmaps.emplace(key, tm);
+  *out = tm;
+  return RKV_OK;
+}
+
+// positions per CTA: one balanced wave over 2 CTAs per SM when that keeps chunks moderate,
+// otherwise fixed 2048-position chunks over several waves (ragged batches balance by count)
+int choose_chunk(const rkv_ctx* ctx, int n_max, int* grid_x) {
+  const int bg = ctx->cfg.n_seq * ctx->cfg.n_kv_heads;
+  const int slots = 2 * ctx->sm_count;
+  int splits = slots / bg;
+  if (splits < 1) splits = 1;
+  if (splits > ctx->max_splits) splits = ctx->max_splits;
+  int chunk = (n_max + splits - 1) / splits;
+  if (chunk > 4096) chunk = 2048;
+  if (chunk < rkv::kTile) chunk = rkv::kTile;
+  chunk = (chunk + 15) & ~15;
+  int gx = (n_max + chunk - 1) / chunk;
+  while (gx > ctx->max_splits) {  // keep the partial buffer's bound
+    chunk *= 2;
+    gx = (n_max + chunk - 1) / chunk;
+  }
+  *grid_x = gx < 1 ? 1 : gx;
+  return chunk;
+}
+
+rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
+                         void* q_last_full, int n_max, int limit, bool logits, cudaStream_t st) {
+  CUtensorMap tm_k, tm_v;
+  rkv_status s = tensor_map(ctx, cache->k, cache->n_rows, &tm_k);
+  if (s != RKV_OK) return s;
+  s = tensor_map(ctx, cache->v, cache->n_rows, &tm_v);
+  if (s != RKV_OK) return s;
+  AttnParams p;
+  memset(&p, 0, sizeof(p));
+  int gx = 1;
+  p.chunk = choose_chunk(ctx, n_max, &gx);
+  p.q = q;
+  p.row_offset = cache->row_offset;
+  p.cap = cache->cap;
+  p.len = cache->len;
+  p.active = active;
+  p.out = out;
+  p.partials = ctx->partials;
+  p.tickets = ctx->tickets;
+  p.lse = ctx->lse;
+  p.logits = logits ? ctx->logits : nullptr;
+  p.q_last_full = q_last_full;
+  p.status = ctx->status;
+  p.logit_stride = ctx->logit_stride;
+  p.n_q_heads = ctx->cfg.n_q_heads;
+  p.n_kv_heads = ctx->cfg.n_kv_heads;
+  p.group = ctx->group;
+  p.max_splits = ctx->max_splits;
+  p.max_len = limit;
+  p.scale = ctx->cfg.softmax_scale;
+  cudaError_t e = rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
+  ctx->launches += 1;
+  return RKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rkv_workspace_bytes(const rkv_config* cfg) {
+  rkv_status why;
+  if (!config_ok(cfg, &why)) return 0;
+  return ws_layout(cfg).total;
+}
+
+rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
+  if (out == nullptr) return RKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  rkv_status why;
+  if (!config_ok(cfg, &why)) return why;
+  rkv_ctx* ctx = new (std::nothrow) rkv_ctx();
+  if (ctx == nullptr) return RKV_ERR_WORKSPACE;
+  ctx->cfg = *cfg;
+  if (ctx->cfg.softmax_scale == 0.f) ctx->cfg.softmax_scale = 1.0f / sqrtf((float)cfg->head_dim);
+  ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
+  ctx->max_splits = splits_for(cfg);
+  ctx->launches = 0;
+  ctx->workspace = nullptr;
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
+  if (e != cudaSuccess) { delete ctx; return RKV_ERR_CUDA; }
+  if (!g_prepared) {
+    e = rkv::prepare_attention();
+    if (e == cudaSuccess) e = rkv::prepare_select();
+    if (e != cudaSuccess) { delete ctx; return RKV_ERR_CUDA; }
+    g_prepared = true;
+  }
+  const WsLayout w = ws_layout(cfg);
+  e = cudaMalloc(reinterpret_cast<void**>(&ctx->workspace), w.total);
+  if (e != cudaSuccess) { delete ctx; return RKV_ERR_WORKSPACE; }
+  e = cudaMemset(ctx->workspace, 0, w.total);
+  if (e != cudaSuccess) { cudaFree(ctx->workspace); delete ctx; return RKV_ERR_CUDA; }
+  ctx->workspace_bytes = w.total;
+  ctx->partials = reinterpret_cast<float*>(ctx->workspace + w.partials);
+  ctx->tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.tickets);
+  ctx->lse = reinterpret_cast<double*>(ctx->workspace + w.lse);
+  ctx->logits = reinterpret_cast<float*>(ctx->workspace + w.logits);
+  ctx->status = reinterpret_cast<int32_t*>(ctx->workspace + w.status);
+  ctx->logit_stride = w.logit_stride;
+  *out = ctx;
+  return RKV_OK;
+}
+
+rkv_status rkv_destroy(rkv_ctx* ctx) {
+  if (ctx == nullptr) return RKV_ERR_INVALID_ARG;
+  cudaError_t e = cudaSuccess;
+  if (ctx->workspace) e = cudaFree(ctx->workspace);
+  delete ctx;
+  return e == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+}
+
+rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
+                         const int32_t* active, void* out, float* scores, int64_t score_stride, int32_t* topk_idx,
+                         void* q_last_full, int32_t max_len_hint, void* stream) {
+  if (!ctx || !q || !cache_ok(full) || !k_small || !out || !topk_idx) return RKV_ERR_INVALID_ARG;
+  if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+  int n_max = max_len_hint == 0 ? ctx->cfg.max_len : max_len_hint;
+  if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
+  if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rkv_status s = run_attention(ctx, q, full, active, out, q_last_full, n_max, n_max, true, st);
+  if (s != RKV_OK) return s;
+  SelectParams sp;
+  memset(&sp, 0, sizeof(sp));
+  sp.logits = ctx->logits;
+  sp.lse = ctx->lse;
+  sp.len = full->len;
+  sp.k_small = k_small;
+  sp.active = active;
+  sp.scores = scores;
+  sp.topk_idx = topk_idx;
+  sp.status = ctx->status;
+  sp.logit_stride = ctx->logit_stride;
+  sp.score_stride = score_stride;
+  sp.n_q_heads = ctx->cfg.n_q_heads;
+  sp.n_kv_heads = ctx->cfg.n_kv_heads;
+  sp.group = ctx->group;
+  sp.agg = ctx->cfg.agg;
+  sp.k_max = k_max;
+  sp.max_len = n_max;
+  int per = (n_max + rkv::kSelectCluster - 1) / rkv::kSelectCluster;
+  sp.keys_per_cta = (per + 3) & ~3;
+  cudaError_t e = rkv::launch_select(sp, ctx->cfg.n_seq, st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
+  ctx->launches += 1;
+  return RKV_OK;
+}
+
+rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t* k_small, int32_t k_max,
+                            const rkv_cache* full, const rkv_cache* small_cache, const int32_t* active,
+                            void* stream) {
+  if (!ctx || !topk_idx || !k_small || !cache_ok(full) || !cache_ok(small_cache)) return RKV_ERR_INVALID_ARG;
+  if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+  cudaError_t e = rkv::launch_gather(topk_idx, k_small, k_max, dev_of(full), dev_of(small_cache), active,
+                                     ctx->cfg.n_seq, ctx->cfg.n_kv_heads, ctx->status,
+                                     static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "gather launch");
+  ctx->launches += 1;
+  return RKV_OK;
+}
+
+rkv_status rkv_small_step(rkv_ctx* ctx, const void* q, const rkv_cache* small_cache, const int32_t* active,
+                          void* out, int32_t max_len_hint, void* stream) {
+  if (!ctx || !q || !cache_ok(small_cache) || !out) return RKV_ERR_INVALID_ARG;
+  int n_max = max_len_hint == 0 ? ctx->cfg.max_small : max_len_hint;
+  if (n_max < 1 || n_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+  return run_attention(ctx, q, small_cache, active, out, nullptr, n_max, n_max, false,
+                       static_cast<cudaStream_t>(stream));
+}
+
+rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const rkv_cache* full,
+                      const rkv_cache* small_cache, void* stream) {
+  if (!ctx || !k_new || !v_new || (full == nullptr && small_cache == nullptr)) return RKV_ERR_INVALID_ARG;
+  if ((full && !cache_ok(full)) || (small_cache && !cache_ok(small_cache))) return RKV_ERR_INVALID_ARG;
+  CacheDev none = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  cudaError_t e = rkv::launch_append(k_new, v_new, full ? dev_of(full) : none, small_cache ? dev_of(small_cache) : none,
+                                     full != nullptr, small_cache != nullptr, ctx->cfg.n_seq, ctx->cfg.n_kv_heads,
+                                     ctx->status, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "append launch");
+  ctx->launches += 1;
+  return RKV_OK;
+}
+
+rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_last_full, float threshold,
+                              int32_t* flag, float* sim, void* stream) {
+  if (!ctx || !q_now || !q_last_full || !flag) return RKV_ERR_INVALID_ARG;
+  cudaError_t e = rkv::launch_trigger(q_now, q_last_full, threshold, flag, sim, ctx->cfg.n_seq, ctx->cfg.n_q_heads,
+                                      static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "trigger launch");
+  ctx->launches += 1;
+  return RKV_OK;
+}
+
+rkv_status rkv_get_device_status(rkv_ctx* ctx, int32_t* host_bits, void* stream) {
+  if (!ctx || !host_bits) return RKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t bits = 0;
+  cudaError_t e = cudaMemcpyAsync(&bits, ctx->status, sizeof(bits), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, sizeof(int32_t), st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "status read");
+  *host_bits = bits;
+  return bits == 0 ? RKV_OK : RKV_ERR_DEVICE_CHECK;
+}
+
+const char* rkv_status_string(rkv_status s) {
+  switch (s) {
+    case RKV_OK: return "ok";
+    case RKV_ERR_INVALID_ARG: return "invalid argument";
+    case RKV_ERR_UNSUPPORTED: return "unsupported configuration";
+    case RKV_ERR_WORKSPACE: return "workspace allocation failed";
+    case RKV_ERR_CUDA: return "CUDA error";
+    case RKV_ERR_DEVICE_CHECK: return "device-side check failed";
+  }
+  return "unknown status";
+}
+
+const char* rkv_last_cuda_error(const rkv_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+int64_t rkv_launch_count(const rkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

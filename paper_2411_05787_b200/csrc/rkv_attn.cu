@@ -1,0 +1,429 @@
+// Split-K grouped-query decode attention over a packed bf16 KV cache (sm_100a).
+//
+// What it computes (RefreshKV, arXiv 2411.05787, Sec. 2.2 "Decoding with full
+// cache" / "Decoding with partial cache"): for one query token per sequence,
+//   s[h][j] = scale <q[h], K[g][j]>,  p = softmax_j s,  out[h] = sum_j p[h][j] V[g][j],
+// g = h / G.  The full step additionally needs the attention scores a_L of the
+// current token (App. A.1: the paper recomputes them in a second pass because
+// its library attention hides them); here the scaled logits are written out by
+// the same pass that streams K, so the cache is read from HBM exactly once.
+//
+// Shape of the kernel: one CTA per (sequence, KV head, chunk of positions).
+// A copy warp streams 64-position tiles of K and V into a 3-stage shared-memory
+// ring with 2-D tensor-map TMA loads (128-byte swizzle, completion on
+// mbarriers).  Four MMA warps each own 16 positions of a tile: S^T = K Q^T and
+// O^T += V^T P^T with m16n8k16 bf16 tensor-core MMAs (fp32 accumulate), where
+// the N=8 dimension holds all query heads of the group, so K/V are read once
+// per group.  Online softmax lives in registers; the split partials are merged
+// by the last CTA of each (sequence, KV head) to arrive (atomic ticket, no
+// spinning).
+#include <cuda_bf16.h>
+
+#include "rkv_internal.h"
+
+namespace rkv {
+namespace {
+
+constexpr int kStageBytes = 4 * kTile * 128;  // K lo/hi + V lo/hi halves, 64 rows x 128 B each
+constexpr int kHalfBytes = kTile * 128;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kOPad = 132;  // floats per head row in the merge buffer (bank spread)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls so that a lost copy can never hang the GPU.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
+                                            uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+      "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+template <bool kLogits>
+__global__ void __launch_bounds__(kAttnThreads, 2)
+attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+            const AttnParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int s_last;
+
+  const int b = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
+  if (p.active != nullptr && p.active[b] == 0) return;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = p.group;
+  const int cap = p.cap[b];
+  int n = p.len[b];
+  {
+    const int lim = cap < p.max_len ? cap : p.max_len;
+    if (n > lim) {
+      n = lim;
+      if (tid == 0 && split == 0) atomicOr(p.status, RKV_DEV_LEN_CLAMPED);
+    }
+    if (n < 0) n = 0;
+  }
+  __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
+  const __nv_bfloat16* qg =
+      static_cast<const __nv_bfloat16*>(p.q) + ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
+  if (n == 0) {  // nothing cached: the output is defined as zero
+    if (split == 0 && tid < kHeadDim)
+      for (int h = 0; h < G; ++h) out[h * kHeadDim + tid] = __float2bfloat16(0.f);
+    return;
+  }
+  const int start = split * p.chunk;
+  if (start >= n) return;
+  const int end = (start + p.chunk < n) ? start + p.chunk : n;
+  const int n_tiles = (end - start + kTile - 1) / kTile;
+  const int n_splits = (n + p.chunk - 1) / p.chunk;
+  const int64_t row0 = p.row_offset[b] + (int64_t)g * cap + start;
+
+  // shared memory: [stages][K lo | K hi | V lo | V hi], then the barriers
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_full = smem_base + kStages * kStageBytes;
+  const uint32_t bar_empty = bar_full + 8 * kStages;
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == 4) {
+    // ------------------------------------------------------------ copy warp
+    if (lane == 0) {
+      uint64_t policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      for (int t = 0; t < n_tiles; ++t) {
+        const int s = t % kStages, use = t / kStages;
+        if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1)) {
+          atomicOr(p.status, kDevTimeoutBit);
+          break;
+        }
+        const uint32_t dst = smem_base + s * kStageBytes;
+        const uint32_t bar = bar_full + 8 * s;
+        const int y = (int)(row0 + (int64_t)t * kTile);
+        mbar_expect_tx(bar, kStageBytes);
+        tma_load_2d(dst, &tm_k, 0, y, bar, policy);
+        tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar, policy);
+        tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
+        tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
+      }
+    }
+    return;
+  }
+
+  // ---------------------------------------------------------------- MMA warps
+  const int qd = lane >> 2;       // row inside an 8-row group
+  const int qc = (lane & 3) * 2;  // first of the two columns this lane holds
+  uint32_t qb[8][2];              // B fragments of Q^T: [k = channel][n = head]
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    if (qd < G) {
+      qb[ks][0] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc);
+      qb[ks][1] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc + 8);
+    } else {
+      qb[ks][0] = 0u;
+      qb[ks][1] = 0u;
+    }
+  }
+  const float ninf = -INFINITY;
+  float m0 = ninf, m1 = ninf, l0 = 0.f, l1 = 0.f;
+  float o[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+
+  float* lg0 = nullptr;
+  if (kLogits) lg0 = p.logits + ((int64_t)(b * p.n_kv_heads + g) * G + qc) * p.logit_stride;
+
+  const int krow = 16 * warp + (lane & 15);
+  const int vrow = 16 * warp + ((lane >> 4) << 3) + (lane & 7);
+  bool ok = true;
+
+  for (int t = 0; t < n_tiles; ++t) {
+    const int s = t % kStages;
+    if (!mbar_wait(bar_full + 8 * s, (t / kStages) & 1)) {
+      if (lane == 0) atomicOr(p.status, kDevTimeoutBit);
+      ok = false;
+      break;
+    }
+    const int pos_base = start + t * kTile + 16 * warp;
+    if (pos_base < end) {
+      const uint32_t kbase = smem_base + s * kStageBytes;
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const int chunk = 2 * ks + (lane >> 4);
+        uint32_t a[4];
+        ldsm_x4(a, kbase + (chunk >> 3) * kHalfBytes + krow * 128 + (((chunk & 7) ^ (krow & 7)) << 4));
+        mma_bf16(c, a, qb[ks][0], qb[ks][1]);
+      }
+      const int r0 = pos_base + qd, r1 = r0 + 8;
+      float s0 = c[0] * p.scale, s1 = c[1] * p.scale, s2 = c[2] * p.scale, s3 = c[3] * p.scale;
+      if (kLogits) {
+        if (qc < G) {
+          if (r0 < end) lg0[r0] = s0;
+          if (r1 < end) lg0[r1] = s2;
+        }
+        if (qc + 1 < G) {
+          if (r0 < end) lg0[p.logit_stride + r0] = s1;
+          if (r1 < end) lg0[p.logit_stride + r1] = s3;
+        }
+      }
+      if (r0 >= end) s0 = s1 = ninf;
+      if (r1 >= end) s2 = s3 = ninf;
+      float t0 = fmaxf(s0, s2), t1 = fmaxf(s1, s3);
+#pragma unroll
+      for (int sh = 4; sh <= 16; sh <<= 1) {
+        t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, sh));
+        t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, sh));
+      }
+      const float n0 = fmaxf(m0, t0), n1 = fmaxf(m1, t1);
+      if (__any_sync(0xffffffffu, (n0 > m0) || (n1 > m1))) {
+        const float a0 = (n0 == m0) ? 1.f : ex2((m0 - n0) * kLog2e);
+        const float a1 = (n1 == m1) ? 1.f : ex2((m1 - n1) * kLog2e);
+        l0 *= a0;
+        l1 *= a1;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          o[i][0] *= a0;
+          o[i][1] *= a1;
+          o[i][2] *= a0;
+          o[i][3] *= a1;
+        }
+        m0 = n0;
+        m1 = n1;
+      }
+      const float nm0 = (m0 == ninf) ? 0.f : -m0 * kLog2e;
+      const float nm1 = (m1 == ninf) ? 0.f : -m1 * kLog2e;
+      const float p0 = ex2(fmaf(s0, kLog2e, nm0)), p1 = ex2(fmaf(s1, kLog2e, nm1));
+      const float p2 = ex2(fmaf(s2, kLog2e, nm0)), p3 = ex2(fmaf(s3, kLog2e, nm1));
+      l0 += p0 + p2;
+      l1 += p1 + p3;
+      // P^T as the B operand: transpose the two 8x8 [position][head] blocks inside the warp
+      const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1));
+      const uint32_t pb1 = movmatrix_t(pack_bf16(p2, p3));
+      const uint32_t vbase = kbase + 2 * kHalfBytes;
+      const bool tail = pos_base + 16 > end;
+      uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
+      if (tail) {  // rows past the end may hold anything (even NaN): zero them so that 0 * x stays 0
+        const int pa = pos_base + qc;
+        mk0 = (pa < end ? 0x0000ffffu : 0u) | (pa + 1 < end ? 0xffff0000u : 0u);
+        mk1 = (pa + 8 < end ? 0x0000ffffu : 0u) | (pa + 9 < end ? 0xffff0000u : 0u);
+      }
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        const int chunk = 2 * mt + ((lane >> 3) & 1);
+        uint32_t a[4];
+        ldsm_x4_t(a, vbase + (chunk >> 3) * kHalfBytes + vrow * 128 + (((chunk & 7) ^ (vrow & 7)) << 4));
+        if (tail) {
+          a[0] &= mk0;
+          a[1] &= mk0;
+          a[2] &= mk1;
+          a[3] &= mk1;
+        }
+        mma_bf16(o[mt], a, pb0, pb1);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+  }
+
+#pragma unroll
+  for (int sh = 4; sh <= 16; sh <<= 1) {
+    l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+  }
+
+  // ------------------------------------------------ merge the four warps (stage memory is free now)
+  consumer_bar();
+  float* sm_o = reinterpret_cast<float*>(smem_gen);   // [4][8][kOPad]
+  float* sm_ml = sm_o + 4 * 8 * kOPad;                // [4][8][2]
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    const int d = 16 * mt + qd;
+    float* base = sm_o + (warp * 8 + qc) * kOPad;
+    base[d] = o[mt][0];
+    base[kOPad + d] = o[mt][1];
+    base[d + 8] = o[mt][2];
+    base[kOPad + d + 8] = o[mt][3];
+  }
+  if (lane < 4) {
+    float* ml = sm_ml + (warp * 8 + qc) * 2;
+    ml[0] = m0;
+    ml[1] = l0;
+    ml[2] = m1;
+    ml[3] = l1;
+  }
+  consumer_bar();
+
+  const int d = tid;  // 0..127: one output channel per thread
+  float accO[kMaxGroup], accM[kMaxGroup], accL[kMaxGroup];
+#pragma unroll
+  for (int h = 0; h < kMaxGroup; ++h) {
+    float M = ninf;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) M = fmaxf(M, sm_ml[(w * 8 + h) * 2]);
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float mw = sm_ml[(w * 8 + h) * 2];
+      const float e = (mw == ninf) ? 0.f : ex2((mw - M) * kLog2e);
+      L += sm_ml[(w * 8 + h) * 2 + 1] * e;
+      O += sm_o[(w * 8 + h) * kOPad + d] * e;
+    }
+    accO[h] = O;
+    accM[h] = M;
+    accL[h] = L;
+  }
+
+  const int bg = b * p.n_kv_heads + g;
+  if (n_splits > 1) {
+    float* part = p.partials + ((int64_t)bg * p.max_splits + split) * PartialLayout::kFloats;
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h)
+      if (h < G) part[h * kHeadDim + d] = accO[h];
+    if (d < G) {
+      float Md = ninf, Ld = 0.f;
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h == d) {
+          Md = accM[h];
+          Ld = accL[h];
+        }
+      part[kMaxGroup * kHeadDim + d] = Md;
+      part[kMaxGroup * kHeadDim + kMaxGroup + d] = Ld;
+    }
+    __threadfence();
+    consumer_bar();
+    if (tid == 0) {
+      const int old = atomicAdd(p.tickets + bg, 1);
+      s_last = (old == n_splits - 1) ? 1 : 0;
+    }
+    consumer_bar();
+    if (!s_last) return;
+    __threadfence();
+    // last CTA of this (sequence, KV head): fold all split partials
+    const float* pbase = p.partials + (int64_t)bg * p.max_splits * PartialLayout::kFloats;
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) {
+      if (h < G) {
+        float M = ninf;
+        for (int sidx = 0; sidx < n_splits; ++sidx)
+          M = fmaxf(M, __ldcg(pbase + (int64_t)sidx * PartialLayout::kFloats + kMaxGroup * kHeadDim + h));
+        float L = 0.f, O = 0.f;
+        for (int sidx = 0; sidx < n_splits; ++sidx) {
+          const float* ps = pbase + (int64_t)sidx * PartialLayout::kFloats;
+          const float ms = __ldcg(ps + kMaxGroup * kHeadDim + h);
+          const float e = (ms == ninf) ? 0.f : ex2((ms - M) * kLog2e);
+          L += __ldcg(ps + kMaxGroup * kHeadDim + kMaxGroup + h) * e;
+          O += __ldcg(ps + h * kHeadDim + d) * e;
+        }
+        accO[h] = O;
+        accM[h] = M;
+        accL[h] = L;
+      }
+    }
+    if (tid == 0) p.tickets[bg] = 0;  // ready for the next call on this stream
+  }
+
+  if (!ok) return;
+#pragma unroll
+  for (int h = 0; h < kMaxGroup; ++h) {
+    if (h < G) {
+      out[h * kHeadDim + d] = __float2bfloat16(accO[h] / accL[h]);
+      if (d == 0) p.lse[(int64_t)b * p.n_q_heads + g * G + h] = (double)accM[h] + log((double)accL[h]);
+    }
+  }
+  if (p.q_last_full != nullptr) {
+    __nv_bfloat16* ql =
+        static_cast<__nv_bfloat16*>(p.q_last_full) + ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
+    for (int h = 0; h < G; ++h) ql[h * kHeadDim + d] = qg[h * kHeadDim + d];
+  }
+}
+
+}  // namespace
+
+size_t attention_smem_bytes() { return (size_t)kStages * kStageBytes + 16 * kStages + 1024; }
+
+cudaError_t prepare_attention() {
+  cudaError_t e = cudaFuncSetAttribute(attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)attention_smem_bytes());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)attention_smem_bytes());
+}
+
+cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                             int n_seq, int grid_x, bool write_logits, cudaStream_t st) {
+  dim3 grid(grid_x, p.n_kv_heads, n_seq);
+  if (write_logits)
+    attn_kernel<true><<<grid, kAttnThreads, attention_smem_bytes(), st>>>(tm_k, tm_v, p);
+  else
+    attn_kernel<false><<<grid, kAttnThreads, attention_smem_bytes(), st>>>(tm_k, tm_v, p);
+  return cudaGetLastError();
+}
+
+}  // namespace rkv

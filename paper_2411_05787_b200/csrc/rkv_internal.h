@@ -1,0 +1,106 @@
+// Internal declarations shared by the translation units of librkv (not part of the ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <unordered_map>
+
+#include "rkv.h"
+
+namespace rkv {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxGroup = 8;
+constexpr int kMaxSplits = 128;        // split-K partials kept per (sequence, KV head)
+constexpr int kTile = 64;              // positions per pipeline stage
+constexpr int kStages = 3;
+constexpr int kAttnThreads = 160;      // 4 MMA warps + 1 copy warp
+constexpr int kSelectCluster = 8;      // CTAs that share one top-K problem
+constexpr int kSelectThreads = 256;
+constexpr int kSelectMaxKeysPerCta = 40960;
+constexpr int kDevTimeoutBit = 16;     // internal: a bounded barrier wait ran out
+
+struct PartialLayout {                 // split-K partial of one (b, g, split)
+  // o: [8 heads][128] fp32 unnormalised, then m[8], l[8]
+  static constexpr int kFloats = kMaxGroup * kHeadDim + 2 * kMaxGroup;
+};
+
+struct AttnParams {
+  const void* q;              // bf16 [B][Hq][128]
+  const int64_t* row_offset;  // [B]
+  const int32_t* cap;         // [B]
+  const int32_t* len;         // [B]
+  const int32_t* active;      // [B] or null
+  void* out;                  // bf16 [B][Hq][128]
+  float* partials;            // [B*Hkv][max_splits][PartialLayout::kFloats]
+  int32_t* tickets;           // [B*Hkv]
+  double* lse;                // [B][Hq]   (log-sum-exp of the scaled logits)
+  float* logits;              // [B*Hkv][G][logit_stride] or null
+  void* q_last_full;          // bf16 [B][Hq][128] or null
+  int32_t* status;
+  int64_t logit_stride;
+  int32_t n_q_heads, n_kv_heads, group;
+  int32_t chunk;              // positions per CTA
+  int32_t max_splits;
+  int32_t max_len;            // clamp for len[b]
+  float scale;
+};
+
+struct SelectParams {
+  const float* logits;        // [B*Hkv][G][logit_stride]
+  const double* lse;          // [B][Hq]
+  const int32_t* len;
+  const int32_t* k_small;     // [B]
+  const int32_t* active;
+  float* scores;              // [B][Hkv][score_stride] or null
+  int32_t* topk_idx;          // [B][Hkv][k_max]
+  int32_t* status;
+  int64_t logit_stride, score_stride;
+  int32_t n_q_heads, n_kv_heads, group, agg;
+  int32_t k_max, max_len;
+  int32_t keys_per_cta;       // capacity of the shared-memory key array
+};
+
+struct CacheDev {
+  void* k; void* v;
+  const int64_t* row_offset; const int32_t* cap; int32_t* len;
+};
+
+cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                             int n_seq, int grid_x, bool write_logits, cudaStream_t st);
+cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st);
+cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
+                          CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
+                          int32_t* status, cudaStream_t st);
+cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, CacheDev small_cache,
+                          bool has_full, bool has_small, int n_seq, int n_kv_heads, int32_t* status,
+                          cudaStream_t st);
+cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag,
+                           float* sim, int n_seq, int n_q_heads, cudaStream_t st);
+cudaError_t prepare_attention();  // one-time function attributes (dynamic shared memory sizes)
+cudaError_t prepare_select();
+size_t attention_smem_bytes();
+size_t select_smem_bytes(int keys_per_cta);
+
+}  // namespace rkv
+
+struct rkv_ctx {
+  rkv_config cfg;
+  int group;
+  int max_splits;
+  int64_t logit_stride;
+  char* workspace;
+  size_t workspace_bytes;
+  float* partials;
+  int32_t* tickets;
+  double* lse;
+  float* logits;
+  int32_t* status;
+  int64_t launches;
+  int device;
+  int sm_count;
+  std::string last_error;
+  std::unordered_map<uint64_t, CUtensorMap> tmaps;
+};

@@ -1,0 +1,160 @@
+// Small kernels of the RefreshKV decode path: small-cache rebuild (gather), cache append,
+// and the query-similarity refresh trigger (arXiv 2411.05787, Sec. 2.2).
+#include <cuda_bf16.h>
+
+#include "rkv_internal.h"
+
+namespace rkv {
+namespace {
+
+// small.K[b][g][r] = full.K[b][g][idx[b][g][r]] (and V): 16 threads move one 256-byte row as uint4.
+__global__ void __launch_bounds__(256) gather_kernel(const int32_t* __restrict__ topk_idx,
+                                                     const int32_t* __restrict__ k_small, int k_max,
+                                                     CacheDev full, CacheDev small_cache,
+                                                     const int32_t* __restrict__ active, int n_kv_heads,
+                                                     int32_t* status) {
+  const int b = blockIdx.z, g = blockIdx.y;
+  if (active != nullptr && active[b] == 0) return;
+  const int n = full.len[b];
+  int m = k_small[b];
+  if (m > k_max) m = k_max;
+  if (m > n) m = n;
+  if (m < 0) m = 0;
+  const int cap_s = small_cache.cap[b];
+  if (m > cap_s) {
+    m = cap_s;
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(status, RKV_DEV_LEN_CLAMPED);
+  }
+  if (blockIdx.x == 0 && g == 0 && threadIdx.x == 0) small_cache.len[b] = m;
+  const int cap_f = full.cap[b];
+  const int64_t src0 = full.row_offset[b] + (int64_t)g * cap_f;
+  const int64_t dst0 = small_cache.row_offset[b] + (int64_t)g * cap_s;
+  const int32_t* idx = topk_idx + (int64_t)(b * n_kv_heads + g) * k_max;
+  const uint4* fk = static_cast<const uint4*>(full.k);
+  const uint4* fv = static_cast<const uint4*>(full.v);
+  uint4* sk = static_cast<uint4*>(small_cache.k);
+  uint4* sv = static_cast<uint4*>(small_cache.v);
+  const int sub = threadIdx.x & 15;
+  for (int r = blockIdx.x * 16 + (threadIdx.x >> 4); r < m; r += gridDim.x * 16) {
+    const int j = idx[r];
+    if (j < 0) continue;
+    if (j >= n) {
+      if (sub == 0) atomicOr(status, RKV_DEV_BAD_INDEX);
+      continue;
+    }
+    const uint4 kv = __ldcs(fk + (src0 + j) * 16 + sub);
+    const uint4 vv = __ldcs(fv + (src0 + j) * 16 + sub);
+    sk[(dst0 + r) * 16 + sub] = kv;
+    sv[(dst0 + r) * 16 + sub] = vv;
+  }
+}
+
+// one block per sequence; thread t copies 16 bytes of one head's new row
+__global__ void __launch_bounds__(256) append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                                                     CacheDev full, CacheDev small_cache, int has_full,
+                                                     int has_small, int n_kv_heads, int32_t* status) {
+  const int b = blockIdx.x;
+  __shared__ int s_pos[2];
+  if (threadIdx.x < 2) {
+    const CacheDev& c = threadIdx.x == 0 ? full : small_cache;
+    const bool on = threadIdx.x == 0 ? has_full != 0 : has_small != 0;
+    int pos = -1;
+    if (on) {
+      pos = c.len[b];
+      if (pos < 0 || pos >= c.cap[b]) {
+        pos = -1;
+        atomicOr(status, RKV_DEV_APPEND_OVERFLOW);
+      }
+    }
+    s_pos[threadIdx.x] = pos;
+  }
+  __syncthreads();
+  for (int which = 0; which < 2; ++which) {
+    const int pos = s_pos[which];
+    if (pos < 0) continue;
+    const CacheDev& c = which == 0 ? full : small_cache;
+    const int cap = c.cap[b];
+    const int64_t off = c.row_offset[b];
+    uint4* ck = static_cast<uint4*>(c.k);
+    uint4* cv = static_cast<uint4*>(c.v);
+    for (int i = threadIdx.x; i < n_kv_heads * 16; i += blockDim.x) {
+      const int g = i >> 4, sub = i & 15;
+      const int64_t row = off + (int64_t)g * cap + pos;
+      ck[row * 16 + sub] = k_new[((int64_t)b * n_kv_heads + g) * 16 + sub];
+      cv[row * 16 + sub] = v_new[((int64_t)b * n_kv_heads + g) * 16 + sub];
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < 2 && s_pos[threadIdx.x] >= 0) {
+    const CacheDev& c = threadIdx.x == 0 ? full : small_cache;
+    c.len[b] = s_pos[threadIdx.x] + 1;
+  }
+}
+
+// one block of 128 threads per sequence: thread d owns channel d of the head-averaged queries
+__global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __restrict__ q_now,
+                                                      const __nv_bfloat16* __restrict__ q_last, float threshold,
+                                                      int32_t* flag, float* sim, int n_q_heads) {
+  const int b = blockIdx.x, d = threadIdx.x;
+  float a = 0.f, c = 0.f;
+  for (int h = 0; h < n_q_heads; ++h) {
+    a += __bfloat162float(q_now[((int64_t)b * n_q_heads + h) * kHeadDim + d]);
+    c += __bfloat162float(q_last[((int64_t)b * n_q_heads + h) * kHeadDim + d]);
+  }
+  const float inv = 1.f / (float)n_q_heads;
+  a *= inv;
+  c *= inv;
+  float dot = a * c, na = a * a, nc = c * c;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    na += __shfl_xor_sync(0xffffffffu, na, o);
+    nc += __shfl_xor_sync(0xffffffffu, nc, o);
+  }
+  __shared__ float red[3][4];
+  if ((d & 31) == 0) {
+    red[0][d >> 5] = dot;
+    red[1][d >> 5] = na;
+    red[2][d >> 5] = nc;
+  }
+  __syncthreads();
+  if (d == 0) {
+    const float dt = (red[0][0] + red[0][1]) + (red[0][2] + red[0][3]);
+    const float n1 = (red[1][0] + red[1][1]) + (red[1][2] + red[1][3]);
+    const float n2 = (red[2][0] + red[2][1]) + (red[2][2] + red[2][3]);
+    const float cs = dt / (sqrtf(n1) * sqrtf(n2));  // 0/0 -> NaN -> not "higher" -> refresh
+    flag[b] = (cs > threshold) ? 0 : 1;
+    if (sim != nullptr) sim[b] = cs;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
+                          CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
+                          int32_t* status, cudaStream_t st) {
+  int gx = (k_max + 15) / 16;
+  if (gx > 64) gx = 64;
+  if (gx < 1) gx = 1;
+  dim3 grid(gx, n_kv_heads, n_seq);
+  gather_kernel<<<grid, 256, 0, st>>>(topk_idx, k_small, k_max, full, small_cache, active, n_kv_heads, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, CacheDev small_cache,
+                          bool has_full, bool has_small, int n_seq, int n_kv_heads, int32_t* status,
+                          cudaStream_t st) {
+  append_kernel<<<n_seq, 128, 0, st>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), full,
+                                       small_cache, has_full ? 1 : 0, has_small ? 1 : 0, n_kv_heads, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, float* sim,
+                           int n_seq, int n_q_heads, cudaStream_t st) {
+  trigger_kernel<<<n_seq, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(q_now),
+                                        static_cast<const __nv_bfloat16*>(q_last), threshold, flag, sim,
+                                        n_q_heads);
+  return cudaGetLastError();
+}
+
+}  // namespace rkv

@@ -1,0 +1,56 @@
+"""Per-layer decode state on the GPU: both caches of a layer plus the buffers the calls write.
+
+A convenience wrapper over the C-ABI calls (rkv.Context).  It allocates device
+tensors with torch and sequences the calls of one decode step; every
+computation happens inside librkv.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import rkv
+from .synth import HEAD_DIM, LayerCache, alloc_cache
+
+
+class LayerState:
+    """C_f and C_p of one layer for a batch of sequences, and the step calls on them."""
+
+    def __init__(self, ctx: rkv.Context, full: LayerCache, k_small: list, small_extra: int, n_q_heads: int,
+                 n_kv_heads: int, want_scores: bool = False):
+        dev = full.k.device
+        self.ctx, self.full = ctx, full
+        self.n_seq, self.n_q, self.n_kv = len(k_small), n_q_heads, n_kv_heads
+        self.k_max = max(max(k_small), 1)
+        self.k_small = torch.tensor(k_small, dtype=torch.int32, device=dev)
+        self.small = alloc_cache([k + small_extra for k in k_small], [0] * self.n_seq, n_kv_heads, dev, fill=0.0)
+        self.full_c = rkv.cache_struct(full.k, full.v, full.row_offset, full.cap, full.len)
+        self.small_c = rkv.cache_struct(self.small.k, self.small.v, self.small.row_offset, self.small.cap,
+                                        self.small.len)
+        self.out = torch.zeros((self.n_seq, n_q_heads, HEAD_DIM), dtype=torch.bfloat16, device=dev)
+        self.topk_idx = torch.full((self.n_seq, n_kv_heads, self.k_max), -2, dtype=torch.int32, device=dev)
+        self.q_last_full = torch.zeros((self.n_seq, n_q_heads, HEAD_DIM), dtype=torch.bfloat16, device=dev)
+        self.flag = torch.zeros((self.n_seq,), dtype=torch.int32, device=dev)
+        self.not_flag = torch.zeros((self.n_seq,), dtype=torch.int32, device=dev)
+        self.sim = torch.zeros((self.n_seq,), dtype=torch.float32, device=dev)
+        self.scores = None
+        if want_scores:
+            stride = int(full.cap.max().item())
+            self.scores = torch.zeros((self.n_seq, n_kv_heads, stride), dtype=torch.float32, device=dev)
+
+    def refresh(self, q, active=None, max_len_hint=0):
+        """Full step followed by the rebuild of the small cache."""
+        self.ctx.full_step(q, self.full_c, self.k_small, self.k_max, self.out, self.topk_idx, active=active,
+                           scores=self.scores, q_last_full=self.q_last_full, max_len_hint=max_len_hint)
+        self.ctx.gather_small(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c, active=active)
+        return self.out
+
+    def partial(self, q, active=None, max_len_hint=0):
+        self.ctx.small_step(q, self.small_c, self.out, active=active, max_len_hint=max_len_hint)
+        return self.out
+
+    def append(self, k_new, v_new):
+        self.ctx.append(k_new, v_new, self.full_c, self.small_c)
+
+    def check_trigger(self, q, threshold):
+        self.ctx.should_refresh(q, self.q_last_full, threshold, self.flag, self.sim)
+        return self.flag
