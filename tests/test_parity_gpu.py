@@ -397,7 +397,7 @@ def test_config1_planted_positions_are_selected(mods):
     cache = synth.fill_layer(w, 0, dev)
     qs = synth.query_trajectory(w, 0).to(dev)
     synth.plant_heavy(w, cache, 0, qs[0])
-    ctx = rkv.Context(1, 32, 8, 2048 + 32, 256 + 32)
+    ctx = rkv.Context(1, 32, 8, int(cache.cap.max()), 256 + 32)
     st = runner.LayerState(ctx, cache, [256], 32, 32, 8, want_scores=True)
     st.refresh(qs[0])
     heavy = synth.heavy_positions(w, 0, 0, 0, 2048, "cpu").numpy()
