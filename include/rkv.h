@@ -179,6 +179,23 @@ const char* rkv_last_cuda_error(const rkv_ctx* ctx);
  * above launches a fixed, documented number; used by benchmarks to report it). */
 int64_t rkv_launch_count(const rkv_ctx* ctx);
 
+/*
+ * Optional per-kernel timing (no counterpart in the paper, which reports wall-clock decode time
+ * only).  While profiling is on, every kernel launch is bracketed by CUDA events on the caller's
+ * stream; rkv_get_profile waits for them, adds up the elapsed device time per kernel kind, returns
+ * the sums and the launch counts and forgets the samples.  Do not enable it during stream capture.
+ *   total_us, launches   host arrays of RKV_KERNEL_KINDS entries
+ */
+#define RKV_KERNEL_ATTN_FULL 0  /* full-cache attention + logit emission (rkv_full_step, 1st kernel) */
+#define RKV_KERNEL_SELECT 1     /* score finalisation + top-K            (rkv_full_step, 2nd kernel) */
+#define RKV_KERNEL_ATTN_SMALL 2 /* small-cache attention                 (rkv_small_step)            */
+#define RKV_KERNEL_GATHER 3     /* rkv_gather_small                                                  */
+#define RKV_KERNEL_APPEND 4     /* rkv_append                                                        */
+#define RKV_KERNEL_TRIGGER 5    /* rkv_should_refresh                                                */
+#define RKV_KERNEL_KINDS 6
+rkv_status rkv_set_profiling(rkv_ctx* ctx, int32_t on);
+rkv_status rkv_get_profile(rkv_ctx* ctx, double* total_us /*host*/, int64_t* launches /*host*/);
+
 #ifdef __cplusplus
 }
 #endif

@@ -64,6 +64,26 @@ bool cache_ok(const rkv_cache* c) {
          (reinterpret_cast<uintptr_t>(c->k) & 15) == 0 && (reinterpret_cast<uintptr_t>(c->v) & 15) == 0;
 }
 
+// Brackets one kernel launch with events when profiling is on.
+struct LaunchScope {
+  rkv_ctx* ctx; cudaStream_t st; int kind; cudaEvent_t stop = nullptr;
+  static cudaEvent_t get(rkv_ctx* c) {
+    cudaEvent_t e = nullptr;
+    if (!c->event_pool.empty()) { e = c->event_pool.back(); c->event_pool.pop_back(); return e; }
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    return e;
+  }
+  LaunchScope(rkv_ctx* c, cudaStream_t s, int k) : ctx(c), st(s), kind(k) {
+    if (!ctx->profiling) return;
+    cudaEvent_t start = get(ctx);
+    stop = get(ctx);
+    if (start == nullptr || stop == nullptr) { stop = nullptr; return; }
+    cudaEventRecord(start, st);
+    ctx->timed.push_back({kind, start, stop});
+  }
+  ~LaunchScope() { if (stop != nullptr) cudaEventRecord(stop, st); }
+};
+
 CacheDev dev_of(const rkv_cache* c) { return CacheDev{c->k, c->v, c->row_offset, c->cap, c->len}; }
 
 // 2-D view [n_rows][128] bf16, box = 64 rows x 64 channels (128 bytes), 128-byte swizzle
@@ -148,7 +168,11 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.max_splits = ctx->max_splits;
   p.max_len = limit;
   p.scale = ctx->cfg.softmax_scale;
-  cudaError_t e = rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
+  cudaError_t e;
+  {
+    LaunchScope scope(ctx, st, logits ? RKV_KERNEL_ATTN_FULL : RKV_KERNEL_ATTN_SMALL);
+    e = rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
   ctx->launches += 1;
   return RKV_OK;
@@ -176,6 +200,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
   ctx->max_splits = splits_for(cfg);
   ctx->launches = 0;
+  ctx->profiling = false;
   ctx->workspace = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -206,6 +231,8 @@ rkv_status rkv_destroy(rkv_ctx* ctx) {
   if (ctx == nullptr) return RKV_ERR_INVALID_ARG;
   cudaError_t e = cudaSuccess;
   if (ctx->workspace) e = cudaFree(ctx->workspace);
+  for (auto& t : ctx->timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
+  for (auto ev : ctx->event_pool) cudaEventDestroy(ev);
   delete ctx;
   return e == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
@@ -241,7 +268,11 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, con
   sp.max_len = n_max;
   int per = (n_max + rkv::kSelectCluster - 1) / rkv::kSelectCluster;
   sp.keys_per_cta = (per + 3) & ~3;
-  cudaError_t e = rkv::launch_select(sp, ctx->cfg.n_seq, st);
+  cudaError_t e;
+  {
+    LaunchScope scope(ctx, st, RKV_KERNEL_SELECT);
+    e = rkv::launch_select(sp, ctx->cfg.n_seq, st);
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
   ctx->launches += 1;
   return RKV_OK;
@@ -252,9 +283,12 @@ rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t
                             void* stream) {
   if (!ctx || !topk_idx || !k_small || !cache_ok(full) || !cache_ok(small_cache)) return RKV_ERR_INVALID_ARG;
   if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
-  cudaError_t e = rkv::launch_gather(topk_idx, k_small, k_max, dev_of(full), dev_of(small_cache), active,
-                                     ctx->cfg.n_seq, ctx->cfg.n_kv_heads, ctx->status,
-                                     static_cast<cudaStream_t>(stream));
+  cudaError_t e;
+  {
+    LaunchScope scope(ctx, static_cast<cudaStream_t>(stream), RKV_KERNEL_GATHER);
+    e = rkv::launch_gather(topk_idx, k_small, k_max, dev_of(full), dev_of(small_cache), active, ctx->cfg.n_seq,
+                           ctx->cfg.n_kv_heads, ctx->status, static_cast<cudaStream_t>(stream));
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "gather launch");
   ctx->launches += 1;
   return RKV_OK;
@@ -274,9 +308,13 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const 
   if (!ctx || !k_new || !v_new || (full == nullptr && small_cache == nullptr)) return RKV_ERR_INVALID_ARG;
   if ((full && !cache_ok(full)) || (small_cache && !cache_ok(small_cache))) return RKV_ERR_INVALID_ARG;
   CacheDev none = {nullptr, nullptr, nullptr, nullptr, nullptr};
-  cudaError_t e = rkv::launch_append(k_new, v_new, full ? dev_of(full) : none, small_cache ? dev_of(small_cache) : none,
-                                     full != nullptr, small_cache != nullptr, ctx->cfg.n_seq, ctx->cfg.n_kv_heads,
-                                     ctx->status, static_cast<cudaStream_t>(stream));
+  cudaError_t e;
+  {
+    LaunchScope scope(ctx, static_cast<cudaStream_t>(stream), RKV_KERNEL_APPEND);
+    e = rkv::launch_append(k_new, v_new, full ? dev_of(full) : none, small_cache ? dev_of(small_cache) : none,
+                           full != nullptr, small_cache != nullptr, ctx->cfg.n_seq, ctx->cfg.n_kv_heads, ctx->status,
+                           static_cast<cudaStream_t>(stream));
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "append launch");
   ctx->launches += 1;
   return RKV_OK;
@@ -285,8 +323,12 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const 
 rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_last_full, float threshold,
                               int32_t* flag, float* sim, void* stream) {
   if (!ctx || !q_now || !q_last_full || !flag) return RKV_ERR_INVALID_ARG;
-  cudaError_t e = rkv::launch_trigger(q_now, q_last_full, threshold, flag, sim, ctx->cfg.n_seq, ctx->cfg.n_q_heads,
-                                      static_cast<cudaStream_t>(stream));
+  cudaError_t e;
+  {
+    LaunchScope scope(ctx, static_cast<cudaStream_t>(stream), RKV_KERNEL_TRIGGER);
+    e = rkv::launch_trigger(q_now, q_last_full, threshold, flag, sim, ctx->cfg.n_seq, ctx->cfg.n_q_heads,
+                            static_cast<cudaStream_t>(stream));
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "trigger launch");
   ctx->launches += 1;
   return RKV_OK;
@@ -319,5 +361,28 @@ const char* rkv_status_string(rkv_status s) {
 const char* rkv_last_cuda_error(const rkv_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
 
 int64_t rkv_launch_count(const rkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+rkv_status rkv_set_profiling(rkv_ctx* ctx, int32_t on) {
+  if (!ctx) return RKV_ERR_INVALID_ARG;
+  ctx->profiling = on != 0;
+  return RKV_OK;
+}
+
+rkv_status rkv_get_profile(rkv_ctx* ctx, double* total_us, int64_t* launches) {
+  if (!ctx || !total_us || !launches) return RKV_ERR_INVALID_ARG;
+  for (int i = 0; i < RKV_KERNEL_KINDS; ++i) { total_us[i] = 0.0; launches[i] = 0; }
+  for (auto& t : ctx->timed) {
+    cudaError_t e = cudaEventSynchronize(t.stop);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, t.start, t.stop);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "profile read");
+    total_us[t.kind] += 1000.0 * ms;
+    launches[t.kind] += 1;
+    ctx->event_pool.push_back(t.start);
+    ctx->event_pool.push_back(t.stop);
+  }
+  ctx->timed.clear();
+  return RKV_OK;
+}
 
 }  // extern "C"

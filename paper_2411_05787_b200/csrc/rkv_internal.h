@@ -6,6 +6,7 @@
 
 #include <string>
 #include <unordered_map>
+#include <vector>
 
 #include "rkv.h"
 
@@ -103,4 +104,9 @@ struct rkv_ctx {
   int sm_count;
   std::string last_error;
   std::unordered_map<uint64_t, CUtensorMap> tmaps;
+  // optional per-kernel timing (rkv_set_profiling): event pairs recorded around every launch
+  bool profiling;
+  struct Timed { int kind; cudaEvent_t start, stop; };
+  std::vector<Timed> timed;
+  std::vector<cudaEvent_t> event_pool;
 };

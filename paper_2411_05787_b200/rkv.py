@@ -20,7 +20,8 @@ DEV_APPEND_OVERFLOW, DEV_LEN_CLAMPED, DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT 
 
 EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", "rkv_gather_small",
            "rkv_small_step", "rkv_append", "rkv_should_refresh", "rkv_get_device_status",
-           "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count"]
+           "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile"]
+KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
 
 
 class RkvConfig(ctypes.Structure):
@@ -57,6 +58,10 @@ def _load() -> ctypes.CDLL:
     lib.rkv_last_cuda_error.restype = ctypes.c_char_p
     lib.rkv_launch_count.argtypes = [vp]
     lib.rkv_launch_count.restype = i64
+    lib.rkv_set_profiling.argtypes = [vp, i32]
+    lib.rkv_set_profiling.restype = i32
+    lib.rkv_get_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
+    lib.rkv_get_profile.restype = i32
     for name in ("rkv_create", "rkv_destroy", "rkv_full_step", "rkv_gather_small", "rkv_small_step",
                  "rkv_append", "rkv_should_refresh", "rkv_get_device_status"):
         getattr(lib, name).restype = i32
@@ -155,6 +160,16 @@ class Context:
     def should_refresh(self, q_now, q_last_full, threshold, flag, sim=None, stream=None):
         self._check(lib.rkv_should_refresh(self._h, _ptr(q_now), _ptr(q_last_full), float(threshold), _ptr(flag),
                                            _ptr(sim), _stream(stream)))
+
+    def set_profiling(self, on: bool):
+        self._check(lib.rkv_set_profiling(self._h, 1 if on else 0))
+
+    def get_profile(self) -> dict:
+        """{kernel name: (total microseconds, launches)} since the last call; waits for the recorded events."""
+        us = (ctypes.c_double * len(KERNEL_NAMES))()
+        cnt = (ctypes.c_int64 * len(KERNEL_NAMES))()
+        self._check(lib.rkv_get_profile(self._h, us, cnt))
+        return {n: (us[i], cnt[i]) for i, n in enumerate(KERNEL_NAMES)}
 
     def device_status(self, stream=None) -> int:
         """Synchronises the stream; returns and clears the sticky device status bits."""
