@@ -36,7 +36,7 @@ int splits_for(const rkv_config* c) {
   return s < rkv::kMaxSplits ? (s < 1 ? 1 : s) : rkv::kMaxSplits;
 }
 
-struct WsLayout { size_t partials, tickets, lse, logits, status, total; int64_t logit_stride; };
+struct WsLayout { size_t partials, tickets, logits, status, total; int64_t logit_stride; };
 
 WsLayout ws_layout(const rkv_config* c) {
   WsLayout w;
@@ -47,7 +47,6 @@ WsLayout ws_layout(const rkv_config* c) {
   size_t off = 0;
   w.partials = off; off = up(off + bg * splits_for(c) * rkv::PartialLayout::kFloats * sizeof(float));
   w.tickets = off;  off = up(off + bg * sizeof(int32_t));
-  w.lse = off;      off = up(off + (size_t)c->n_seq * c->n_q_heads * sizeof(double));
   w.logits = off;   off = up(off + bg * group * (size_t)w.logit_stride * sizeof(float));
   w.status = off;   off = up(off + sizeof(int32_t));
   w.total = off;
@@ -117,9 +116,11 @@ rkv_status tensor_map(rkv_ctx* ctx, void* base, int64_t n_rows, CUtensorMap* out
   return RKV_OK;
 }
 
-// positions per CTA: one balanced wave over 2 CTAs per SM when that keeps chunks moderate,
-// otherwise fixed 2048-position chunks over several waves (ragged batches balance by count)
-int choose_chunk(const rkv_ctx* ctx, int n_max, int* grid_x) {
+// Positions per CTA.  Full step: one balanced wave over 2 CTAs per SM when that keeps chunks moderate,
+// otherwise fixed 2048-position chunks over several waves (ragged batches then balance by count).
+// Small step: the work is tiny and latency-bound, so chunks of at least 256 positions keep the
+// number of partials that the last CTA has to fold small.
+int choose_chunk(const rkv_ctx* ctx, int n_max, bool full, int* grid_x) {
   const int bg = ctx->cfg.n_seq * ctx->cfg.n_kv_heads;
   const int slots = 2 * ctx->sm_count;
   int splits = slots / bg;
@@ -127,7 +128,8 @@ int choose_chunk(const rkv_ctx* ctx, int n_max, int* grid_x) {
   if (splits > ctx->max_splits) splits = ctx->max_splits;
   int chunk = (n_max + splits - 1) / splits;
   if (chunk > 4096) chunk = 2048;
-  if (chunk < rkv::kTile) chunk = rkv::kTile;
+  const int floor_chunk = full ? rkv::kTile : ctx->small_min_chunk;
+  if (chunk < floor_chunk) chunk = floor_chunk;
   chunk = (chunk + 15) & ~15;
   int gx = (n_max + chunk - 1) / chunk;
   while (gx > ctx->max_splits) {  // keep the partial buffer's bound
@@ -139,7 +141,7 @@ int choose_chunk(const rkv_ctx* ctx, int n_max, int* grid_x) {
 }
 
 rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
-                         void* q_last_full, int n_max, int limit, bool logits, cudaStream_t st) {
+                         int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out) {
   CUtensorMap tm_k, tm_v;
   rkv_status s = tensor_map(ctx, cache->k, cache->n_rows, &tm_k);
   if (s != RKV_OK) return s;
@@ -148,7 +150,8 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   AttnParams p;
   memset(&p, 0, sizeof(p));
   int gx = 1;
-  p.chunk = choose_chunk(ctx, n_max, &gx);
+  p.chunk = choose_chunk(ctx, n_max, logits, &gx);
+  if (chunk_out) *chunk_out = p.chunk;
   p.q = q;
   p.row_offset = cache->row_offset;
   p.cap = cache->cap;
@@ -157,9 +160,7 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.out = out;
   p.partials = ctx->partials;
   p.tickets = ctx->tickets;
-  p.lse = ctx->lse;
   p.logits = logits ? ctx->logits : nullptr;
-  p.q_last_full = q_last_full;
   p.status = ctx->status;
   p.logit_stride = ctx->logit_stride;
   p.n_q_heads = ctx->cfg.n_q_heads;
@@ -201,6 +202,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->max_splits = splits_for(cfg);
   ctx->launches = 0;
   ctx->profiling = false;
+  ctx->small_min_chunk = 256;
   ctx->workspace = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -219,7 +221,6 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->workspace_bytes = w.total;
   ctx->partials = reinterpret_cast<float*>(ctx->workspace + w.partials);
   ctx->tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.tickets);
-  ctx->lse = reinterpret_cast<double*>(ctx->workspace + w.lse);
   ctx->logits = reinterpret_cast<float*>(ctx->workspace + w.logits);
   ctx->status = reinterpret_cast<int32_t*>(ctx->workspace + w.status);
   ctx->logit_stride = w.logit_stride;
@@ -246,12 +247,19 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, con
   if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
   if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  rkv_status s = run_attention(ctx, q, full, active, out, q_last_full, n_max, n_max, true, st);
+  int chunk = 0;
+  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk);
   if (s != RKV_OK) return s;
   SelectParams sp;
   memset(&sp, 0, sizeof(sp));
   sp.logits = ctx->logits;
-  sp.lse = ctx->lse;
+  sp.partials = ctx->partials;
+  sp.q = q;
+  sp.out = out;
+  sp.q_last_full = q_last_full;
+  sp.cap = full->cap;
+  sp.chunk = chunk;
+  sp.max_splits = ctx->max_splits;
   sp.len = full->len;
   sp.k_small = k_small;
   sp.active = active;
@@ -299,8 +307,8 @@ rkv_status rkv_small_step(rkv_ctx* ctx, const void* q, const rkv_cache* small_ca
   if (!ctx || !q || !cache_ok(small_cache) || !out) return RKV_ERR_INVALID_ARG;
   int n_max = max_len_hint == 0 ? ctx->cfg.max_small : max_len_hint;
   if (n_max < 1 || n_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
-  return run_attention(ctx, q, small_cache, active, out, nullptr, n_max, n_max, false,
-                       static_cast<cudaStream_t>(stream));
+  return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, static_cast<cudaStream_t>(stream),
+                       nullptr);
 }
 
 rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const rkv_cache* full,

@@ -19,6 +19,7 @@
 // spinning).
 #include <cuda_bf16.h>
 
+#include "rkv_fold.cuh"
 #include "rkv_internal.h"
 
 namespace rkv {
@@ -340,12 +341,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   }
 
   const int bg = b * p.n_kv_heads + g;
-  if (n_splits > 1) {
+  const bool single = (!kLogits) && n_splits == 1;   // the full step always leaves its partials to the selector
+  if (!single) {
     float* part = p.partials + ((int64_t)bg * p.max_splits + split) * PartialLayout::kFloats;
 #pragma unroll
     for (int h = 0; h < kMaxGroup; ++h)
       if (h < G) part[h * kHeadDim + d] = accO[h];
-    if (d < G) {
+    if (d < kMaxGroup) {
       float Md = ninf, Ld = 0.f;
 #pragma unroll
       for (int h = 0; h < kMaxGroup; ++h)
@@ -356,6 +358,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       part[kMaxGroup * kHeadDim + d] = Md;
       part[kMaxGroup * kHeadDim + kMaxGroup + d] = Ld;
     }
+    if (kLogits) return;   // full step: the selection kernel folds the partials (in parallel, per head)
     __threadfence();
     consumer_bar();
     if (tid == 0) {
@@ -367,23 +370,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     __threadfence();
     // last CTA of this (sequence, KV head): fold all split partials
     const float* pbase = p.partials + (int64_t)bg * p.max_splits * PartialLayout::kFloats;
+    float* sm_red = reinterpret_cast<float*>(smem_gen);                 // [4][8][128]
+    float* sm_w = sm_red + 4 * kMaxGroup * kHeadDim;                    // [n_splits][16]
+    float* sm_ML = sm_w + kMaxSplits * 16;                              // [16]
+    auto bar = [] { consumer_bar(); };
+    fold_weights<128>(pbase, n_splits, tid, sm_w, sm_ML, bar);
+    fold_out<128, kMaxGroup>(pbase, n_splits, 0, G, tid, sm_w, sm_red, bar);
 #pragma unroll
     for (int h = 0; h < kMaxGroup; ++h) {
       if (h < G) {
-        float M = ninf;
-        for (int sidx = 0; sidx < n_splits; ++sidx)
-          M = fmaxf(M, __ldcg(pbase + (int64_t)sidx * PartialLayout::kFloats + kMaxGroup * kHeadDim + h));
-        float L = 0.f, O = 0.f;
-        for (int sidx = 0; sidx < n_splits; ++sidx) {
-          const float* ps = pbase + (int64_t)sidx * PartialLayout::kFloats;
-          const float ms = __ldcg(ps + kMaxGroup * kHeadDim + h);
-          const float e = (ms == ninf) ? 0.f : ex2((ms - M) * kLog2e);
-          L += __ldcg(ps + kMaxGroup * kHeadDim + kMaxGroup + h) * e;
-          O += __ldcg(ps + h * kHeadDim + d) * e;
-        }
-        accO[h] = O;
-        accM[h] = M;
-        accL[h] = L;
+        accO[h] = sm_red[h * kHeadDim + d];
+        accL[h] = sm_ML[8 + h];
       }
     }
     if (tid == 0) p.tickets[bg] = 0;  // ready for the next call on this stream
@@ -391,17 +388,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
 
   if (!ok) return;
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) {
-    if (h < G) {
-      out[h * kHeadDim + d] = __float2bfloat16(accO[h] / accL[h]);
-      if (d == 0) p.lse[(int64_t)b * p.n_q_heads + g * G + h] = (double)accM[h] + log((double)accL[h]);
-    }
-  }
-  if (p.q_last_full != nullptr) {
-    __nv_bfloat16* ql =
-        static_cast<__nv_bfloat16*>(p.q_last_full) + ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
-    for (int h = 0; h < G; ++h) ql[h * kHeadDim + d] = qg[h * kHeadDim + d];
-  }
+  for (int h = 0; h < kMaxGroup; ++h)
+    if (h < G) out[h * kHeadDim + d] = __float2bfloat16(accO[h] / accL[h]);
 }
 
 }  // namespace

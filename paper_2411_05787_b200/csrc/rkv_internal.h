@@ -19,7 +19,7 @@ constexpr int kTile = 64;              // positions per pipeline stage
 constexpr int kStages = 3;
 constexpr int kAttnThreads = 160;      // 4 MMA warps + 1 copy warp
 constexpr int kSelectCluster = 8;      // CTAs that share one top-K problem
-constexpr int kSelectThreads = 256;
+constexpr int kSelectThreads = 512;
 constexpr int kSelectMaxKeysPerCta = 40960;
 constexpr int kDevTimeoutBit = 16;     // internal: a bounded barrier wait ran out
 
@@ -37,9 +37,7 @@ struct AttnParams {
   void* out;                  // bf16 [B][Hq][128]
   float* partials;            // [B*Hkv][max_splits][PartialLayout::kFloats]
   int32_t* tickets;           // [B*Hkv]
-  double* lse;                // [B][Hq]   (log-sum-exp of the scaled logits)
   float* logits;              // [B*Hkv][G][logit_stride] or null
-  void* q_last_full;          // bf16 [B][Hq][128] or null
   int32_t* status;
   int64_t logit_stride;
   int32_t n_q_heads, n_kv_heads, group;
@@ -51,7 +49,11 @@ struct AttnParams {
 
 struct SelectParams {
   const float* logits;        // [B*Hkv][G][logit_stride]
-  const double* lse;          // [B][Hq]
+  const float* partials;      // split partials written by the attention kernel
+  const void* q;              // bf16 [B][Hq][128]
+  void* out;                  // bf16 [B][Hq][128]
+  void* q_last_full;          // bf16 [B][Hq][128] or null
+  const int32_t* cap;
   const int32_t* len;
   const int32_t* k_small;     // [B]
   const int32_t* active;
@@ -62,6 +64,7 @@ struct SelectParams {
   int32_t n_q_heads, n_kv_heads, group, agg;
   int32_t k_max, max_len;
   int32_t keys_per_cta;       // capacity of the shared-memory key array
+  int32_t chunk, max_splits;  // split geometry of the attention launch that produced the partials
 };
 
 struct CacheDev {
@@ -96,12 +99,12 @@ struct rkv_ctx {
   size_t workspace_bytes;
   float* partials;
   int32_t* tickets;
-  double* lse;
   float* logits;
   int32_t* status;
   int64_t launches;
   int device;
   int sm_count;
+  int small_min_chunk;
   std::string last_error;
   std::unordered_map<uint64_t, CUtensorMap> tmaps;
   // optional per-kernel timing (rkv_set_profiling): event pairs recorded around every launch
