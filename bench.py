@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--ctx", type=int, default=32768)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--small-min-chunk", type=int, default=0, help="override rkv_small_step chunking (0: library default)")
+    ap.add_argument("--no-dependent-launch", action="store_true", help="plain stream order between kernels")
     return ap.parse_args()
 
 
@@ -205,6 +207,10 @@ def run_ours(args):
     L, K, Hq, Hkv = w.lens[0], w.k_small[0], w.n_q_heads, w.n_kv_heads
     max_len = L + total_tokens + 1
     ctx = rkv.Context(1, Hq, Hkv, max_len, K + STRIDE + 2)
+    if args.small_min_chunk:
+        ctx.set_option(rkv.OPT_SMALL_MIN_CHUNK, args.small_min_chunk)
+    if args.no_dependent_launch:
+        ctx.set_option(rkv.OPT_DEPENDENT_LAUNCH, 0)
 
     layers = []
     q0 = synth.query_trajectory(synth.scaled(w, steps=1), 0).to(dev)

@@ -180,6 +180,18 @@ const char* rkv_last_cuda_error(const rkv_ctx* ctx);
 int64_t rkv_launch_count(const rkv_ctx* ctx);
 
 /*
+ * Launch-geometry knobs (no counterpart in the paper).  Results never depend on them beyond
+ * floating-point summation order.
+ *   RKV_OPT_SMALL_MIN_CHUNK   positions per CTA (at least) in rkv_small_step; default 256, >= 64
+ *   RKV_OPT_DEPENDENT_LAUNCH  1 (default): kernels are launched with programmatic stream
+ *                             serialisation so that a kernel's launch overlaps the tail of its
+ *                             predecessor; 0: plain stream order.  Process-wide.
+ */
+#define RKV_OPT_SMALL_MIN_CHUNK 1
+#define RKV_OPT_DEPENDENT_LAUNCH 2
+rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
+
+/*
  * Optional per-kernel timing (no counterpart in the paper, which reports wall-clock decode time
  * only).  While profiling is on, every kernel launch is bracketed by CUDA events on the caller's
  * stream; rkv_get_profile waits for them, adds up the elapsed device time per kernel kind, returns

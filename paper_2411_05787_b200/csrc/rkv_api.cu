@@ -181,6 +181,10 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
 
 }  // namespace
 
+namespace rkv {
+bool g_use_pdl = true;
+}
+
 extern "C" {
 
 size_t rkv_workspace_bytes(const rkv_config* cfg) {
@@ -369,6 +373,21 @@ const char* rkv_status_string(rkv_status s) {
 const char* rkv_last_cuda_error(const rkv_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
 
 int64_t rkv_launch_count(const rkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value) {
+  if (!ctx) return RKV_ERR_INVALID_ARG;
+  switch (option) {
+    case RKV_OPT_SMALL_MIN_CHUNK:
+      if (value < rkv::kTile || value > (1 << 20)) return RKV_ERR_INVALID_ARG;
+      ctx->small_min_chunk = value;
+      return RKV_OK;
+    case RKV_OPT_DEPENDENT_LAUNCH:
+      rkv::g_use_pdl = value != 0;
+      return RKV_OK;
+    default:
+      return RKV_ERR_INVALID_ARG;
+  }
+}
 
 rkv_status rkv_set_profiling(rkv_ctx* ctx, int32_t on) {
   if (!ctx) return RKV_ERR_INVALID_ARG;

@@ -109,8 +109,22 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   __shared__ int s_last;
 
   const int b = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
-  if (p.active != nullptr && p.active[b] == 0) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  pdl_launch();
+  // shared memory: [stages][K lo | K hi | V lo | V hi], then the barriers
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_full = smem_base + kStages * kStageBytes;
+  const uint32_t bar_empty = bar_full + 8 * kStages;
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  pdl_wait();   // nothing above reads global memory
+  if (p.active != nullptr && p.active[b] == 0) return;
   const int G = p.group;
   const int cap = p.cap[b];
   int n = p.len[b];
@@ -137,20 +151,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   const int n_splits = (n + p.chunk - 1) / p.chunk;
   const int64_t row0 = p.row_offset[b] + (int64_t)g * cap + start;
 
-  // shared memory: [stages][K lo | K hi | V lo | V hi], then the barriers
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_full = smem_base + kStages * kStageBytes;
-  const uint32_t bar_empty = bar_full + 8 * kStages;
-
-  if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, 4);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
+  __syncthreads();   // barrier initialisation (above) is visible to every warp
 
   if (warp == 4) {
     // ------------------------------------------------------------ copy warp
@@ -408,10 +409,8 @@ cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const
                              int n_seq, int grid_x, bool write_logits, cudaStream_t st) {
   dim3 grid(grid_x, p.n_kv_heads, n_seq);
   if (write_logits)
-    attn_kernel<true><<<grid, kAttnThreads, attention_smem_bytes(), st>>>(tm_k, tm_v, p);
-  else
-    attn_kernel<false><<<grid, kAttnThreads, attention_smem_bytes(), st>>>(tm_k, tm_v, p);
-  return cudaGetLastError();
+    return launch_ex(attn_kernel<true>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
+  return launch_ex(attn_kernel<false>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
 }
 
 }  // namespace rkv

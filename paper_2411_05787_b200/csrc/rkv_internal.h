@@ -83,6 +83,44 @@ cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, C
                           cudaStream_t st);
 cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag,
                            float* sim, int n_seq, int n_q_heads, cudaStream_t st);
+// Launch with optional programmatic dependent launch (the kernel may start while its predecessor on
+// the stream drains; every kernel waits with pdl_wait() before touching global memory) and an
+// optional thread-block cluster along x.
+extern bool g_use_pdl;
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             int cluster_x, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (g_use_pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+#ifdef __CUDACC__
+// Programmatic dependent launch: let the next kernel on the stream begin its launch now / wait until
+// everything the previous kernel wrote is visible.  Both are no-ops without the launch attribute.
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 cudaError_t prepare_attention();  // one-time function attributes (dynamic shared memory sizes)
 cudaError_t prepare_select();
 size_t attention_smem_bytes();

@@ -14,6 +14,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const int32_t* __restrict__
                                                      const int32_t* __restrict__ active, int n_kv_heads,
                                                      int32_t* status) {
   const int b = blockIdx.z, g = blockIdx.y;
+  pdl_launch();
+  pdl_wait();
   if (active != nullptr && active[b] == 0) return;
   const int n = full.len[b];
   int m = k_small[b];
@@ -49,45 +51,48 @@ __global__ void __launch_bounds__(256) gather_kernel(const int32_t* __restrict__
   }
 }
 
-// one block per sequence; thread t copies 16 bytes of one head's new row
-__global__ void __launch_bounds__(256) append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+// One block per sequence; thread t moves 16 bytes of one head's new K row and V row.  Every load is
+// issued before the first dependent use, so the kernel costs one memory round trip.
+__global__ void __launch_bounds__(128) append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                                                      CacheDev full, CacheDev small_cache, int has_full,
                                                      int has_small, int n_kv_heads, int32_t* status) {
-  const int b = blockIdx.x;
-  __shared__ int s_pos[2];
-  if (threadIdx.x < 2) {
-    const CacheDev& c = threadIdx.x == 0 ? full : small_cache;
-    const bool on = threadIdx.x == 0 ? has_full != 0 : has_small != 0;
-    int pos = -1;
-    if (on) {
-      pos = c.len[b];
-      if (pos < 0 || pos >= c.cap[b]) {
-        pos = -1;
-        atomicOr(status, RKV_DEV_APPEND_OVERFLOW);
-      }
-    }
-    s_pos[threadIdx.x] = pos;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  pdl_launch();
+  pdl_wait();
+  int pos_f = -1, cap_f = 0, pos_s = -1, cap_s = 0;
+  int64_t off_f = 0, off_s = 0;
+  if (has_full) {
+    pos_f = full.len[b];
+    cap_f = full.cap[b];
+    off_f = full.row_offset[b];
   }
-  __syncthreads();
-  for (int which = 0; which < 2; ++which) {
-    const int pos = s_pos[which];
-    if (pos < 0) continue;
-    const CacheDev& c = which == 0 ? full : small_cache;
-    const int cap = c.cap[b];
-    const int64_t off = c.row_offset[b];
-    uint4* ck = static_cast<uint4*>(c.k);
-    uint4* cv = static_cast<uint4*>(c.v);
-    for (int i = threadIdx.x; i < n_kv_heads * 16; i += blockDim.x) {
-      const int g = i >> 4, sub = i & 15;
-      const int64_t row = off + (int64_t)g * cap + pos;
-      ck[row * 16 + sub] = k_new[((int64_t)b * n_kv_heads + g) * 16 + sub];
-      cv[row * 16 + sub] = v_new[((int64_t)b * n_kv_heads + g) * 16 + sub];
+  if (has_small) {
+    pos_s = small_cache.len[b];
+    cap_s = small_cache.cap[b];
+    off_s = small_cache.row_offset[b];
+  }
+  const bool ok_f = has_full && pos_f >= 0 && pos_f < cap_f;
+  const bool ok_s = has_small && pos_s >= 0 && pos_s < cap_s;
+  for (int i = tid; i < n_kv_heads * 16; i += blockDim.x) {
+    const int g = i >> 4, sub = i & 15;
+    const uint4 kv = k_new[((int64_t)b * n_kv_heads + g) * 16 + sub];
+    const uint4 vv = v_new[((int64_t)b * n_kv_heads + g) * 16 + sub];
+    if (ok_f) {
+      const int64_t row = off_f + (int64_t)g * cap_f + pos_f;
+      static_cast<uint4*>(full.k)[row * 16 + sub] = kv;
+      static_cast<uint4*>(full.v)[row * 16 + sub] = vv;
+    }
+    if (ok_s) {
+      const int64_t row = off_s + (int64_t)g * cap_s + pos_s;
+      static_cast<uint4*>(small_cache.k)[row * 16 + sub] = kv;
+      static_cast<uint4*>(small_cache.v)[row * 16 + sub] = vv;
     }
   }
-  __syncthreads();
-  if (threadIdx.x < 2 && s_pos[threadIdx.x] >= 0) {
-    const CacheDev& c = threadIdx.x == 0 ? full : small_cache;
-    c.len[b] = s_pos[threadIdx.x] + 1;
+  __syncthreads();   // every thread has read the old lengths
+  if (tid == 0) {
+    if (ok_f) full.len[b] = pos_f + 1;
+    if (ok_s) small_cache.len[b] = pos_s + 1;
+    if ((has_full && !ok_f) || (has_small && !ok_s)) atomicOr(status, RKV_DEV_APPEND_OVERFLOW);
   }
 }
 
@@ -96,6 +101,8 @@ __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __res
                                                       const __nv_bfloat16* __restrict__ q_last, float threshold,
                                                       int32_t* flag, float* sim, int n_q_heads) {
   const int b = blockIdx.x, d = threadIdx.x;
+  pdl_launch();
+  pdl_wait();
   float a = 0.f, c = 0.f;
   for (int h = 0; h < n_q_heads; ++h) {
     a += __bfloat162float(q_now[((int64_t)b * n_q_heads + h) * kHeadDim + d]);
@@ -137,24 +144,22 @@ cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k
   if (gx > 64) gx = 64;
   if (gx < 1) gx = 1;
   dim3 grid(gx, n_kv_heads, n_seq);
-  gather_kernel<<<grid, 256, 0, st>>>(topk_idx, k_small, k_max, full, small_cache, active, n_kv_heads, status);
-  return cudaGetLastError();
+  return launch_ex(gather_kernel, grid, dim3(256), 0, st, 1, topk_idx, k_small, k_max, full, small_cache, active,
+                   n_kv_heads, status);
 }
 
 cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, CacheDev small_cache,
                           bool has_full, bool has_small, int n_seq, int n_kv_heads, int32_t* status,
                           cudaStream_t st) {
-  append_kernel<<<n_seq, 128, 0, st>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), full,
-                                       small_cache, has_full ? 1 : 0, has_small ? 1 : 0, n_kv_heads, status);
-  return cudaGetLastError();
+  return launch_ex(append_kernel, dim3(n_seq), dim3(128), 0, st, 1, static_cast<const uint4*>(k_new),
+                   static_cast<const uint4*>(v_new), full, small_cache, has_full ? 1 : 0, has_small ? 1 : 0,
+                   n_kv_heads, status);
 }
 
 cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, float* sim,
                            int n_seq, int n_q_heads, cudaStream_t st) {
-  trigger_kernel<<<n_seq, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(q_now),
-                                        static_cast<const __nv_bfloat16*>(q_last), threshold, flag, sim,
-                                        n_q_heads);
-  return cudaGetLastError();
+  return launch_ex(trigger_kernel, dim3(n_seq), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(q_now),
+                   static_cast<const __nv_bfloat16*>(q_last), threshold, flag, sim, n_q_heads);
 }
 
 }  // namespace rkv

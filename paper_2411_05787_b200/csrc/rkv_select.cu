@@ -46,7 +46,7 @@ struct SelectShared {
   alignas(16) double lse[kMaxGroup];
   alignas(16) float ML[16];
   uint32_t warp_tot[NT / 32];
-  uint32_t totals[2];                    // this CTA's number of keys below / equal to the threshold key
+  uint32_t peer_totals[kSelectCluster];  // per CTA of the cluster: keys below (low 16 bits) / equal to (high) the threshold key
   uint32_t cand_count;                   // CTA 0 only: pool fill
   uint32_t digit, want, count;
 };
@@ -163,11 +163,14 @@ __device__ __forceinline__ void local_pass(SelectShared* sh, int n_cand, uint32_
   locate(sh, mine, want);
 }
 
+template <int GMAX>
 __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x;
+  pdl_launch();
+  pdl_wait();
   if (p.active != nullptr && p.active[b] == 0) return;  // same decision in all CTAs of the cluster
 
   SelectShared* sh = reinterpret_cast<SelectShared*>(smem_raw);
@@ -228,27 +231,30 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   bool bad = false;
   const bool all_selected = (kk == n);
   const int agg = p.agg;
-  double lse_r[kMaxGroup];
+  double lse_r[GMAX];
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) lse_r[h] = sh->lse[h];
-  for (int i0 = 0; i0 < cnt; i0 += 4 * NT) {
-    float v[4][kMaxGroup];
+  for (int h = 0; h < GMAX; ++h) lse_r[h] = sh->lse[h];
+  constexpr int U = 32 / GMAX;   // positions per thread per round: all their loads are in flight together
+  for (int i0 = 0; i0 < cnt; i0 += U * NT) {
+    float v[U][GMAX];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < U; ++u) {
       const int i = i0 + u * NT + tid;
 #pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h)
-        v[u][h] = (h < G && i < cnt && (agg != RKV_AGG_FIRST || h == 0)) ? __ldcg(lg + (int64_t)h * p.logit_stride + lo + i) : 0.f;
+      for (int h = 0; h < GMAX; ++h)
+        v[u][h] = (h < G && i < cnt && (agg != RKV_AGG_FIRST || h == 0))
+                      ? __ldcg(lg + (int64_t)h * p.logit_stride + lo + i)
+                      : 0.f;
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < U; ++u) {
       const int i = i0 + u * NT + tid;
       if (i >= cnt) continue;
       double ell;
       if (agg == RKV_AGG_MAX) {
         ell = -INFINITY;
 #pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h) {
+        for (int h = 0; h < GMAX; ++h) {
           if (h < G) {
             const double x = (double)v[u][h] - lse_r[h];
             if (x != x) bad = true;
@@ -258,7 +264,7 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
       } else if (agg == RKV_AGG_MEAN) {
         double acc = 0.0;
 #pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h)
+        for (int h = 0; h < GMAX; ++h)
           if (h < G) acc += exp((double)v[u][h] - lse_r[h]);
         if (acc != acc) bad = true;
         ell = log(acc / (double)G);
@@ -284,6 +290,7 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
     for (int i = tid; i < cnt; i += NT) idx_out[lo + i] = lo + i;
     return;
   }
+  if (kk == 0) return;  // nothing to select (uniform over the cluster); scores and out are written
 
   // ---------------------------------------------------------------- locate the kk-th smallest key
   // prefix = the key's bits above `shift` that are already fixed
@@ -312,11 +319,18 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
     // pool the candidates (keys whose fixed bits match) in CTA 0, then finish locally in every CTA
     const uint32_t pool = map_rank(smem_u32(&sh->cand[0]), 0);
     const uint32_t pool_cnt = map_rank(smem_u32(&sh->cand_count), 0);
-    for (int i = tid; i < cnt; i += NT) {
+    uint32_t mine_c = 0;
+    for (int i = tid; i < cnt; i += NT) mine_c += ((keys[i] >> shift) == prefix);
+    uint32_t tot_c;
+    uint32_t slot = block_excl_scan(mine_c, sh->warp_tot, &tot_c);
+    if (tid == 0) sh->digit = tot_c ? atom_add_cluster(pool_cnt, tot_c) : 0u;   // one reservation per CTA
+    __syncthreads();
+    slot += sh->digit;
+    for (int i = tid; i < cnt && mine_c; i += NT) {
       const uint32_t key = keys[i];
       if ((key >> shift) == prefix) {
-        const uint32_t slot = atom_add_cluster(pool_cnt, 1u);
         if (slot < (uint32_t)kCand) st_cluster(pool + 4 * slot, key);
+        ++slot;
       }
     }
     cluster.sync();
@@ -347,33 +361,30 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
     c_less += (key < tau);
     c_eq += (key == tau);
   }
-  uint32_t tot_less, tot_eq;
-  block_excl_scan(c_less, sh->warp_tot, &tot_less);
-  const uint32_t e_eq = block_excl_scan(c_eq, sh->warp_tot, &tot_eq);
-  if (tid == 0) {
-    sh->totals[0] = tot_less;
-    sh->totals[1] = tot_eq;
+  // counts fit 16 bits each (at most 40960 keys per CTA): one packed scan gives both prefixes
+  uint32_t tot_packed;
+  const uint32_t e_packed = block_excl_scan(c_less | (c_eq << 16), sh->warp_tot, &tot_packed);
+  const uint32_t e_less = e_packed & 0xffffu, e_eq = e_packed >> 16;
+  if (tid < kSelectCluster) {  // push this CTA's totals to every peer: no remote read is needed later
+    const uint32_t dst = map_rank(smem_u32(&sh->peer_totals[rank]), tid);
+    st_cluster(dst, tot_packed);
   }
   cluster.sync();
   uint32_t ties_before = 0, winners_before = 0, my_quota = 0;
-  {
-    const uint32_t tl = smem_u32(&sh->totals[0]);
-    for (int r = 0; r <= rank; ++r) {
-      const uint32_t ra = map_rank(tl, r);
-      const uint32_t less_r = ld_cluster(ra), eq_r = ld_cluster(ra + 4);
-      const uint32_t left = ties_to_take > ties_before ? ties_to_take - ties_before : 0u;
-      const uint32_t take = left < eq_r ? left : eq_r;
-      if (r < rank) {
-        winners_before += less_r + take;
-        ties_before += eq_r;
-      } else {
-        my_quota = take;
-      }
+  for (int r = 0; r <= rank; ++r) {
+    const uint32_t t = sh->peer_totals[r];
+    const uint32_t less_r = t & 0xffffu, eq_r = t >> 16;
+    const uint32_t left = ties_to_take > ties_before ? ties_to_take - ties_before : 0u;
+    const uint32_t take = left < eq_r ? left : eq_r;
+    if (r < rank) {
+      winners_before += less_r + take;
+      ties_before += eq_r;
+    } else {
+      my_quota = take;
     }
   }
-  const uint32_t my_eq_take = (my_quota > e_eq) ? ((my_quota - e_eq < c_eq) ? my_quota - e_eq : c_eq) : 0u;
-  uint32_t tot_w;
-  uint32_t offs = block_excl_scan(c_less + my_eq_take, sh->warp_tot, &tot_w) + winners_before;
+  // ties are kept in position order, so min(e_eq, quota) of them precede this thread's run
+  uint32_t offs = winners_before + e_less + (e_eq < my_quota ? e_eq : my_quota);
   uint32_t eq_seen = e_eq;
   for (int i = r_lo; i < r_hi; ++i) {
     const uint32_t key = keys[i];
@@ -387,7 +398,7 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
       ++offs;
     }
   }
-  cluster.sync();  // nobody leaves while its shared memory may still be read by a peer
+  // no cluster barrier here: after the one above nobody touches a peer's shared memory any more
 }
 
 }  // namespace
@@ -397,25 +408,18 @@ size_t select_smem_bytes(int keys_per_cta) {
 }
 
 cudaError_t prepare_select() {
-  cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(select_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)select_smem_bytes(kSelectMaxKeysPerCta));
-  return e;
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)select_smem_bytes(kSelectMaxKeysPerCta));
 }
 
 cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(kSelectCluster, p.n_kv_heads, n_seq);
-  cfg.blockDim = dim3(NT, 1, 1);
-  cfg.dynamicSmemBytes = select_smem_bytes(p.keys_per_cta);
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = kSelectCluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_kernel, p);
+  const dim3 grid(kSelectCluster, p.n_kv_heads, n_seq);
+  if (p.group <= 4)
+    return launch_ex(select_kernel<4>, grid, dim3(NT), select_smem_bytes(p.keys_per_cta), st, kSelectCluster, p);
+  return launch_ex(select_kernel<8>, grid, dim3(NT), select_smem_bytes(p.keys_per_cta), st, kSelectCluster, p);
 }
 
 }  // namespace rkv

@@ -20,7 +20,8 @@ DEV_APPEND_OVERFLOW, DEV_LEN_CLAMPED, DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT 
 
 EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", "rkv_gather_small",
            "rkv_small_step", "rkv_append", "rkv_should_refresh", "rkv_get_device_status",
-           "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile"]
+           "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile", "rkv_set_option"]
+OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH = 1, 2
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
 
 
@@ -58,6 +59,8 @@ def _load() -> ctypes.CDLL:
     lib.rkv_last_cuda_error.restype = ctypes.c_char_p
     lib.rkv_launch_count.argtypes = [vp]
     lib.rkv_launch_count.restype = i64
+    lib.rkv_set_option.argtypes = [vp, i32, i32]
+    lib.rkv_set_option.restype = i32
     lib.rkv_set_profiling.argtypes = [vp, i32]
     lib.rkv_set_profiling.restype = i32
     lib.rkv_get_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
@@ -160,6 +163,9 @@ class Context:
     def should_refresh(self, q_now, q_last_full, threshold, flag, sim=None, stream=None):
         self._check(lib.rkv_should_refresh(self._h, _ptr(q_now), _ptr(q_last_full), float(threshold), _ptr(flag),
                                            _ptr(sim), _stream(stream)))
+
+    def set_option(self, option: int, value: int):
+        self._check(lib.rkv_set_option(self._h, option, value))
 
     def set_profiling(self, on: bool):
         self._check(lib.rkv_set_profiling(self._h, 1 if on else 0))
