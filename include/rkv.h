@@ -167,6 +167,44 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new,
 rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_last_full,
                               float threshold, int32_t* flag, float* sim, void* stream);
 
+/*
+ * Partial step without a context and without any allocation (the paper has no counterpart: this
+ * exists for deployment reasons only).
+ *
+ * Who needs it: hosts that cannot call cudaMalloc where they run attention - a serving runtime
+ * whose own arena already owns the device heap, a plugin that must stay inside another program's
+ * memory budget, a latency path on which an allocation (which synchronises the device) is not
+ * allowed.  rkv_create allocates a workspace, so such callers cannot hold an rkv_ctx.  This call
+ * computes exactly what rkv_small_step computes, but its scratch (split partials, arrival
+ * tickets, a status word) is a fixed array inside the library image: every device that loads the
+ * library holds those ~2.1 MB until the process exits.  The call never calls cudaMalloc, cudaFree
+ * or any other allocating routine; the caller passes inputs and outputs as usual.
+ *
+ * Limits (the array is sized for them; beyond them the call returns RKV_ERR_UNSUPPORTED and, if
+ * err_msg is given, says which limit was hit):
+ *   cfg->n_seq * cfg->n_kv_heads <= RKV_NOALLOC_MAX_PROBLEMS
+ *   length bound (max_len_hint, or cfg->max_small when the hint is 0) <= RKV_NOALLOC_MAX_LEN
+ * Of cfg only n_seq, n_q_heads, n_kv_heads, head_dim, max_small and softmax_scale are read.
+ *
+ * First call on a device: looks up the array's device address, sets the kernel's shared-memory
+ * attribute and resolves the tensor-map encoder (host work, once per device, under a lock).  Make
+ * that first call outside any stream capture.
+ * Sharing: every call on a device uses the same array, which keeps the previous call's contents;
+ * the call clears the tickets (and the built-in status word) on the stream before it launches.
+ * Two calls that overlap on the GPU (different streams, no ordering) race on the array: order them.
+ *   device_status  optional device int32: receives the RKV_DEV_* bits the kernel raises (sticky,
+ *                  the caller clears it).  NULL: the bits go to the built-in word and are dropped.
+ *   err_msg        optional host buffer of err_cap bytes for a one-line reason on failure.
+ * Other arguments as in rkv_small_step.
+ */
+#define RKV_NOALLOC_MAX_PROBLEMS 32
+#define RKV_NOALLOC_MAX_SPLITS 16
+#define RKV_NOALLOC_MAX_LEN 65536
+rkv_status rkv_small_step_noalloc(const rkv_config* cfg /*host*/, const void* q,
+                                  const rkv_cache* small_cache /*host struct*/, const int32_t* active,
+                                  void* out, int32_t max_len_hint, int32_t* device_status, void* stream,
+                                  char* err_msg /*host*/, size_t err_cap);
+
 /* Host.  Synchronises the stream, copies the sticky device status word to
  * *host_bits, clears it, and returns RKV_ERR_DEVICE_CHECK if it was non-zero. */
 rkv_status rkv_get_device_status(rkv_ctx* ctx, int32_t* host_bits /*host*/, void* stream);

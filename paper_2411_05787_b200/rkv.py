@@ -20,7 +20,9 @@ DEV_APPEND_OVERFLOW, DEV_LEN_CLAMPED, DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT 
 
 EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", "rkv_gather_small",
            "rkv_small_step", "rkv_append", "rkv_should_refresh", "rkv_get_device_status",
-           "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile", "rkv_set_option"]
+           "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
+           "rkv_set_option", "rkv_small_step_noalloc"]
+NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH = 1, 2
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
 
@@ -65,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.rkv_set_profiling.restype = i32
     lib.rkv_get_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     lib.rkv_get_profile.restype = i32
+    lib.rkv_small_step_noalloc.argtypes = [cfgp, vp, cachep, vp, vp, i32, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
+    lib.rkv_small_step_noalloc.restype = i32
     for name in ("rkv_create", "rkv_destroy", "rkv_full_step", "rkv_gather_small", "rkv_small_step",
                  "rkv_append", "rkv_should_refresh", "rkv_get_device_status"):
         getattr(lib, name).restype = i32
@@ -102,6 +106,18 @@ def cache_struct(k, v, row_offset, cap, length) -> RkvCache:
     assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.shape == v.shape and k.shape[-1] == 128
     assert row_offset.dtype == torch.int64 and cap.dtype == torch.int32 and length.dtype == torch.int32
     return RkvCache(_ptr(k), _ptr(v), k.numel() // 128, _ptr(row_offset), _ptr(cap), _ptr(length))
+
+
+def small_step_noalloc(cfg: RkvConfig, q, small: RkvCache, out, active=None, max_len_hint=0, device_status=None,
+                       stream=None):
+    """Partial step for callers that may not allocate device memory (no context; see include/rkv.h).
+
+    Raises RkvError carrying the library's one-line reason, e.g. when a size exceeds the static scratch."""
+    msg = ctypes.create_string_buffer(256)
+    rc = lib.rkv_small_step_noalloc(ctypes.byref(cfg), _ptr(q), ctypes.byref(small), _ptr(active), _ptr(out),
+                                    max_len_hint, _ptr(device_status), _stream(stream), msg, len(msg))
+    if rc != RKV_OK:
+        raise RkvError(rc, msg.value.decode())
 
 
 class Context:
