@@ -220,13 +220,18 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
 /*
  * Launch-geometry knobs (no counterpart in the paper).  Results never depend on them beyond
  * floating-point summation order.
- *   RKV_OPT_SMALL_MIN_CHUNK   positions per CTA (at least) in rkv_small_step; default 256, >= 64
+ *   RKV_OPT_SMALL_MIN_CHUNK   positions per CTA (at least) in rkv_small_step when its splits are merged
+ *                             through the workspace; default 256, >= 64
+ *   RKV_OPT_SMALL_CLUSTER     1 (default): rkv_small_step merges the splits of one (sequence, KV head)
+ *                             inside a thread-block cluster (no workspace traffic) when the length
+ *                             bound is at most 8192 positions; 0: always through the workspace
  *   RKV_OPT_DEPENDENT_LAUNCH  1 (default): kernels are launched with programmatic stream
  *                             serialisation so that a kernel's launch overlaps the tail of its
  *                             predecessor; 0: plain stream order.  Process-wide.
  */
 #define RKV_OPT_SMALL_MIN_CHUNK 1
 #define RKV_OPT_DEPENDENT_LAUNCH 2
+#define RKV_OPT_SMALL_CLUSTER 3
 rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
 
 /*

@@ -47,7 +47,8 @@ WsLayout ws_layout(const rkv_config* c) {
   size_t off = 0;
   w.partials = off; off = up(off + bg * splits_for(c) * rkv::PartialLayout::kFloats * sizeof(float));
   w.tickets = off;  off = up(off + bg * sizeof(int32_t));
-  w.logits = off;   off = up(off + bg * group * (size_t)w.logit_stride * sizeof(float));
+  const int gp = group <= 4 ? 4 : 8;   // position-major logits, padded to a vector width
+  w.logits = off;   off = up(off + bg * gp * (size_t)w.logit_stride * sizeof(float));
   w.status = off;   off = up(off + sizeof(int32_t));
   w.total = off;
   return w;
@@ -140,8 +141,11 @@ int choose_chunk(const rkv_ctx* ctx, int n_max, bool full, int* grid_x) {
   return chunk;
 }
 
+// Longest small cache that the clustered partial step takes (8 CTAs x 1024 positions).
+constexpr int kClusterMaxLen = 8192;
+
 rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
-                         int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out) {
+                         int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out, int* gx_out) {
   CUtensorMap tm_k, tm_v;
   rkv_status s = tensor_map(ctx, cache->k, cache->n_rows, &tm_k);
   if (s != RKV_OK) return s;
@@ -150,8 +154,16 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   AttnParams p;
   memset(&p, 0, sizeof(p));
   int gx = 1;
-  p.chunk = choose_chunk(ctx, n_max, logits, &gx);
+  const bool cluster = !logits && ctx->small_cluster != 0 && n_max <= kClusterMaxLen;
+  if (cluster) {   // 1, 2, 4 or 8 CTAs per (sequence, KV head), whole tiles each
+    const int tiles = (n_max + rkv::kTile - 1) / rkv::kTile;
+    gx = tiles >= 5 ? 8 : tiles >= 3 ? 4 : tiles >= 2 ? 2 : 1;
+    p.chunk = ((tiles + gx - 1) / gx) * rkv::kTile;
+  } else {
+    p.chunk = choose_chunk(ctx, n_max, logits, &gx);
+  }
   if (chunk_out) *chunk_out = p.chunk;
+  if (gx_out) *gx_out = gx;
   p.q = q;
   p.row_offset = cache->row_offset;
   p.cap = cache->cap;
@@ -166,13 +178,15 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.n_q_heads = ctx->cfg.n_q_heads;
   p.n_kv_heads = ctx->cfg.n_kv_heads;
   p.group = ctx->group;
+  p.gp = ctx->gp;
   p.max_splits = ctx->max_splits;
   p.max_len = limit;
   p.scale = ctx->cfg.softmax_scale;
   cudaError_t e;
   {
     LaunchScope scope(ctx, st, logits ? RKV_KERNEL_ATTN_FULL : RKV_KERNEL_ATTN_SMALL);
-    e = rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
+    e = cluster ? rkv::launch_attention_cluster(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
+                : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
   ctx->launches += 1;
@@ -207,6 +221,8 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->launches = 0;
   ctx->profiling = false;
   ctx->small_min_chunk = 256;
+  ctx->small_cluster = 1;
+  ctx->gp = ctx->group <= 4 ? 4 : 8;
   ctx->workspace = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -251,8 +267,8 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, con
   if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
   if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int chunk = 0;
-  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk);
+  int chunk = 0, gx = 1;
+  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx);
   if (s != RKV_OK) return s;
   SelectParams sp;
   memset(&sp, 0, sizeof(sp));
@@ -278,8 +294,9 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, con
   sp.agg = ctx->cfg.agg;
   sp.k_max = k_max;
   sp.max_len = n_max;
-  int per = (n_max + rkv::kSelectCluster - 1) / rkv::kSelectCluster;
-  sp.keys_per_cta = (per + 3) & ~3;
+  const int per = (n_max + rkv::kSelectCluster - 1) / rkv::kSelectCluster;
+  sp.per_cta = (per + 3) & ~3;
+  sp.grid_splits = gx;
   cudaError_t e;
   {
     LaunchScope scope(ctx, st, RKV_KERNEL_SELECT);
@@ -312,7 +329,7 @@ rkv_status rkv_small_step(rkv_ctx* ctx, const void* q, const rkv_cache* small_ca
   int n_max = max_len_hint == 0 ? ctx->cfg.max_small : max_len_hint;
   if (n_max < 1 || n_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
   return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, static_cast<cudaStream_t>(stream),
-                       nullptr);
+                       nullptr, nullptr);
 }
 
 rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const rkv_cache* full,
@@ -380,6 +397,9 @@ rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value) {
     case RKV_OPT_SMALL_MIN_CHUNK:
       if (value < rkv::kTile || value > (1 << 20)) return RKV_ERR_INVALID_ARG;
       ctx->small_min_chunk = value;
+      return RKV_OK;
+    case RKV_OPT_SMALL_CLUSTER:
+      ctx->small_cluster = value != 0;
       return RKV_OK;
     case RKV_OPT_DEPENDENT_LAUNCH:
       rkv::g_use_pdl = value != 0;

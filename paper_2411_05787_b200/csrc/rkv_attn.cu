@@ -14,9 +14,14 @@
 // mbarriers).  Four MMA warps each own 16 positions of a tile: S^T = K Q^T and
 // O^T += V^T P^T with m16n8k16 bf16 tensor-core MMAs (fp32 accumulate), where
 // the N=8 dimension holds all query heads of the group, so K/V are read once
-// per group.  Online softmax lives in registers; the split partials are merged
-// by the last CTA of each (sequence, KV head) to arrive (atomic ticket, no
-// spinning).
+// per group.  Online softmax lives in registers.  Three ways to merge the splits:
+//   full step      partials go to the workspace, the selection kernel folds them;
+//   partial step   (a) the CTAs of one (sequence, KV head) form a thread-block cluster:
+//                  each pushes its slice of the partial output into the peer that owns
+//                  that slice through distributed shared memory, one cluster barrier,
+//                  each CTA finishes 128/C channels of every head;
+//                  (b) long small caches: partials to the workspace, folded by the last
+//                  CTA of each (sequence, KV head) to arrive (atomic ticket, no spin).
 #include <cuda_bf16.h>
 
 #include "rkv_fold.cuh"
@@ -30,6 +35,9 @@ constexpr int kHalfBytes = kTile * 128;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kOPad = 132;  // floats per head row in the merge buffer (bank spread)
+constexpr int kRecvFloats = kMaxGroup * kHeadDim + kAttnCluster * kMaxGroup * 2;   // pushed slices + (m, l) pairs
+
+enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -68,6 +76,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
       "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
       : "memory");
 }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tm) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -100,18 +111,31 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ uint32_t map_rank(uint32_t local_addr, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+// Cluster barrier (all five warps of every CTA of the cluster arrive).
+__device__ __forceinline__ void cluster_sync_alive() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
-template <bool kLogits>
+template <int kMode>
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
             const AttnParams p) {
+  constexpr bool kLogits = (kMode == kModeFull);
   extern __shared__ uint8_t smem_raw[];
   __shared__ int s_last;
 
   const int b = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   pdl_launch();
-  // shared memory: [stages][K lo | K hi | V lo | V hi], then the barriers
+  // shared memory: [stages][K lo | K hi | V lo | V hi], the barriers, then (cluster mode) the receive buffer
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t bar_full = smem_base + kStages * kStageBytes;
@@ -123,11 +147,37 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  pdl_wait();   // nothing above reads global memory
-  if (p.active != nullptr && p.active[b] == 0) return;
+  if (tid == kAttnThreads - 32) {
+    prefetch_tensormap(&tm_k);
+    prefetch_tensormap(&tm_v);
+  }
   const int G = p.group;
-  const int cap = p.cap[b];
-  int n = p.len[b];
+  const int64_t head0 = ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
+  __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out) + head0;
+  const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + head0;
+  const int qd = lane >> 2;       // row inside an 8-row group
+  const int qc = (lane & 3) * 2;  // first of the two columns this lane holds
+  pdl_wait();   // nothing above reads global memory
+
+  // per-sequence sizes and (MMA warps) the query fragments: independent loads, one round trip
+  const int act = (p.active != nullptr) ? __ldcg(p.active + b) : 1;
+  const int cap = __ldcg(p.cap + b);
+  int n = __ldcg(p.len + b);
+  const int64_t roff = __ldcg(p.row_offset + b);
+  uint32_t qb[8][2];              // B fragments of Q^T: [k = channel][n = head]
+  if (warp < 4) {
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      if (qd < G) {
+        qb[ks][0] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc);
+        qb[ks][1] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc + 8);
+      } else {
+        qb[ks][0] = 0u;
+        qb[ks][1] = 0u;
+      }
+    }
+  }
+  if (act == 0) return;   // the same for every CTA of a cluster
   {
     const int lim = cap < p.max_len ? cap : p.max_len;
     if (n > lim) {
@@ -136,20 +186,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     }
     if (n < 0) n = 0;
   }
-  __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
-  const __nv_bfloat16* qg =
-      static_cast<const __nv_bfloat16*>(p.q) + ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
   if (n == 0) {  // nothing cached: the output is defined as zero
     if (split == 0 && tid < kHeadDim)
       for (int h = 0; h < G; ++h) out[h * kHeadDim + tid] = __float2bfloat16(0.f);
     return;
   }
   const int start = split * p.chunk;
-  if (start >= n) return;
+  if (kMode != kModeCluster && start >= n) return;   // in a cluster an idle CTA still owns a slice of the output
   const int end = (start + p.chunk < n) ? start + p.chunk : n;
-  const int n_tiles = (end - start + kTile - 1) / kTile;
+  const int n_tiles = (end > start) ? (end - start + kTile - 1) / kTile : 0;
   const int n_splits = (n + p.chunk - 1) / p.chunk;
-  const int64_t row0 = p.row_offset[b] + (int64_t)g * cap + start;
+  const int64_t row0 = roff + (int64_t)g * cap + start;
 
   __syncthreads();   // barrier initialisation (above) is visible to every warp
 
@@ -174,31 +221,24 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
       }
     }
+    if (kMode == kModeCluster) {   // stay until the peers have pushed: every warp of the cluster meets at one barrier
+      __syncwarp();
+      cluster_sync_alive();
+    }
     return;
   }
 
   // ---------------------------------------------------------------- MMA warps
-  const int qd = lane >> 2;       // row inside an 8-row group
-  const int qc = (lane & 3) * 2;  // first of the two columns this lane holds
-  uint32_t qb[8][2];              // B fragments of Q^T: [k = channel][n = head]
-#pragma unroll
-  for (int ks = 0; ks < 8; ++ks) {
-    if (qd < G) {
-      qb[ks][0] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc);
-      qb[ks][1] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc + 8);
-    } else {
-      qb[ks][0] = 0u;
-      qb[ks][1] = 0u;
-    }
-  }
   const float ninf = -INFINITY;
   float m0 = ninf, m1 = ninf, l0 = 0.f, l1 = 0.f;
   float o[8][4];
 #pragma unroll
   for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
 
+  // logit scratch is position-major: [position][GP] floats, GP = 4 or 8; this lane holds heads qc, qc+1
   float* lg0 = nullptr;
-  if (kLogits) lg0 = p.logits + ((int64_t)(b * p.n_kv_heads + g) * G + qc) * p.logit_stride;
+  if (kLogits) lg0 = p.logits + (int64_t)(b * p.n_kv_heads + g) * p.logit_stride * p.gp + qc;
+  const bool lg_on = kLogits && qc < p.gp;
 
   const int krow = 16 * warp + (lane & 15);
   const int vrow = 16 * warp + ((lane >> 4) << 3) + (lane & 7);
@@ -225,13 +265,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       const int r0 = pos_base + qd, r1 = r0 + 8;
       float s0 = c[0] * p.scale, s1 = c[1] * p.scale, s2 = c[2] * p.scale, s3 = c[3] * p.scale;
       if (kLogits) {
-        if (qc < G) {
-          if (r0 < end) lg0[r0] = s0;
-          if (r1 < end) lg0[r1] = s2;
-        }
-        if (qc + 1 < G) {
-          if (r0 < end) lg0[p.logit_stride + r0] = s1;
-          if (r1 < end) lg0[p.logit_stride + r1] = s3;
+        if (lg_on) {
+          if (r0 < end) *reinterpret_cast<float2*>(lg0 + (int64_t)r0 * p.gp) = make_float2(s0, s1);
+          if (r1 < end) *reinterpret_cast<float2*>(lg0 + (int64_t)r1 * p.gp) = make_float2(s2, s3);
         }
       }
       if (r0 >= end) s0 = s1 = ninf;
@@ -342,7 +378,52 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   }
 
   const int bg = b * p.n_kv_heads + g;
-  const bool single = (!kLogits) && n_splits == 1;   // the full step always leaves its partials to the selector
+
+  if (kMode == kModeCluster) {
+    // ---------------------------------------------- merge the CTAs of the cluster through shared memory
+    const int C = (int)gridDim.x;                       // cluster size = CTAs per (sequence, KV head)
+    const int dchunk = kHeadDim / C;                    // channels of every head that one CTA finishes
+    float* recv = reinterpret_cast<float*>(smem_gen + kStages * kStageBytes + 16 * kStages + 16);
+    float* recv_ml = recv + kMaxGroup * kHeadDim;       // [source CTA][head][2]
+    const uint32_t recv_u32 = smem_u32(recv), recv_ml_u32 = smem_u32(recv_ml);
+    {
+      const int owner = d / dchunk, dd = d - owner * dchunk;
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h < G) st_cluster_f32(map_rank(recv_u32 + 4u * ((split * kMaxGroup + h) * dchunk + dd), owner), accO[h]);
+      if (d < kMaxGroup * C) {   // (m, l) of head d % 8 to peer d / 8
+        const int h = d & 7, peer = d >> 3;
+        float Md = ninf, Ld = 0.f;
+#pragma unroll
+        for (int hh = 0; hh < kMaxGroup; ++hh)
+          if (hh == h) {
+            Md = accM[hh];
+            Ld = accL[hh];
+          }
+        const uint32_t dst = map_rank(recv_ml_u32 + 4u * ((split * kMaxGroup + h) * 2), peer);
+        st_cluster_f32(dst, Md);
+        st_cluster_f32(dst + 4u, Ld);
+      }
+    }
+    cluster_sync_alive();
+    if (!ok) return;
+    for (int item = d; item < G * dchunk; item += 128) {
+      const int h = item / dchunk, dd = item - h * dchunk;
+      float M = ninf;
+      for (int r = 0; r < C; ++r) M = fmaxf(M, recv_ml[(r * kMaxGroup + h) * 2]);
+      float L = 0.f, O = 0.f;
+      for (int r = 0; r < C; ++r) {
+        const float mr = recv_ml[(r * kMaxGroup + h) * 2];
+        const float e = (mr == ninf) ? 0.f : ex2((mr - M) * kLog2e);
+        L = fmaf(recv_ml[(r * kMaxGroup + h) * 2 + 1], e, L);
+        O = fmaf(recv[(r * kMaxGroup + h) * dchunk + dd], e, O);
+      }
+      out[h * kHeadDim + split * dchunk + dd] = __float2bfloat16(O / L);
+    }
+    return;
+  }
+
+  const bool single = (kMode == kModeTicket) && n_splits == 1;   // the full step always leaves its partials to the selector
   if (!single) {
     float* part = p.partials + ((int64_t)bg * p.max_splits + split) * PartialLayout::kFloats;
 #pragma unroll
@@ -359,7 +440,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       part[kMaxGroup * kHeadDim + d] = Md;
       part[kMaxGroup * kHeadDim + kMaxGroup + d] = Ld;
     }
-    if (kLogits) return;   // full step: the selection kernel folds the partials (in parallel, per head)
+    if (kLogits) return;   // full step: the selection kernel folds the partials
     __threadfence();
     consumer_bar();
     if (tid == 0) {
@@ -395,22 +476,31 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
 
 }  // namespace
 
-size_t attention_smem_bytes() { return (size_t)kStages * kStageBytes + 16 * kStages + 1024; }
+size_t attention_smem_bytes() {
+  return (size_t)kStages * kStageBytes + 16 * kStages + 16 + (size_t)kRecvFloats * sizeof(float) + 1024;
+}
 
 cudaError_t prepare_attention() {
-  cudaError_t e = cudaFuncSetAttribute(attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)attention_smem_bytes());
+  const int bytes = (int)attention_smem_bytes();
+  cudaError_t e = cudaFuncSetAttribute(attn_kernel<kModeFull>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)attention_smem_bytes());
+  e = cudaFuncSetAttribute(attn_kernel<kModeTicket>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_kernel<kModeCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                              int n_seq, int grid_x, bool write_logits, cudaStream_t st) {
   dim3 grid(grid_x, p.n_kv_heads, n_seq);
   if (write_logits)
-    return launch_ex(attn_kernel<true>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
-  return launch_ex(attn_kernel<false>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
+    return launch_ex(attn_kernel<kModeFull>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
+  return launch_ex(attn_kernel<kModeTicket>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
+}
+
+cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                     int n_seq, int cluster, cudaStream_t st) {
+  dim3 grid(cluster, p.n_kv_heads, n_seq);
+  return launch_ex(attn_kernel<kModeCluster>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, cluster, tm_k, tm_v, p);
 }
 
 }  // namespace rkv

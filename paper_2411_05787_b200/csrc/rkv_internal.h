@@ -19,6 +19,7 @@ constexpr int kTile = 64;              // positions per pipeline stage
 constexpr int kStages = 3;
 constexpr int kAttnThreads = 160;      // 4 MMA warps + 1 copy warp
 constexpr int kSelectCluster = 8;      // CTAs that share one top-K problem
+constexpr int kAttnCluster = 8;        // most CTAs that share one (sequence, KV head) in the clustered partial step
 constexpr int kSelectThreads = 512;
 constexpr int kSelectMaxKeysPerCta = 40960;
 constexpr int kDevTimeoutBit = 16;     // internal: a bounded barrier wait ran out
@@ -37,10 +38,11 @@ struct AttnParams {
   void* out;                  // bf16 [B][Hq][128]
   float* partials;            // [B*Hkv][max_splits][PartialLayout::kFloats]
   int32_t* tickets;           // [B*Hkv]
-  float* logits;              // [B*Hkv][G][logit_stride] or null
+  float* logits;              // [B*Hkv][logit_stride][gp] (position-major) or null
   int32_t* status;
   int64_t logit_stride;
   int32_t n_q_heads, n_kv_heads, group;
+  int32_t gp;                 // floats per position in the logit scratch: 4 (G <= 4) or 8
   int32_t chunk;              // positions per CTA
   int32_t max_splits;
   int32_t max_len;            // clamp for len[b]
@@ -48,7 +50,7 @@ struct AttnParams {
 };
 
 struct SelectParams {
-  const float* logits;        // [B*Hkv][G][logit_stride]
+  const float* logits;        // [B*Hkv][logit_stride][gp]
   const float* partials;      // split partials written by the attention kernel
   const void* q;              // bf16 [B][Hq][128]
   void* out;                  // bf16 [B][Hq][128]
@@ -63,8 +65,9 @@ struct SelectParams {
   int64_t logit_stride, score_stride;
   int32_t n_q_heads, n_kv_heads, group, agg;
   int32_t k_max, max_len;
-  int32_t keys_per_cta;       // capacity of the shared-memory key array
+  int32_t per_cta;            // positions per CTA of the cluster (from the host's length bound; multiple of 4)
   int32_t chunk, max_splits;  // split geometry of the attention launch that produced the partials
+  int32_t grid_splits;        // CTAs per (sequence, KV head) that launch had
 };
 
 struct CacheDev {
@@ -74,6 +77,8 @@ struct CacheDev {
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                              int n_seq, int grid_x, bool write_logits, cudaStream_t st);
+cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                     int n_seq, int cluster, cudaStream_t st);
 cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st);
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
@@ -143,6 +148,8 @@ struct rkv_ctx {
   int device;
   int sm_count;
   int small_min_chunk;
+  int small_cluster;   // 1: the partial step merges its splits inside a thread-block cluster when the length allows
+  int gp;              // floats per position in the logit scratch
   std::string last_error;
   std::unordered_map<uint64_t, CUtensorMap> tmaps;
   // optional per-kernel timing (rkv_set_profiling): event pairs recorded around every launch

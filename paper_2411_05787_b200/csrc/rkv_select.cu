@@ -6,51 +6,67 @@
 // attention the scores of the query heads of a group are aggregated by max
 // (footnote of Sec. 2.2; mean / first head are the ablation modes of App. A.3).
 //
-// Input: the scaled logits s[h][j] and the split partials the attention kernel
-// wrote.  The cluster first folds the partials (CTA r produces out[] of query
-// head r of the group; every CTA derives the log-sum-exp of all heads), then
-//   log p[h][j] = s[h][j] - LSE[h],   ell[j] = agg_h log p[h][j],
-// and the K largest scores are the K largest ell.  Selection works on a 31-bit
-// fixed-point image of -ell (2^-24 resolution = 6e-8 relative in the score;
-// equal images are ties and go to the lower position): a histogram pass over
-// the top 11 bits, merged across the cluster through distributed shared
-// memory, isolates the bin that holds the K-th key; while that bin is too
-// crowded further histogram passes refine it; then the few candidates are
-// pooled in CTA 0's shared memory and every CTA finishes the exact selection
-// locally.  Winners are written in ascending position order (deterministic,
-// and the later gather walks the cache monotonically).
-#include <cooperative_groups.h>
+// Input: the scaled logits s[j][h] (position-major, GP = 4 or 8 floats per position)
+// and the split partials the attention kernel wrote.  Every CTA derives the
+// log-sum-exp of all heads of the group from the partials and folds one eighth of
+// out[] of the group.  Then
+//   ell[j] = agg_h (s[j][h] - LSE[h])            (log of the aggregated probability)
+// and the K largest scores are the K smallest keys  key = bits(max(-ell, 0)),  an
+// order-preserving 31-bit image of -ell (equal images are ties and go to the lower
+// position).  The kernel is a chain of latencies, so it is laid out to have few links:
+//   1  one round trip fetches the per-sequence sizes, the split weights, this CTA's
+//      slice of the partial outputs and its first logits, all at once;
+//   2  keys + a 2048-bin histogram (1/64 nat per bin) in shared memory;
+//   3  cluster barrier; the eight histograms are merged through distributed shared
+//      memory and the bin T that holds the K-th key is located (while T holds more
+//      than 256 keys, a finer histogram over T's key range repeats this step);
+//   4  every CTA pushes its few keys of bin T into a flat array in all peers, plus
+//      its count of keys below T;
+//   5  cluster barrier; every CTA finds the threshold key by brute force over the
+//      <= 256 pushed keys and knows how many winners precede its slice;
+//   6  winners are written in ascending position order (deterministic, and the later
+//      gather walks the cache monotonically).
+// No global store precedes the first barrier (a release would wait for it); the
+// score output is regenerated from the keys between arrive and wait of the second.
 #include <cuda_bf16.h>
 
 #include <cstddef>
 
-#include "rkv_fold.cuh"
 #include "rkv_internal.h"
-
-namespace cg = cooperative_groups;
 
 namespace rkv {
 namespace {
 
 constexpr int NT = kSelectThreads;
-constexpr int kBins = 2048;        // pass over bits 30..20; later passes use 1024 of them
-constexpr int kCand = 2048;        // candidate pool (keys) kept in CTA 0
-constexpr uint32_t kWorstKey = 0x7fffffffu;
+constexpr int NW = NT / 32;
+constexpr int kBins = 2048;
+constexpr int kHistWords = kBins / 2;     // two 16-bit counters per word (a CTA holds at most 40960 keys)
+constexpr int kCandMax = 256;             // keys of the final bin that are resolved by brute force
+constexpr int kMaxPasses = 5;             // pass 0 + refinements of 11 bits each cover the 31-bit key
+constexpr int kOPre = 10;                 // partial-output values per thread fetched in the first round trip
+constexpr uint32_t kWorstKey = 0x7f800000u;   // bits of +inf: probability 0, or a NaN score
+constexpr uint32_t kPadKey = 0xffffffffu;     // filler behind a CTA's last key: never a winner, never in a bin
+constexpr float kLog2eF = 1.4426950408889634f;
+constexpr float kLn2F = 0.6931471805599453f;
+static_assert(kSelectMaxKeysPerCta < 65536, "packed 16-bit histogram counters");
+static_assert(kSelectCluster == 8 && NT == 512, "merge and finish assume 8 CTAs of 16 warps");
+static_assert(kMaxSplits <= 128, "four weight loads per lane cover every split");
 
 struct SelectShared {
-  alignas(16) uint32_t hist[3][kBins];   // one histogram per cluster-wide pass (kept: peers may still read them)
-  alignas(16) uint32_t cand[kCand];      // CTA 0: pooled candidates; every CTA: its local copy afterwards
-  alignas(16) uint32_t lhist[1024];      // local passes over the candidate pool
-  alignas(16) float w[kMaxSplits * 16];  // fold weights
-  alignas(16) float red[(NT / 32) * kHeadDim];
-  alignas(16) double lse[kMaxGroup];
-  alignas(16) float ML[16];
-  uint32_t warp_tot[NT / 32];
-  uint32_t peer_totals[kSelectCluster];  // per CTA of the cluster: keys below (low 16 bits) / equal to (high) the threshold key
-  uint32_t cand_count;                   // CTA 0 only: pool fill
-  uint32_t digit, want, count;
+  alignas(16) uint32_t hist[2][kHistWords];   // double-buffered: peers may still read the previous pass
+  alignas(16) uint32_t flat[kCandMax];        // final-bin keys of the whole cluster, in CTA order (pushed by peers)
+  alignas(16) float w[kMaxSplits * 8];        // w[s][h]: weight of split s for head h
+  alignas(16) float red[4][kHeadDim];
+  float lse[kMaxGroup], linv[kMaxGroup];
+  uint32_t below[kSelectCluster];             // pushed by CTA r: its keys below the final bin
+  uint32_t inbin[kSelectCluster];             // per CTA: its keys inside the located bin (from the merge)
+  uint32_t warp_a[NW];
+  uint32_t sel_bin, sel_want, sel_count;
+  uint32_t own_below, own_in, cand_fill;
+  uint32_t tau, ties, less_pre, eq_pre;
+  uint32_t bad;
 };
-static_assert(offsetof(SelectShared, red) % 16 == 0 && offsetof(SelectShared, hist) % 16 == 0, "vector access");
+static_assert(offsetof(SelectShared, hist) % 16 == 0 && offsetof(SelectShared, flat) % 16 == 0, "vector access");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -65,346 +81,469 @@ __device__ __forceinline__ uint4 ld_cluster_v4(uint32_t addr) {
   asm volatile("ld.shared::cluster.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ uint32_t ld_cluster(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
 __device__ __forceinline__ void st_cluster(uint32_t addr, uint32_t v) {
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
-__device__ __forceinline__ uint32_t atom_add_cluster(uint32_t addr, uint32_t v) {
-  uint32_t old;
-  asm volatile("atom.shared::cluster.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
-  return old;
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Split cluster barrier: work placed between arrive and wait hides the barrier's latency.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float lg2f(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float max_nan(float a, float b) {   // NaN if either operand is NaN
+  float y;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(y) : "f"(a), "f"(b));
+  return y;
+}
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
 }
 
-// exclusive block scan of one value per thread; *total receives the block sum
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* warp_tot, uint32_t* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t inc = v;
+// After a cluster barrier: merge hist[buf] of the eight CTAs and locate the bin that holds the
+// want-th smallest key.  Leaves sel_bin / sel_want (rank inside the bin) / sel_count (bin size) and
+// inbin[r] (CTA r's share of the bin) in shared memory.
+__device__ __forceinline__ void merge_locate(SelectShared* sh, int buf, uint32_t want) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t m[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+  uint4 v[kSelectCluster];
+  if (tid < kHistWords / 4) {
+    const uint32_t local = smem_u32(&sh->hist[buf][tid * 4]);
+#pragma unroll
+    for (int r = 0; r < kSelectCluster; ++r) v[r] = ld_cluster_v4(map_rank(local, r));
+#pragma unroll
+    for (int r = 0; r < kSelectCluster; ++r) {
+      m[0] += v[r].x & 0xffffu; m[1] += v[r].x >> 16;
+      m[2] += v[r].y & 0xffffu; m[3] += v[r].y >> 16;
+      m[4] += v[r].z & 0xffffu; m[5] += v[r].z >> 16;
+      m[6] += v[r].w & 0xffffu; m[7] += v[r].w >> 16;
+    }
+  }
+  uint32_t sum = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) sum += m[i];
+  uint32_t inc = sum;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= o) inc += t;
   }
-  if (lane == 31) warp_tot[warp] = inc;
+  if (lane == 31) sh->warp_a[warp] = inc;
   __syncthreads();
-  uint32_t base = 0, tot = 0;
+  if (tid < kHistWords / 4) {
+    uint32_t base = 0;
 #pragma unroll
-  for (int w = 0; w < NT / 32; ++w) {
-    const uint32_t t = warp_tot[w];
-    if (w < warp) base += t;
-    tot += t;
-  }
-  __syncthreads();
-  *total = tot;
-  return base + inc - v;
-}
-
-// Given a histogram of kB bins (4 per thread held in `mine`), find the bin holding the want-th
-// smallest element; results in sh->digit / sh->want (rank inside the bin) / sh->count (bin size).
-__device__ __forceinline__ void locate(SelectShared* sh, const uint32_t (&mine)[4], uint32_t want) {
-  const int tid = threadIdx.x;
-  const uint32_t sum = mine[0] + mine[1] + mine[2] + mine[3];
-  uint32_t total;
-  const uint32_t excl = block_excl_scan(sum, sh->warp_tot, &total);
-  if (excl < want && want <= excl + sum) {
-    uint32_t run = excl;
+    for (int w2 = 0; w2 < kHistWords / 128; ++w2)
+      if (w2 < warp) base += sh->warp_a[w2];
+    const uint32_t excl = base + inc - sum;
+    if (excl < want && want <= excl + sum) {   // exactly one thread
+      uint32_t run = excl;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      if (run < want && want <= run + mine[i]) {
-        sh->digit = tid * 4 + i;
-        sh->want = want - run;
-        sh->count = mine[i];
+      for (int i = 0; i < 8; ++i) {
+        if (run < want && want <= run + m[i]) {
+          sh->sel_bin = tid * 8 + i;
+          sh->sel_want = want - run;
+          sh->sel_count = m[i];
+#pragma unroll
+          for (int r = 0; r < kSelectCluster; ++r) {
+            const uint32_t word = (i >> 1) == 0 ? v[r].x : (i >> 1) == 1 ? v[r].y : (i >> 1) == 2 ? v[r].z : v[r].w;
+            sh->inbin[r] = (i & 1) ? (word >> 16) : (word & 0xffffu);
+          }
+        }
+        run += m[i];
       }
-      run += mine[i];
     }
   }
   __syncthreads();
 }
 
-// cluster-wide pass: every CTA has filled sh->hist[pass]; merge the 8 copies and locate the bin
-__device__ __forceinline__ void cluster_pass(cg::cluster_group& cluster, SelectShared* sh, int pass, int bins,
-                                             uint32_t want) {
-  cluster.sync();
-  const int tid = threadIdx.x;
-  uint32_t mine[4] = {0u, 0u, 0u, 0u};
-  if (tid * 4 < bins) {
-    const uint32_t local = smem_u32(&sh->hist[pass][tid * 4]);
-#pragma unroll
-    for (int r = 0; r < kSelectCluster; ++r) {
-      const uint4 v = ld_cluster_v4(map_rank(local, r));
-      mine[0] += v.x;
-      mine[1] += v.y;
-      mine[2] += v.z;
-      mine[3] += v.w;
-    }
-  }
-  locate(sh, mine, want);
-}
-
-// local pass over the candidate pool: digits (key >> shift) & 1023 of candidates whose bits above match `prefix`
-__device__ __forceinline__ void local_pass(SelectShared* sh, int n_cand, uint32_t prefix, int prefix_shift, int shift,
-                                           uint32_t want) {
-  const int tid = threadIdx.x;
-  for (int i = tid; i < 1024; i += NT) sh->lhist[i] = 0;
-  __syncthreads();
-  for (int i = tid; i < n_cand; i += NT) {
-    const uint32_t key = sh->cand[i];
-    if ((key >> prefix_shift) == prefix) atomicAdd(&sh->lhist[(key >> shift) & 1023u], 1u);
-  }
-  __syncthreads();
-  uint32_t mine[4] = {0u, 0u, 0u, 0u};
-  if (tid * 4 < 1024) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) mine[i] = sh->lhist[tid * 4 + i];
-  }
-  locate(sh, mine, want);
-}
-
-template <int GMAX>
+template <int GP>   // floats per position in the logit scratch: 4 (G <= 4) or 8
 __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  cg::cluster_group cluster = cg::this_cluster();
-  const int rank = (int)cluster.block_rank();
-  const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x;
-  pdl_launch();
-  pdl_wait();
-  if (p.active != nullptr && p.active[b] == 0) return;  // same decision in all CTAs of the cluster
-
+  const int rank = (int)cluster_rank();
+  const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   SelectShared* sh = reinterpret_cast<SelectShared*>(smem_raw);
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + ((sizeof(SelectShared) + 15) & ~size_t(15)));
-
+  pdl_launch();
+  for (int i = tid; i < 2 * kHistWords; i += NT) (&sh->hist[0][0])[i] = 0u;
+  if (tid == 0) {
+    sh->cand_fill = 0u;
+    sh->own_below = 0u;
+    sh->own_in = 0u;
+    sh->bad = 0u;
+  }
   const int G = p.group;
-  int n = p.len[b];
+  const int bg = b * p.n_kv_heads + g;
+  const int per = p.per_cta;                  // positions per CTA, fixed by the host from its length bound
+  const int lo = rank * per;
+  const float* pbase = p.partials + (int64_t)bg * p.max_splits * PartialLayout::kFloats;
+  const float* lg = p.logits + ((int64_t)bg * p.logit_stride + lo) * GP;
+  constexpr int U = 32 / GP;                  // positions per thread per round: all their loads are in flight together
+  const int gx = p.grid_splits;               // splits the attention launch had room for (>= the sequence's own count)
+  // slice of out[] this CTA folds: 16*G consecutive (head, channel) pairs of the group
+  const int o_local = tid & 127, sgrp = tid >> 7;
+  const bool o_on = o_local < 16 * G;
+  const int o_flat = rank * 16 * G + o_local;
+  const int64_t hrow0 = ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
+  pdl_wait();
+
+  // ---------------------------------------------------------------- 1: everything the kernel reads, in one round trip
+  const int act = (p.active != nullptr) ? __ldcg(p.active + b) : 1;
+  int n = __ldcg(p.len + b);
+  const int cap = __ldcg(p.cap + b);
+  int kk = __ldcg(p.k_small + b);
+  float wm[4], wl[4];                          // warps 0..7: (m, l) of head `warp` for splits lane, lane+32, ...
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int s = lane + 32 * k;
+    const bool on = warp < kMaxGroup && s < gx;
+    const float* ps = pbase + (int64_t)s * PartialLayout::kFloats + kMaxGroup * kHeadDim;
+    wm[k] = on ? __ldcg(ps + warp) : -INFINITY;
+    wl[k] = on ? __ldcg(ps + kMaxGroup + warp) : 0.f;
+  }
+  float opre[kOPre];
+#pragma unroll
+  for (int k = 0; k < kOPre; ++k) {
+    const int s = sgrp + 4 * k;
+    opre[k] = (o_on && s < gx) ? __ldcg(pbase + (int64_t)s * PartialLayout::kFloats + o_flat) : 0.f;
+  }
+  __nv_bfloat16 qv = __float2bfloat16(0.f);
+  if (p.q_last_full != nullptr && sgrp == 0 && o_on) qv = static_cast<const __nv_bfloat16*>(p.q)[hrow0 + o_flat];
+  float4 v[U][GP / 4];
+  auto load_round = [&](int i0) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * NT + tid;
+      const bool on = i < per && lo + i < p.logit_stride;
+#pragma unroll
+      for (int c = 0; c < GP / 4; ++c)
+        v[u][c] = on ? __ldcg(reinterpret_cast<const float4*>(lg + (int64_t)i * GP) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  load_round(0);
+
+  if (act == 0) return;   // same decision in all CTAs of the cluster
   {
-    const int cap = p.cap[b];
     const int lim = cap < p.max_len ? cap : p.max_len;
     if (n > lim) n = lim;
     if (n < 0) n = 0;
   }
-  int kk = p.k_small[b];
   if (kk > p.k_max) kk = p.k_max;
   if (kk > n) kk = n;
   if (kk < 0) kk = 0;
-  const int bg = b * p.n_kv_heads + g;
   int32_t* idx_out = p.topk_idx + (int64_t)bg * p.k_max;
-
-  // padding entries
-  for (int i = kk + rank * NT + tid; i < p.k_max; i += kSelectCluster * NT) idx_out[i] = -1;
-  if (n == 0) return;  // the attention kernel has zeroed out[]
-
-  // ---------------------------------------------------------------- fold the split partials
-  const int n_splits = (n + p.chunk - 1) / p.chunk;
-  const float* pbase = p.partials + (int64_t)bg * p.max_splits * PartialLayout::kFloats;
-  auto bar = [] { __syncthreads(); };
-  fold_weights<NT>(pbase, n_splits, tid, sh->w, sh->ML, bar);
-  if (tid < kMaxGroup) sh->lse[tid] = (double)sh->ML[tid] + log((double)sh->ML[8 + tid]);
-  if (rank < G) {  // CTA r writes the attention output of query head r of this group
-    fold_out<NT, 1>(pbase, n_splits, rank, 1, tid, sh->w, sh->red, bar);
-    const int64_t hrow = ((int64_t)b * p.n_q_heads + (int64_t)g * G + rank) * kHeadDim;
-    if (tid < kHeadDim) {
-      static_cast<__nv_bfloat16*>(p.out)[hrow + tid] = __float2bfloat16(sh->red[tid] / sh->ML[8 + rank]);
-      if (p.q_last_full != nullptr)
-        static_cast<__nv_bfloat16*>(p.q_last_full)[hrow + tid] = static_cast<const __nv_bfloat16*>(p.q)[hrow + tid];
-    }
-  }
-  for (int i = tid; i < kBins; i += NT) {
-    sh->hist[0][i] = 0;
-    sh->hist[1][i] = 0;
-    sh->hist[2][i] = 0;
-  }
-  if (tid == 0) sh->cand_count = 0;
-  __syncthreads();
-
-  int per = (n + kSelectCluster - 1) / kSelectCluster;
-  per = (per + 3) & ~3;
-  if (per > p.keys_per_cta) per = p.keys_per_cta;  // host guarantees this never bites
-  const int lo = (rank * per < n) ? rank * per : n;
-  const int hi = (lo + per < n) ? lo + per : n;
-  const int cnt = hi - lo;
-
-  // ---------------------------------------------------------------- keys (+ optional score output)
-  const float* lg = p.logits + (int64_t)bg * G * p.logit_stride;
-  float* sc = p.scores ? p.scores + (int64_t)bg * p.score_stride : nullptr;
-  bool bad = false;
-  const bool all_selected = (kk == n);
-  const int agg = p.agg;
-  double lse_r[GMAX];
-#pragma unroll
-  for (int h = 0; h < GMAX; ++h) lse_r[h] = sh->lse[h];
-  constexpr int U = 32 / GMAX;   // positions per thread per round: all their loads are in flight together
-  for (int i0 = 0; i0 < cnt; i0 += U * NT) {
-    float v[U][GMAX];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * NT + tid;
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h)
-        v[u][h] = (h < G && i < cnt && (agg != RKV_AGG_FIRST || h == 0))
-                      ? __ldcg(lg + (int64_t)h * p.logit_stride + lo + i)
-                      : 0.f;
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * NT + tid;
-      if (i >= cnt) continue;
-      double ell;
-      if (agg == RKV_AGG_MAX) {
-        ell = -INFINITY;
-#pragma unroll
-        for (int h = 0; h < GMAX; ++h) {
-          if (h < G) {
-            const double x = (double)v[u][h] - lse_r[h];
-            if (x != x) bad = true;
-            ell = fmax(ell, x);
-          }
-        }
-      } else if (agg == RKV_AGG_MEAN) {
-        double acc = 0.0;
-#pragma unroll
-        for (int h = 0; h < GMAX; ++h)
-          if (h < G) acc += exp((double)v[u][h] - lse_r[h]);
-        if (acc != acc) bad = true;
-        ell = log(acc / (double)G);
-      } else {
-        ell = (double)v[u][0] - lse_r[0];
-        if (ell != ell) bad = true;
-      }
-      uint32_t key;
-      if (ell != ell) {
-        key = kWorstKey;
-      } else {
-        const double uu = -ell * 16777216.0;
-        key = (uu <= 0.0) ? 0u : (uu >= 2147483647.0 ? kWorstKey : (uint32_t)uu);
-      }
-      keys[i] = key;
-      if (sc) sc[lo + i] = expf((float)ell);
-      if (!all_selected) atomicAdd(&sh->hist[0][key >> 20], 1u);
-    }
-  }
-  if (bad) atomicOr(p.status, RKV_DEV_NONFINITE);
-
-  if (all_selected) {  // K >= n: every position is kept (uniform over the cluster)
-    for (int i = tid; i < cnt; i += NT) idx_out[lo + i] = lo + i;
+  if (n == 0) {   // the attention kernel has zeroed out[]
+    for (int i = rank * NT + tid; i < p.k_max; i += kSelectCluster * NT) idx_out[i] = -1;
     return;
   }
-  if (kk == 0) return;  // nothing to select (uniform over the cluster); scores and out are written
+  const int cnt = (n - lo < 0) ? 0 : (n - lo < per ? n - lo : per);
+  const int R = (((cnt + NT - 1) / NT) + 3) & ~3;   // keys per thread in the ordered phases (multiple of 4)
+  const int cnt_pad = R * NT;
+  const bool all_selected = (kk == n);
+  const bool need_keys = (!all_selected && kk > 0) || p.scores != nullptr;
+  int n_splits = (n + p.chunk - 1) / p.chunk;
+  if (n_splits > gx) n_splits = gx;
 
-  // ---------------------------------------------------------------- locate the kk-th smallest key
-  // prefix = the key's bits above `shift` that are already fixed
-  cluster_pass(cluster, sh, 0, kBins, (uint32_t)kk);
-  uint32_t prefix = sh->digit, want = sh->want, count = sh->count;
-  int shift = 20;
-  int pass = 0;
-  while (count > (uint32_t)kCand && shift > 0) {  // crowded bin: refine by the next 10 bits, cluster-wide
-    ++pass;
-    const int nshift = shift - 10;
-    for (int i = tid; i < cnt; i += NT) {
-      const uint32_t key = keys[i];
-      if ((key >> shift) == prefix) atomicAdd(&sh->hist[pass][(key >> nshift) & 1023u], 1u);
+  // ---------------------------------------------------------------- log-sum-exp and split weights, one warp per head
+  if (warp < kMaxGroup) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (lane + 32 * k >= n_splits) wm[k] = -INFINITY;
+      M = fmaxf(M, wm[k]);
     }
-    cluster_pass(cluster, sh, pass, 1024, want);
-    prefix = (prefix << 10) | sh->digit;
-    want = sh->want;
-    count = sh->count;
-    shift = nshift;
+    M = warp_max_f(M);
+    float L = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float e = (wm[k] == -INFINITY) ? 0.f : ex2f((wm[k] - M) * kLog2eF);
+      L = fmaf(wl[k], e, L);
+      if (lane + 32 * k < kMaxSplits) sh->w[(lane + 32 * k) * 8 + warp] = e;
+    }
+    L = warp_sum_f(L);
+    if (lane == 0) {
+      sh->lse[warp] = M + logf(L);
+      sh->linv[warp] = 1.f / L;
+    }
   }
-  uint32_t tau, ties_to_take;
-  if (shift == 0) {  // fully resolved by histograms (only when > kCand keys are identical in all 31 bits... or share 21)
-    tau = prefix;
-    ties_to_take = want;
-  } else {
-    // pool the candidates (keys whose fixed bits match) in CTA 0, then finish locally in every CTA
-    const uint32_t pool = map_rank(smem_u32(&sh->cand[0]), 0);
-    const uint32_t pool_cnt = map_rank(smem_u32(&sh->cand_count), 0);
-    uint32_t mine_c = 0;
-    for (int i = tid; i < cnt; i += NT) mine_c += ((keys[i] >> shift) == prefix);
-    uint32_t tot_c;
-    uint32_t slot = block_excl_scan(mine_c, sh->warp_tot, &tot_c);
-    if (tid == 0) sh->digit = tot_c ? atom_add_cluster(pool_cnt, tot_c) : 0u;   // one reservation per CTA
+  __syncthreads();
+
+  // this CTA's slice of out[] (and of the trigger's reference query); run where it hides a cluster barrier
+  auto fold_slice = [&] {
+    const int h = o_flat >> 7;
+    float acc = 0.f;
+    if (o_on) {
+#pragma unroll
+      for (int k = 0; k < kOPre; ++k) {
+        const int s = sgrp + 4 * k;
+        if (s < n_splits) acc = fmaf(opre[k], sh->w[s * 8 + h], acc);
+      }
+      for (int s = sgrp + 4 * kOPre; s < n_splits; s += 4)
+        acc = fmaf(__ldcg(pbase + (int64_t)s * PartialLayout::kFloats + o_flat), sh->w[s * 8 + h], acc);
+    }
+    sh->red[sgrp][o_local] = acc;
     __syncthreads();
-    slot += sh->digit;
-    for (int i = tid; i < cnt && mine_c; i += NT) {
-      const uint32_t key = keys[i];
-      if ((key >> shift) == prefix) {
-        if (slot < (uint32_t)kCand) st_cluster(pool + 4 * slot, key);
-        ++slot;
+    if (sgrp == 0 && o_on) {
+      const float o = (sh->red[0][o_local] + sh->red[1][o_local]) + (sh->red[2][o_local] + sh->red[3][o_local]);
+      static_cast<__nv_bfloat16*>(p.out)[hrow0 + o_flat] = __float2bfloat16(o * sh->linv[h]);
+      if (p.q_last_full != nullptr) static_cast<__nv_bfloat16*>(p.q_last_full)[hrow0 + o_flat] = qv;
+    }
+    for (int i = kk + rank * NT + tid; i < p.k_max; i += kSelectCluster * NT) idx_out[i] = -1;   // padding
+  };
+  // score[j] = exp(ell[j]) regenerated from the keys (a NaN score has been flagged and reads as 0)
+  auto write_scores = [&] {
+    if (p.scores != nullptr) {
+      float* sc = p.scores + (int64_t)bg * p.score_stride + lo;
+      for (int i = tid; i < cnt; i += NT) sc[i] = ex2f(-__uint_as_float(keys[i]) * kLog2eF);
+    }
+    if (tid == 0 && sh->bad != 0u) atomicOr(p.status, RKV_DEV_NONFINITE);
+  };
+
+  // ---------------------------------------------------------------- 2: keys and the pass-0 histogram
+  if (need_keys) {
+    float lse_r[GP];
+#pragma unroll
+    for (int h = 0; h < GP; ++h) lse_r[h] = (h < G) ? sh->lse[h] : INFINITY;
+    const int agg = p.agg;
+    const float inv_g = 1.f / (float)G;
+    bool bad = false;
+    for (int i0 = 0; i0 < cnt_pad; i0 += U * NT) {
+      if (i0 > 0) load_round(i0);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * NT + tid;
+        if (i >= cnt_pad) continue;
+        const float* x = reinterpret_cast<const float*>(&v[u][0]);
+        float ell;
+        if (agg == RKV_AGG_MAX) {   // heads >= G carry LSE = +inf and drop out of the max
+          ell = x[0] - lse_r[0];
+#pragma unroll
+          for (int h = 1; h < GP; ++h) ell = max_nan(ell, x[h] - lse_r[h]);
+        } else if (agg == RKV_AGG_MEAN) {
+          float acc = 0.f;
+#pragma unroll
+          for (int h = 0; h < GP; ++h) acc += ex2f((x[h] - lse_r[h]) * kLog2eF);   // ex2(-inf) = 0 for heads >= G
+          ell = lg2f(acc * inv_g) * kLn2F;
+        } else {
+          ell = x[0] - lse_r[0];
+        }
+        uint32_t key = kPadKey;
+        if (i < cnt) {
+          uint32_t bin;
+          if (ell != ell) {
+            bad = true;
+            key = kWorstKey;
+            bin = kBins - 1;
+          } else {
+            const float nl = fmaxf(-ell, 0.f);
+            key = __float_as_uint(nl) & 0x7fffffffu;
+            bin = __float2uint_rz(fminf(nl * 64.f, (float)(kBins - 1)));
+          }
+          if (!all_selected) atomicAdd(&sh->hist[0][bin >> 1], 1u << ((bin & 1u) << 4));
+        }
+        keys[i] = key;
       }
     }
-    cluster.sync();
-    const int n_cand = (int)(count < (uint32_t)kCand ? count : (uint32_t)kCand);
-    if (rank != 0) {
-      for (int i = tid; i < n_cand; i += NT) sh->cand[i] = ld_cluster(pool + 4 * i);
-    }
-    __syncthreads();
-    while (shift > 0) {
-      const int nshift = shift - 10;
-      local_pass(sh, n_cand, prefix, shift, nshift, want);
-      prefix = (prefix << 10) | sh->digit;
-      want = sh->want;
-      shift = nshift;
-    }
-    tau = prefix;
-    ties_to_take = want;
+    if (bad) sh->bad = 1u;
   }
 
-  // ---------------------------------------------------------------- ordered output
-  // thread t owns positions t, t + NT, ... of a block of NT*? no: contiguous runs keep the order simple
-  const int run = (cnt + NT - 1) / NT;
-  const int r_lo = (tid * run < cnt) ? tid * run : cnt;
-  const int r_hi = (r_lo + run < cnt) ? r_lo + run : cnt;
-  uint32_t c_less = 0, c_eq = 0;
-  for (int i = r_lo; i < r_hi; ++i) {
-    const uint32_t key = keys[i];
-    c_less += (key < tau);
-    c_eq += (key == tau);
+  if (all_selected || kk == 0) {   // uniform over the cluster: nothing to choose
+    __syncthreads();
+    fold_slice();
+    write_scores();
+    if (all_selected)
+      for (int i = tid; i < cnt; i += NT) idx_out[lo + i] = lo + i;
+    return;
   }
-  // counts fit 16 bits each (at most 40960 keys per CTA): one packed scan gives both prefixes
-  uint32_t tot_packed;
-  const uint32_t e_packed = block_excl_scan(c_less | (c_eq << 16), sh->warp_tot, &tot_packed);
-  const uint32_t e_less = e_packed & 0xffffu, e_eq = e_packed >> 16;
-  if (tid < kSelectCluster) {  // push this CTA's totals to every peer: no remote read is needed later
-    const uint32_t dst = map_rank(smem_u32(&sh->peer_totals[rank]), tid);
-    st_cluster(dst, tot_packed);
-  }
-  cluster.sync();
-  uint32_t ties_before = 0, winners_before = 0, my_quota = 0;
-  for (int r = 0; r <= rank; ++r) {
-    const uint32_t t = sh->peer_totals[r];
-    const uint32_t less_r = t & 0xffffu, eq_r = t >> 16;
-    const uint32_t left = ties_to_take > ties_before ? ties_to_take - ties_before : 0u;
-    const uint32_t take = left < eq_r ? left : eq_r;
-    if (r < rank) {
-      winners_before += less_r + take;
-      ties_before += eq_r;
+
+  // ---------------------------------------------------------------- 3: locate the bin of the kk-th smallest key
+  uint32_t lo_key = 0u, hi_key = kWorstKey, want = (uint32_t)kk, count = 0u;
+  int shb = 0;
+  for (int pass = 0; pass < kMaxPasses; ++pass) {
+    if (pass > 0) {   // refine inside [lo_key, hi_key]: bins of 2^shb key values
+      const uint32_t span = hi_key - lo_key;
+      shb = 32 - __clz(span) - 11;
+      if (shb < 0) shb = 0;
+      uint32_t* h = sh->hist[pass & 1];
+      for (int i = tid; i < kHistWords; i += NT) h[i] = 0u;
+      __syncthreads();
+      for (int i = tid; i < cnt; i += NT) {
+        const uint32_t key = keys[i];
+        if (key >= lo_key && key <= hi_key) {
+          const uint32_t bin = (key - lo_key) >> shb;
+          atomicAdd(&h[bin >> 1], 1u << ((bin & 1u) << 4));
+        }
+      }
+    }
+    cluster_arrive();
+    if (pass == 0) fold_slice();
+    cluster_wait();
+    merge_locate(sh, pass & 1, want);
+    const uint32_t T = sh->sel_bin;
+    want = sh->sel_want;
+    count = sh->sel_count;
+    if (pass == 0) {   // bin T of pass 0 is  T/64 <= -ell < (T+1)/64  (the last bin is open-ended)
+      lo_key = __float_as_uint((float)T * (1.f / 64.f));
+      hi_key = (T == kBins - 1) ? kWorstKey : __float_as_uint((float)(T + 1) * (1.f / 64.f)) - 1u;
     } else {
-      my_quota = take;
+      lo_key = lo_key + (T << shb);
+      const uint32_t top = lo_key + ((1u << shb) - 1u);
+      hi_key = top < hi_key ? top : hi_key;
+    }
+    if (count <= (uint32_t)kCandMax || lo_key == hi_key) break;
+  }
+  // count > kCandMax here means the bin is a single key value shared by all its members
+  const bool ident = count > (uint32_t)kCandMax;
+
+  // ---------------------------------------------------------------- 4: exchange the final bin
+  uint32_t flat_base = 0;   // where this CTA's keys start in the flat array (CTA order)
+#pragma unroll
+  for (int r = 0; r < kSelectCluster; ++r)
+    if (r < rank) flat_base += sh->inbin[r];
+  const uint4* my_keys = reinterpret_cast<const uint4*>(keys + (size_t)tid * R);   // thread t owns keys [t*R, (t+1)*R)
+  {
+    uint32_t c_below = 0;
+    const uint32_t flat0 = smem_u32(&sh->flat[0]);
+    for (int j = 0; j < R / 4; ++j) {
+      const uint4 k4 = my_keys[j];
+      const uint32_t kv[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        c_below += (kv[e] < lo_key);
+        if (!ident && kv[e] >= lo_key && kv[e] <= hi_key) {   // rare: a handful per CTA
+          const uint32_t slot = flat_base + atomicAdd(&sh->cand_fill, 1u);
+          if (slot < (uint32_t)kCandMax) {
+#pragma unroll
+            for (int r = 0; r < kSelectCluster; ++r) st_cluster(map_rank(flat0 + 4u * slot, r), kv[e]);
+          }
+        }
+      }
+    }
+    c_below = warp_sum(c_below);
+    if (lane == 0 && c_below != 0u) atomicAdd(&sh->own_below, c_below);
+  }
+  __syncthreads();
+  if (tid < kSelectCluster) st_cluster(map_rank(smem_u32(&sh->below[rank]), tid), sh->own_below);
+  cluster_arrive();
+  write_scores();
+  cluster_wait();
+  // from here on nobody touches a peer's shared memory
+
+  // ---------------------------------------------------------------- 5: threshold key; winners before this slice
+  if (ident) {
+    if (tid == 0) {
+      sh->tau = lo_key;
+      sh->ties = want;
+      sh->less_pre = 0u;
+      sh->eq_pre = flat_base;
+    }
+  } else {
+    // P threads share one candidate (P = 512 / 256): each counts over half of the flat array
+    const int ci = tid >> 1, part = tid & 1;
+    const int half = ((int)count + 1) >> 1;
+    const int j0 = part * half, j1 = (j0 + half < (int)count) ? j0 + half : (int)count;
+    const uint32_t c = (ci < (int)count) ? sh->flat[ci] : 0u;
+    uint32_t less = 0, eq = 0, less_p = 0, eq_p = 0;
+    for (int j = j0; j < j1; ++j) {
+      const uint32_t x = sh->flat[j];
+      const bool pre = j < (int)flat_base;
+      less += (x < c);
+      eq += (x == c);
+      less_p += (pre && x < c);
+      eq_p += (pre && x == c);
+    }
+    less += __shfl_xor_sync(0xffffffffu, less, 1);
+    eq += __shfl_xor_sync(0xffffffffu, eq, 1);
+    less_p += __shfl_xor_sync(0xffffffffu, less_p, 1);
+    eq_p += __shfl_xor_sync(0xffffffffu, eq_p, 1);
+    if (part == 0 && ci < (int)count && less < want && want <= less + eq) {
+      // every thread that holds the threshold value writes the same four numbers
+      sh->tau = c;
+      sh->ties = want - less;
+      sh->less_pre = less_p;
+      sh->eq_pre = eq_p;
     }
   }
-  // ties are kept in position order, so min(e_eq, quota) of them precede this thread's run
-  uint32_t offs = winners_before + e_less + (e_eq < my_quota ? e_eq : my_quota);
-  uint32_t eq_seen = e_eq;
-  for (int i = r_lo; i < r_hi; ++i) {
-    const uint32_t key = keys[i];
-    bool win = key < tau;
-    if (key == tau) {
-      win = eq_seen < my_quota;
-      ++eq_seen;
-    }
-    if (win) {
-      if (offs < (uint32_t)kk) idx_out[offs] = lo + i;
-      ++offs;
+  __syncthreads();
+  const uint32_t tau = sh->tau, ties_to_take = sh->ties;
+  uint32_t winners_before = sh->less_pre + (sh->eq_pre < ties_to_take ? sh->eq_pre : ties_to_take);
+#pragma unroll
+  for (int r = 0; r < kSelectCluster; ++r)
+    if (r < rank) winners_before += sh->below[r];
+  const uint32_t ties_before = sh->eq_pre;
+
+  // ---------------------------------------------------------------- 6: ordered output
+  uint32_t c_less = 0, c_eq = 0;
+  for (int j = 0; j < R / 4; ++j) {
+    const uint4 k4 = my_keys[j];
+    c_less += (k4.x < tau) + (k4.y < tau) + (k4.z < tau) + (k4.w < tau);
+    c_eq += (k4.x == tau) + (k4.y == tau) + (k4.z == tau) + (k4.w == tau);
+  }
+  // exclusive block scan of both counts at once (each total fits 16 bits)
+  const uint32_t packed = c_less | (c_eq << 16);
+  uint32_t inc = packed;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) sh->warp_a[warp] = inc;
+  __syncthreads();
+  uint32_t wbase = (lane < warp) ? sh->warp_a[lane] : 0u;   // NW = 16 <= 32 lanes
+  wbase = warp_sum(wbase);
+  const uint32_t excl = wbase + inc - packed;
+  const uint32_t e_less = excl & 0xffffu;
+  uint32_t eq_seen = ties_before + (excl >> 16);
+  // ties are kept in position order: the first ties_to_take of them (cluster-wide) win
+  uint32_t offs = winners_before + e_less +
+                  ((eq_seen < ties_to_take ? eq_seen : ties_to_take) - (ties_before < ties_to_take ? ties_before : ties_to_take));
+  const int i_base = tid * R;
+  for (int j = 0; j < R / 4; ++j) {
+    const uint4 k4 = my_keys[j];
+    const uint32_t kv[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      bool win = kv[e] < tau;
+      if (kv[e] == tau) {
+        win = eq_seen < ties_to_take;
+        ++eq_seen;
+      }
+      if (win) {
+        if (offs < (uint32_t)kk) idx_out[offs] = lo + i_base + 4 * j + e;
+        ++offs;
+      }
     }
   }
-  // no cluster barrier here: after the one above nobody touches a peer's shared memory any more
 }
 
 }  // namespace
 
 size_t select_smem_bytes(int keys_per_cta) {
-  return ((sizeof(SelectShared) + 15) & ~size_t(15)) + (size_t)keys_per_cta * 4;
+  const size_t padded = ((size_t)keys_per_cta + 4 * NT - 1) / (4 * NT) * (4 * NT);   // R * NT keys, R a multiple of 4
+  return ((sizeof(SelectShared) + 15) & ~size_t(15)) + padded * 4;
 }
 
 cudaError_t prepare_select() {
@@ -418,8 +557,8 @@ cudaError_t prepare_select() {
 cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st) {
   const dim3 grid(kSelectCluster, p.n_kv_heads, n_seq);
   if (p.group <= 4)
-    return launch_ex(select_kernel<4>, grid, dim3(NT), select_smem_bytes(p.keys_per_cta), st, kSelectCluster, p);
-  return launch_ex(select_kernel<8>, grid, dim3(NT), select_smem_bytes(p.keys_per_cta), st, kSelectCluster, p);
+    return launch_ex(select_kernel<4>, grid, dim3(NT), select_smem_bytes(p.per_cta), st, kSelectCluster, p);
+  return launch_ex(select_kernel<8>, grid, dim3(NT), select_smem_bytes(p.per_cta), st, kSelectCluster, p);
 }
 
 }  // namespace rkv

@@ -23,7 +23,7 @@ EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", 
            "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
            "rkv_set_option", "rkv_small_step_noalloc"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
-OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH = 1, 2
+OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER = 1, 2, 3
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
 
 

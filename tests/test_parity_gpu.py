@@ -131,9 +131,11 @@ def test_aggregation_modes(mods, agg, name):
     check_full_against_oracle(st, cache, q, lens, k_small, 4, agg=name)
 
 
-def test_small_step_and_K_equals_L_invariant(mods):
+@pytest.mark.parametrize("cluster", [1, 0])
+def test_small_step_and_K_equals_L_invariant(mods, cluster):
     lens = [640, 200]
     ctx, st, cache, q = make_layer(mods, lens, list(lens), 8, 2, seed=9)
+    ctx.set_option(mods[0].OPT_SMALL_CLUSTER, cluster)   # both ways of merging the splits
     full_out = st.refresh(q).clone()
     small_out = st.partial(q).clone()
     assert ctx.device_status() == 0
@@ -144,21 +146,36 @@ def test_small_step_and_K_equals_L_invariant(mods):
         check_out(full_out[b], out, "full step")
 
 
-def test_small_step_on_a_selected_subset(mods):
+@pytest.mark.parametrize("cluster,n_q,n_kv", [(1, 32, 8), (0, 32, 8), (1, 28, 4), (1, 8, 1)])
+def test_small_step_on_a_selected_subset(mods, cluster, n_q, n_kv):
     lens, k_small = [3000, 1111], [300, 64]
-    ctx, st, cache, q = make_layer(mods, lens, k_small, 32, 8, seed=10)
+    ctx, st, cache, q = make_layer(mods, lens, k_small, n_q, n_kv, seed=10)
+    ctx.set_option(mods[0].OPT_SMALL_CLUSTER, cluster)
     st.refresh(q)
     g = torch.Generator(device="cuda"); g.manual_seed(77)
     q2 = torch.randn(q.shape, generator=g, device="cuda").to(torch.bfloat16)
     small_out = st.partial(q2).clone()
     idx_host = st.topk_idx.cpu().numpy()
     for b, n in enumerate(lens):
-        kf, vf = host_heads(cache, b, 8, "k"), host_heads(cache, b, 8, "v")
-        sel = [idx_host[b, h, : k_small[b]] for h in range(8)]
+        kf, vf = host_heads(cache, b, n_kv, "k"), host_heads(cache, b, n_kv, "v")
+        sel = [idx_host[b, h, : k_small[b]] for h in range(n_kv)]
         ks = O.bf16_bits_to_f64(np.stack(O.gather_rows(kf, sel)))
         vs = O.bf16_bits_to_f64(np.stack(O.gather_rows(vf, sel)))
         out, _, _ = O.decode_attention(O.bf16_bits_to_f64(bits(q2[b])), ks, vs)
         check_out(small_out[b], out, f"small step seq {b}")
+
+
+@pytest.mark.parametrize("n_small", [1, 64, 65, 130, 200, 321, 700])
+def test_small_step_every_cluster_shape(mods, n_small):
+    """Small caches from one tile to several per CTA: 1, 2, 4 and 8 CTAs per head, some of them idle."""
+    lens = [n_small, max(1, n_small // 3)]
+    ctx, st, cache, q = make_layer(mods, lens, list(lens), 28, 4, seed=100 + n_small, poison=True)
+    st.refresh(q)
+    out = st.partial(q).clone()
+    assert ctx.device_status() == 0
+    for b, n in enumerate(lens):
+        want, _, _, _ = oracle_full(cache, b, n, q[b], 4, n)
+        check_out(out[b], want, f"small step n={n}")
 
 
 def test_append_and_overflow_flag(mods):
