@@ -3,7 +3,7 @@
 
 One "step" is one decode token through the attention work of ALL layers of the workload
 (default: Llama-3.1-8B attention shape, 32 layers, batch 1, L=32768, K=2048, fixed stride 10):
-per layer  rkv_append + (every 10th token) rkv_full_step + rkv_gather_small, else rkv_small_step.
+per layer  (every 10th token) rkv_append + rkv_full_step + rkv_gather_small, else rkv_append_small_step.
 Each token's launches are replayed from a CUDA graph (one graph per kind of token).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
@@ -239,11 +239,11 @@ def run_ours(args):
     def token(full: bool):
         for l, st in enumerate(layers):
             q, kn, vn = views[l]
-            st.append(kn, vn)
             if full:
+                st.append(kn, vn)
                 st.refresh(q, max_len_hint=max_len)
-            else:
-                st.partial(q, max_len_hint=K + STRIDE + 1)
+            else:      # append + partial step in one call (one launch)
+                st.append_partial(q, kn, vn, max_len_hint=K + STRIDE + 1)
 
     # initial small caches + eager warm-up of every kernel (also creates the tensor maps)
     stage.copy_(inputs_dev[0])
@@ -321,10 +321,13 @@ def run_ours(args):
     full_token_us = ms_full * 1000.0 / (20 * world)
     ms_small, _, nss = timed(STRIDE - 1, force_small=True)   # right after a full token: K .. K+8 rows
     run_tokens(1, always_full=True)
-    # ---- per-kernel device time: eager launches bracketed by events (same schedule, one period)
+    # ---- per-kernel device time: every launch bracketed by CUDA events on its stream (same schedule, two
+    # periods).  A spin kernel first keeps the GPU busy while the host enqueues, so that the launches sit
+    # back to back in the queue and an event pair measures the kernel, not the host's launch latency.
     torch.cuda.synchronize()
     ctx.set_profiling(True)
     ctx.get_profile()
+    torch.cuda._sleep(int(8e7))
     for _ in range(2 * STRIDE):
         t = tok_counter[0]; tok_counter[0] += 1
         stage.copy_(inputs_dev[t % n_in])

@@ -157,6 +157,21 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new,
                       const rkv_cache* small_cache /*host struct or NULL*/, void* stream);
 
 /*
+ * Append + PARTIAL step in one call (Sec. 2.2 "Decoding with partial cache": the step attends over
+ * C_p and stores the input token's K/V; C_f receives the pair as well).  Same result as
+ *   rkv_append(k_new, v_new, full, small_cache)  followed by  rkv_small_step(q, small_cache, active, out):
+ * every sequence (active or not) gets the new row in both caches and its lengths bumped; sequences with
+ * active[b] != 0 (NULL: all) attend over the small cache including the new row.  When the length bound
+ * allows the clustered partial step (see RKV_OPT_SMALL_CLUSTER) this is ONE kernel launch; otherwise the
+ * two kernels are launched back to back.  full may be NULL (only the small cache receives the row).
+ * max_len_hint bounds small->len[b] AFTER the append (0 = cfg.max_small).
+ */
+rkv_status rkv_append_small_step(rkv_ctx* ctx, const void* q, const void* k_new, const void* v_new,
+                                 const rkv_cache* full /*host struct or NULL*/,
+                                 const rkv_cache* small_cache /*host struct*/, const int32_t* active,
+                                 void* out, int32_t max_len_hint, void* stream);
+
+/*
  * Refresh trigger (Sec. 2.2 "Deciding when to decode with full cache").
  *   qbar  = mean over the Hq heads of q_now[b];  qbar' likewise from q_last_full[b]
  *   sim   = <qbar, qbar'> / (|qbar| |qbar'|)          (fp32)

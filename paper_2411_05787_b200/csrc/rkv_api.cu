@@ -36,7 +36,7 @@ int splits_for(const rkv_config* c) {
   return s < rkv::kMaxSplits ? (s < 1 ? 1 : s) : rkv::kMaxSplits;
 }
 
-struct WsLayout { size_t partials, tickets, logits, status, total; int64_t logit_stride; };
+struct WsLayout { size_t partials, tickets, len_tickets, logits, status, total; int64_t logit_stride; };
 
 WsLayout ws_layout(const rkv_config* c) {
   WsLayout w;
@@ -47,6 +47,7 @@ WsLayout ws_layout(const rkv_config* c) {
   size_t off = 0;
   w.partials = off; off = up(off + bg * splits_for(c) * rkv::PartialLayout::kFloats * sizeof(float));
   w.tickets = off;  off = up(off + bg * sizeof(int32_t));
+  w.len_tickets = off; off = up(off + (size_t)c->n_seq * sizeof(int32_t));
   const int gp = group <= 4 ? 4 : 8;   // position-major logits, padded to a vector width
   w.logits = off;   off = up(off + bg * gp * (size_t)w.logit_stride * sizeof(float));
   w.status = off;   off = up(off + sizeof(int32_t));
@@ -144,8 +145,13 @@ int choose_chunk(const rkv_ctx* ctx, int n_max, bool full, int* grid_x) {
 // Longest small cache that the clustered partial step takes (8 CTAs x 1024 positions).
 constexpr int kClusterMaxLen = 8192;
 
+struct AppendArgs { const void* k_new; const void* v_new; const rkv_cache* full; };
+
+bool cluster_eligible(const rkv_ctx* ctx, int n_max) { return ctx->small_cluster != 0 && n_max <= kClusterMaxLen; }
+
 rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
-                         int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out, int* gx_out) {
+                         int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out, int* gx_out,
+                         const AppendArgs* app = nullptr) {
   CUtensorMap tm_k, tm_v;
   rkv_status s = tensor_map(ctx, cache->k, cache->n_rows, &tm_k);
   if (s != RKV_OK) return s;
@@ -154,7 +160,7 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   AttnParams p;
   memset(&p, 0, sizeof(p));
   int gx = 1;
-  const bool cluster = !logits && ctx->small_cluster != 0 && n_max <= kClusterMaxLen;
+  const bool cluster = !logits && cluster_eligible(ctx, n_max);
   if (cluster) {   // 1, 2, 4 or 8 CTAs per (sequence, KV head), whole tiles each
     const int tiles = (n_max + rkv::kTile - 1) / rkv::kTile;
     gx = tiles >= 5 ? 8 : tiles >= 3 ? 4 : tiles >= 2 ? 2 : 1;
@@ -182,11 +188,29 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.max_splits = ctx->max_splits;
   p.max_len = limit;
   p.scale = ctx->cfg.softmax_scale;
+  if (app != nullptr) {   // only the clustered partial step takes the append with it
+    if (!cluster) return RKV_ERR_INVALID_ARG;
+    p.k_new = app->k_new;
+    p.v_new = app->v_new;
+    p.small_k = cache->k;
+    p.small_v = cache->v;
+    p.small_len = cache->len;
+    p.len_tickets = ctx->len_tickets;
+    p.has_full = app->full != nullptr;
+    if (app->full != nullptr) {
+      p.full_k = app->full->k;
+      p.full_v = app->full->v;
+      p.full_row_offset = app->full->row_offset;
+      p.full_cap = app->full->cap;
+      p.full_len = app->full->len;
+    }
+  }
   cudaError_t e;
   {
     LaunchScope scope(ctx, st, logits ? RKV_KERNEL_ATTN_FULL : RKV_KERNEL_ATTN_SMALL);
-    e = cluster ? rkv::launch_attention_cluster(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
-                : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
+    e = app != nullptr ? rkv::launch_attention_cluster_append(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
+        : cluster      ? rkv::launch_attention_cluster(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
+                       : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
   ctx->launches += 1;
@@ -241,6 +265,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->workspace_bytes = w.total;
   ctx->partials = reinterpret_cast<float*>(ctx->workspace + w.partials);
   ctx->tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.tickets);
+  ctx->len_tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.len_tickets);
   ctx->logits = reinterpret_cast<float*>(ctx->workspace + w.logits);
   ctx->status = reinterpret_cast<int32_t*>(ctx->workspace + w.status);
   ctx->logit_stride = w.logit_stride;
@@ -330,6 +355,23 @@ rkv_status rkv_small_step(rkv_ctx* ctx, const void* q, const rkv_cache* small_ca
   if (n_max < 1 || n_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
   return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, static_cast<cudaStream_t>(stream),
                        nullptr, nullptr);
+}
+
+rkv_status rkv_append_small_step(rkv_ctx* ctx, const void* q, const void* k_new, const void* v_new,
+                                 const rkv_cache* full, const rkv_cache* small_cache, const int32_t* active,
+                                 void* out, int32_t max_len_hint, void* stream) {
+  if (!ctx || !q || !k_new || !v_new || !cache_ok(small_cache) || !out) return RKV_ERR_INVALID_ARG;
+  if (full != nullptr && !cache_ok(full)) return RKV_ERR_INVALID_ARG;
+  int n_max = max_len_hint == 0 ? ctx->cfg.max_small : max_len_hint;
+  if (n_max < 1 || n_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cluster_eligible(ctx, n_max)) {   // one launch: the attention kernel appends
+    const AppendArgs app = {k_new, v_new, full};
+    return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, st, nullptr, nullptr, &app);
+  }
+  rkv_status s = rkv_append(ctx, k_new, v_new, full, small_cache, stream);
+  if (s != RKV_OK) return s;
+  return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, st, nullptr, nullptr);
 }
 
 rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const rkv_cache* full,

@@ -22,6 +22,10 @@
 //                  each CTA finishes 128/C channels of every head;
 //                  (b) long small caches: partials to the workspace, folded by the last
 //                  CTA of each (sequence, KV head) to arrive (atomic ticket, no spin).
+// The clustered partial step can also take the append with it (Sec. 2.2: the partial
+// step stores the input token's K/V in C_p, and C_f receives it too): the new rows are
+// written to both caches, patched into the shared-memory tile that covers the new
+// position, and the lengths are bumped by the last cluster of a sequence to finish.
 #include <cuda_bf16.h>
 
 #include "rkv_fold.cuh"
@@ -37,7 +41,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kOPad = 132;  // floats per head row in the merge buffer (bank spread)
 constexpr int kRecvFloats = kMaxGroup * kHeadDim + kAttnCluster * kMaxGroup * 2;   // pushed slices + (m, l) pairs
 
-enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2 };
+enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2, kModeClusterAppend = 3 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -116,6 +120,9 @@ __device__ __forceinline__ uint32_t map_rank(uint32_t local_addr, int rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
 }
+__device__ __forceinline__ void st_shared_v2(uint32_t addr, uint2 v) {
+  asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(v.x), "r"(v.y) : "memory");
+}
 __device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
@@ -129,6 +136,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
             const AttnParams p) {
   constexpr bool kLogits = (kMode == kModeFull);
+  constexpr bool kCluster = (kMode == kModeCluster || kMode == kModeClusterAppend);
+  constexpr bool kAppend = (kMode == kModeClusterAppend);
   extern __shared__ uint8_t smem_raw[];
   __shared__ int s_last;
 
@@ -177,7 +186,61 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       }
     }
   }
-  if (act == 0) return;   // the same for every CTA of a cluster
+  // fused append: this lane's 8 bytes of the new K and V rows, and the second cache's sizes
+  uint2 kn = make_uint2(0u, 0u), vn = make_uint2(0u, 0u);
+  int pos_new = -1;            // where the new row lands in the attended cache (-1: no room, or no append)
+  int new_len_s = -1, new_len_f = -1;
+  if (kAppend) {
+    int len_f = 0, cap_f = 0;
+    int64_t roff_f = 0;
+    if (p.has_full) {
+      len_f = __ldcg(p.full_len + b);
+      cap_f = __ldcg(p.full_cap + b);
+      roff_f = __ldcg(p.full_row_offset + b);
+    }
+    if (warp < 4) {
+      const int64_t nrow = ((int64_t)b * p.n_kv_heads + g) * 32;   // uint2 units: 256 bytes per row
+      kn = __ldcg(static_cast<const uint2*>(p.k_new) + nrow + lane);
+      vn = __ldcg(static_cast<const uint2*>(p.v_new) + nrow + lane);
+    }
+    const bool ok_s = n >= 0 && n < cap;
+    const bool ok_f = p.has_full && len_f >= 0 && len_f < cap_f;
+    if (split == 0 && warp == 0) {   // one warp per (sequence, KV head) writes the rows to global memory
+      if (ok_s) {
+        const int64_t row = (roff + (int64_t)g * cap + n) * 32;
+        static_cast<uint2*>(p.small_k)[row + lane] = kn;
+        static_cast<uint2*>(p.small_v)[row + lane] = vn;
+      }
+      if (ok_f) {
+        const int64_t row = (roff_f + (int64_t)g * cap_f + len_f) * 32;
+        static_cast<uint2*>(p.full_k)[row + lane] = kn;
+        static_cast<uint2*>(p.full_v)[row + lane] = vn;
+      }
+      if (lane == 0 && (!ok_s || (p.has_full && !ok_f))) atomicOr(p.status, RKV_DEV_APPEND_OVERFLOW);
+    }
+    new_len_s = ok_s ? n + 1 : -1;
+    new_len_f = ok_f ? len_f + 1 : -1;
+    if (ok_s) {
+      pos_new = n;
+      n = n + 1;
+    }
+  }
+  // Fused append: the lengths are bumped by the last (sequence, KV head) cluster to get here.  Every cluster
+  // has read the old lengths before it takes its ticket, so nobody can still see them change.
+  auto take_len_ticket = [&] {
+    if (kAppend && split == 0 && tid == 0) {
+      const int old = atomicAdd(p.len_tickets + b, 1);
+      if (old == p.n_kv_heads - 1) {
+        if (new_len_s >= 0) p.small_len[b] = new_len_s;
+        if (new_len_f >= 0) p.full_len[b] = new_len_f;
+        p.len_tickets[b] = 0;   // ready for the next call on this stream
+      }
+    }
+  };
+  if (act == 0) {   // the same for every CTA of a cluster
+    take_len_ticket();
+    return;
+  }
   {
     const int lim = cap < p.max_len ? cap : p.max_len;
     if (n > lim) {
@@ -189,10 +252,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   if (n == 0) {  // nothing cached: the output is defined as zero
     if (split == 0 && tid < kHeadDim)
       for (int h = 0; h < G; ++h) out[h * kHeadDim + tid] = __float2bfloat16(0.f);
+    take_len_ticket();
     return;
   }
   const int start = split * p.chunk;
-  if (kMode != kModeCluster && start >= n) return;   // in a cluster an idle CTA still owns a slice of the output
+  if (!kCluster && start >= n) return;   // in a cluster an idle CTA still owns a slice of the output
   const int end = (start + p.chunk < n) ? start + p.chunk : n;
   const int n_tiles = (end > start) ? (end - start + kTile - 1) / kTile : 0;
   const int n_splits = (n + p.chunk - 1) / p.chunk;
@@ -221,7 +285,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
       }
     }
-    if (kMode == kModeCluster) {   // stay until the peers have pushed: every warp of the cluster meets at one barrier
+    if (kCluster) {   // stay until the peers have pushed: every warp of the cluster meets at one barrier
       __syncwarp();
       cluster_sync_alive();
     }
@@ -252,6 +316,18 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       break;
     }
     const int pos_base = start + t * kTile + 16 * warp;
+    if (kAppend) {
+      // The tile came from global memory, where the new row may not have landed yet: the warp that owns the
+      // row writes it into the tile itself (same 128-byte swizzle as the copy engine uses).
+      const int rel = pos_new - (start + t * kTile);
+      if (rel >= 0 && rel < kTile && (rel >> 4) == warp) {
+        const uint32_t at = smem_base + s * kStageBytes + (lane >> 4) * kHalfBytes + rel * 128 +
+                            ((((lane & 15) >> 1) ^ (rel & 7)) << 4) + (lane & 1) * 8;
+        st_shared_v2(at, kn);
+        st_shared_v2(at + 2 * kHalfBytes, vn);
+        __syncwarp();
+      }
+    }
     if (pos_base < end) {
       const uint32_t kbase = smem_base + s * kStageBytes;
       float c[4] = {0.f, 0.f, 0.f, 0.f};
@@ -379,7 +455,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
 
   const int bg = b * p.n_kv_heads + g;
 
-  if (kMode == kModeCluster) {
+  if (kCluster) {
     // ---------------------------------------------- merge the CTAs of the cluster through shared memory
     const int C = (int)gridDim.x;                       // cluster size = CTAs per (sequence, KV head)
     const int dchunk = kHeadDim / C;                    // channels of every head that one CTA finishes
@@ -406,6 +482,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       }
     }
     cluster_sync_alive();
+    take_len_ticket();
     if (!ok) return;
     for (int item = d; item < G * dchunk; item += 128) {
       const int h = item / dchunk, dd = item - h * dchunk;
@@ -486,7 +563,9 @@ cudaError_t prepare_attention() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_kernel<kModeTicket>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_kernel<kModeCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  e = cudaFuncSetAttribute(attn_kernel<kModeCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_kernel<kModeClusterAppend>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
@@ -501,6 +580,13 @@ cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_
                                      int n_seq, int cluster, cudaStream_t st) {
   dim3 grid(cluster, p.n_kv_heads, n_seq);
   return launch_ex(attn_kernel<kModeCluster>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, cluster, tm_k, tm_v, p);
+}
+
+cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                            int n_seq, int cluster, cudaStream_t st) {
+  dim3 grid(cluster, p.n_kv_heads, n_seq);
+  return launch_ex(attn_kernel<kModeClusterAppend>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, cluster, tm_k,
+                   tm_v, p);
 }
 
 }  // namespace rkv

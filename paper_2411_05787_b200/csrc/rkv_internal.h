@@ -47,6 +47,15 @@ struct AttnParams {
   int32_t max_splits;
   int32_t max_len;            // clamp for len[b]
   float scale;
+  // fused append (clustered partial step only): the new token's rows and where they go
+  const void* k_new;          // bf16 [B][Hkv][128]
+  const void* v_new;
+  void* small_k; void* small_v;         // the cache being attended (same buffers the tensor maps describe)
+  int32_t* small_len;                   // [B] updated by the kernel
+  void* full_k; void* full_v;           // optional second cache that receives the rows
+  const int64_t* full_row_offset; const int32_t* full_cap; int32_t* full_len;
+  int32_t* len_tickets;       // [B] arrival counters of the (sequence, KV head) clusters
+  int32_t has_full;
 };
 
 struct SelectParams {
@@ -79,6 +88,8 @@ cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const
                              int n_seq, int grid_x, bool write_logits, cudaStream_t st);
 cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                      int n_seq, int cluster, cudaStream_t st);
+cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                            int n_seq, int cluster, cudaStream_t st);
 cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st);
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
@@ -142,6 +153,7 @@ struct rkv_ctx {
   size_t workspace_bytes;
   float* partials;
   int32_t* tickets;
+  int32_t* len_tickets;
   float* logits;
   int32_t* status;
   int64_t launches;

@@ -461,30 +461,38 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
       sh->eq_pre = flat_base;
     }
   } else {
-    // P threads share one candidate (P = 512 / 256): each counts over half of the flat array
-    const int ci = tid >> 1, part = tid & 1;
-    const int half = ((int)count + 1) >> 1;
-    const int j0 = part * half, j1 = (j0 + half < (int)count) ? j0 + half : (int)count;
-    const uint32_t c = (ci < (int)count) ? sh->flat[ci] : 0u;
-    uint32_t less = 0, eq = 0, less_p = 0, eq_p = 0;
-    for (int j = j0; j < j1; ++j) {
-      const uint32_t x = sh->flat[j];
-      const bool pre = j < (int)flat_base;
-      less += (x < c);
-      eq += (x == c);
-      less_p += (pre && x < c);
-      eq_p += (pre && x == c);
-    }
-    less += __shfl_xor_sync(0xffffffffu, less, 1);
-    eq += __shfl_xor_sync(0xffffffffu, eq, 1);
-    less_p += __shfl_xor_sync(0xffffffffu, less_p, 1);
-    eq_p += __shfl_xor_sync(0xffffffffu, eq_p, 1);
-    if (part == 0 && ci < (int)count && less < want && want <= less + eq) {
-      // every thread that holds the threshold value writes the same four numbers
-      sh->tau = c;
-      sh->ties = want - less;
-      sh->less_pre = less_p;
-      sh->eq_pre = eq_p;
+    // P threads share one candidate (P a power of two, P * count <= 512): each counts over 1/P of the flat array
+    int lp = 0;                                   // log2(P)
+    while (lp < 5 && ((int)count << (lp + 1)) <= NT) ++lp;
+    const int ci = tid >> lp, part = tid & ((1 << lp) - 1);
+    if (ci < (int)count) {                        // whole groups of P lanes take this branch together
+      const int len = ((int)count + (1 << lp) - 1) >> lp;
+      const int j0 = part * len, j1 = (j0 + len < (int)count) ? j0 + len : (int)count;
+      const uint32_t c = sh->flat[ci];
+      uint32_t less = 0, eq = 0, less_p = 0, eq_p = 0;
+#pragma unroll 4
+      for (int j = j0; j < j1; ++j) {
+        const uint32_t x = sh->flat[j];
+        const bool pre = j < (int)flat_base;
+        less += (x < c);
+        eq += (x == c);
+        less_p += (pre && x < c);
+        eq_p += (pre && x == c);
+      }
+      const uint32_t gmask = __activemask();
+      for (int o = 1; o < (1 << lp); o <<= 1) {
+        less += __shfl_xor_sync(gmask, less, o);
+        eq += __shfl_xor_sync(gmask, eq, o);
+        less_p += __shfl_xor_sync(gmask, less_p, o);
+        eq_p += __shfl_xor_sync(gmask, eq_p, o);
+      }
+      if (part == 0 && less < want && want <= less + eq) {
+        // every thread that holds the threshold value writes the same four numbers
+        sh->tau = c;
+        sh->ties = want - less;
+        sh->less_pre = less_p;
+        sh->eq_pre = eq_p;
+      }
     }
   }
   __syncthreads();

@@ -21,7 +21,7 @@ DEV_APPEND_OVERFLOW, DEV_LEN_CLAMPED, DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT 
 EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", "rkv_gather_small",
            "rkv_small_step", "rkv_append", "rkv_should_refresh", "rkv_get_device_status",
            "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
-           "rkv_set_option", "rkv_small_step_noalloc"]
+           "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER = 1, 2, 3
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
@@ -53,6 +53,8 @@ def _load() -> ctypes.CDLL:
     lib.rkv_gather_small.argtypes = [vp, vp, vp, i32, cachep, cachep, vp, vp]
     lib.rkv_small_step.argtypes = [vp, vp, cachep, vp, vp, i32, vp]
     lib.rkv_append.argtypes = [vp, vp, vp, cachep, cachep, vp]
+    lib.rkv_append_small_step.argtypes = [vp, vp, vp, vp, cachep, cachep, vp, vp, i32, vp]
+    lib.rkv_append_small_step.restype = i32
     lib.rkv_should_refresh.argtypes = [vp, vp, vp, f32, vp, vp, vp]
     lib.rkv_get_device_status.argtypes = [vp, ctypes.POINTER(i32), vp]
     lib.rkv_status_string.argtypes = [i32]
@@ -175,6 +177,12 @@ class Context:
         self._check(lib.rkv_append(self._h, _ptr(k_new), _ptr(v_new),
                                    ctypes.byref(full) if full is not None else None,
                                    ctypes.byref(small) if small is not None else None, _stream(stream)))
+
+    def append_small_step(self, q, k_new, v_new, full: RkvCache | None, small: RkvCache, out, active=None,
+                          max_len_hint=0, stream=None):
+        self._check(lib.rkv_append_small_step(self._h, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                              ctypes.byref(full) if full is not None else None, ctypes.byref(small),
+                                              _ptr(active), _ptr(out), max_len_hint, _stream(stream)))
 
     def should_refresh(self, q_now, q_last_full, threshold, flag, sim=None, stream=None):
         self._check(lib.rkv_should_refresh(self._h, _ptr(q_now), _ptr(q_last_full), float(threshold), _ptr(flag),

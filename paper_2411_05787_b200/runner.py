@@ -48,6 +48,12 @@ class LayerState:
         self.ctx.small_step(q, self.small_c, self.out, active=active, max_len_hint=max_len_hint)
         return self.out
 
+    def append_partial(self, q, k_new, v_new, active=None, max_len_hint=0):
+        """Append to both caches and attend over the small cache, in one call."""
+        self.ctx.append_small_step(q, k_new, v_new, self.full_c, self.small_c, self.out, active=active,
+                                   max_len_hint=max_len_hint)
+        return self.out
+
     def append(self, k_new, v_new):
         self.ctx.append(k_new, v_new, self.full_c, self.small_c)
 

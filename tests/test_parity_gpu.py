@@ -178,6 +178,61 @@ def test_small_step_every_cluster_shape(mods, n_small):
         check_out(out[b], want, f"small step n={n}")
 
 
+@pytest.mark.parametrize("n_small", [0, 1, 63, 64, 127, 128, 320, 639, 640, 2047])
+def test_fused_append_small_step_equals_append_then_small_step(mods, n_small):
+    """rkv_append_small_step against the two separate calls on twin caches: same rows, lengths, flags, output.
+
+    The new row lands at tile and chunk boundaries, in an empty cache, and (third step) in a full one."""
+    rkv, runner, synth = mods
+    dev = torch.device("cuda")
+    n_q, n_kv, B = 28, 4, 3
+    lens_s, caps_s = [n_small, n_small // 2, 5], [n_small + 3, n_small // 2 + 2, 9]
+    lens_f, caps_f = [100, 40, 7], [102, 50, 9]
+    g = torch.Generator(device=dev); g.manual_seed(500 + n_small)
+
+    def twin():
+        sm = synth.alloc_cache(caps_s, lens_s, n_kv, dev)
+        fu = synth.alloc_cache(caps_f, lens_f, n_kv, dev)
+        return sm, fu
+    sm_a, fu_a = twin()
+    for t in (sm_a.k, sm_a.v, fu_a.k, fu_a.v):
+        t.copy_(torch.randn(t.shape, generator=g, device=dev).to(torch.bfloat16))
+    sm_b, fu_b = twin()
+    for x, y in ((sm_a, sm_b), (fu_a, fu_b)):
+        y.k.copy_(x.k); y.v.copy_(x.v)
+    ctx = rkv.Context(B, n_q, n_kv, max(caps_f), max(caps_s))
+    cs = lambda c: rkv.cache_struct(c.k, c.v, c.row_offset, c.cap, c.len)
+    sa, fa, sb, fb = cs(sm_a), cs(fu_a), cs(sm_b), cs(fu_b)
+    out_a = torch.zeros((B, n_q, 128), dtype=torch.bfloat16, device=dev)
+    out_b = torch.zeros_like(out_a)
+    active = torch.tensor([1, 0, 1], dtype=torch.int32, device=dev)
+    for step in range(3):
+        q = torch.randn((B, n_q, 128), generator=g, device=dev).to(torch.bfloat16)
+        kn = torch.randn((B, n_kv, 128), generator=g, device=dev).to(torch.bfloat16)
+        vn = torch.randn((B, n_kv, 128), generator=g, device=dev).to(torch.bfloat16)
+        out_a.fill_(3.0); out_b.fill_(3.0)
+        ctx.append_small_step(q, kn, vn, fa, sa, out_a, active=active)
+        bits_a = ctx.device_status()
+        ctx.append(kn, vn, fb, sb)
+        ctx.small_step(q, sb, out_b, active=active)
+        bits_b = ctx.device_status()
+        assert bits_a == bits_b, (step, bits_a, bits_b)
+        assert sm_a.len.tolist() == sm_b.len.tolist() and fu_a.len.tolist() == fu_b.len.tolist()
+        for x, y in ((sm_a, sm_b), (fu_a, fu_b)):
+            assert torch.equal(x.k, y.k) and torch.equal(x.v, y.v)
+        assert torch.equal(out_a, out_b), f"step {step}"
+        assert (out_a[1] == 3.0).all()      # inactive sequence: output untouched, but its caches grew
+        # and against the oracle, on the bytes now in the cache
+        for b in (0, 2):
+            n = int(sm_a.len[b])
+            k = O.bf16_bits_to_f64(host_heads(sm_a, b, n_kv, "k")[:, :n])
+            v = O.bf16_bits_to_f64(host_heads(sm_a, b, n_kv, "v")[:, :n])
+            want, _, _ = O.decode_attention(O.bf16_bits_to_f64(bits(q[b])), k, v)
+            check_out(out_a[b], want, f"fused step {step} seq {b}")
+    # the third step found sequence 0's full cache and sequence 2's caches at capacity
+    assert fu_a.len.tolist() == [102, 43, 9] and sm_a.len.tolist() == [n_small + 3, n_small // 2 + 2, 8]
+
+
 def test_append_and_overflow_flag(mods):
     rkv, runner, synth = mods
     lens, k_small = [40, 9], [8, 4]
@@ -306,7 +361,7 @@ def test_host_side_argument_errors(mods):
 
 
 # ----------------------------------------------------------------------------- the five workload configs
-def run_trajectory(mods, w, layer, seqs=None, check_every=1):
+def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False):
     """Run workload `w` for one layer on the GPU and step the oracle beside it on the same bytes."""
     rkv, runner, synth = mods
     dev = torch.device("cuda")
@@ -336,14 +391,17 @@ def run_trajectory(mods, w, layer, seqs=None, check_every=1):
             restore = synth.plant_heavy(w, cache, layer, qs[t], epoch=t // w.replant_every)
             for b in seqs:      # the oracle's copy of C_f follows the replanted rows
                 states[b].k_full[:, : w.lens[b]] = host_heads(cache, b, w.n_kv_heads, "k")[:, : w.lens[b]]
-        st.append(kn[t], vn[t])
         for b in seqs:
             states[b].append(bits(kn[t, b]), bits(vn[t, b]))
         if w.schedule == "fixed":
             full_now = [O.fixed_stride_is_full(t, w.stride)] * w.batch
             if full_now[0]:
+                st.append(kn[t], vn[t])
                 st.refresh(qs[t])
+            elif fused:
+                st.append_partial(qs[t], kn[t], vn[t])
             else:
+                st.append(kn[t], vn[t])
                 st.partial(qs[t])
         else:
             full_now = [False] * w.batch
@@ -351,15 +409,23 @@ def run_trajectory(mods, w, layer, seqs=None, check_every=1):
                 st.check_trigger(qs[t], w.threshold)
                 flags = st.flag.cpu().numpy()
                 st.not_flag.copy_(1 - st.flag)
-                st.refresh(qs[t], active=st.flag)
-                st.partial(qs[t], active=st.not_flag)
+                if fused:      # appends for every sequence, attends for those that keep the partial cache
+                    st.append_partial(qs[t], kn[t], vn[t], active=st.not_flag)
+                    st.refresh(qs[t], active=st.flag)
+                else:
+                    st.append(kn[t], vn[t])
+                    st.refresh(qs[t], active=st.flag)
+                    st.partial(qs[t], active=st.not_flag)
                 full_now = [bool(f) for f in flags]
                 for b in seqs:
                     want, cos = O.should_refresh(O.bf16_bits_to_f64(bits(qs[t, b])), states[b].q_last_full, w.threshold)
                     if abs(cos - w.threshold) >= 1e-4:
                         assert flags[b] == want, (t, b, cos)
                     full_now[b] = bool(flags[b])
+            elif fused:
+                st.append_partial(qs[t], kn[t], vn[t])
             else:
+                st.append(kn[t], vn[t])
                 st.partial(qs[t])
         for b in seqs:
             if full_now[b]:
@@ -400,10 +466,11 @@ def follow_gpu_selection(st, state, b, o_score, w):
             assert np.array_equal(gpu_small[g, :take], small[g])
 
 
-def test_config1_every_step_every_head(mods):
+@pytest.mark.parametrize("fused", [False, True])
+def test_config1_every_step_every_head(mods, fused):
     rkv, runner, synth = mods
     w = synth.config1()
-    n_full = run_trajectory(mods, w, 0)
+    n_full = run_trajectory(mods, w, 0, fused=fused)
     assert n_full[0] == 4      # full steps at t = 4, 8, 12, 16
 
 
@@ -433,11 +500,12 @@ def test_config2_shape_one_layer_full_size(mods):
     assert n_full[0] == 1
 
 
-def test_config3_shape_dynamic_flags(mods):
+@pytest.mark.parametrize("fused", [False, True])
+def test_config3_shape_dynamic_flags(mods, fused):
     """Qwen2-7B shape (G=7), batch 4, dynamic refresh; reduced context for the per-step oracle, full K ratio."""
     rkv, runner, synth = mods
     w = synth.scaled(synth.config3(n_layers=1, ctx=8192), steps=40)
-    n_full = run_trajectory(mods, w, 0)
+    n_full = run_trajectory(mods, w, 0, fused=fused)
     # fast-drifting sequences refresh more often than slow ones
     assert n_full[0] >= n_full[3]
     assert n_full[0] >= 1
