@@ -1,12 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the RefreshKV decode-attention hot path.
 
-One "step" is one decode token through the attention work of ALL layers of the workload
-(default: Llama-3.1-8B attention shape, 32 layers, batch 1, L=32768, K=2048, fixed stride 10):
-per layer  (every 10th token) rkv_append + rkv_full_step + rkv_gather_small, else rkv_append_small_step.
-Each token's launches are replayed from a CUDA graph (one graph per kind of token).
+One "step" is one decode token through the attention work of ALL layers of the workload.  Default
+workload: Llama-3.1-8B attention shape, 32 layers, batch 1, L=32768, K=2048, fixed stride 10:
+per layer  rkv_append_small_step  on nine tokens out of ten, and on the tenth
+rkv_append + rkv_full_step + rkv_gather_small.  Dynamic workloads (cfg3) run, every QC-th token,
+rkv_should_refresh and then both branches under the per-sequence masks it wrote.  Each token's launches
+are replayed from a CUDA graph (one graph per kind of token).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2|cfg3|cfg4|cfg1]
 
 Prints ONE JSON line.  `value` is the amortised decode-attention time per token in microseconds
 (all layers), inputs resident in HBM; `e2e` is the same with each token's q/k/v rows coming from
@@ -27,9 +29,8 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-METRIC = "decode attention us/token (all layers, stride-10 refresh; full step and small step also reported)"
+METRIC = "decode attention us/token (all layers, refresh schedule of the workload; full step and small step also reported)"
 UNIT = "us/token"
-STRIDE = 10
 
 
 def parse_args():
@@ -38,12 +39,29 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--layers", type=int, default=32)
-    ap.add_argument("--ctx", type=int, default=32768)
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (0: its own)")
+    ap.add_argument("--ctx", type=int, default=0, help="override the context length of cfg2 / cfg3 (0: its own)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--small-min-chunk", type=int, default=0, help="override rkv_small_step chunking (0: library default)")
     ap.add_argument("--no-dependent-launch", action="store_true", help="plain stream order between kernels")
+    ap.add_argument("--no-small-cluster", action="store_true", help="merge partial-step splits through the workspace")
     return ap.parse_args()
+
+
+def make_workload(args):
+    from paper_2411_05787_b200 import synth
+    if args.workload == "cfg1":
+        w = synth.config1()
+    elif args.workload == "cfg2":
+        w = synth.config2(ctx=args.ctx or 32768)
+    elif args.workload == "cfg3":
+        w = synth.config3(ctx=args.ctx or 65536)
+    else:
+        w = synth.config4(n_layers=8)      # 8 of the 32 layers (23 GB of caches) unless --layers says otherwise
+    if args.layers:
+        w = synth.scaled(w, n_layers=args.layers)
+    return w
 
 
 def load_peaks():
@@ -102,37 +120,35 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------- reference arm
-def oracle_period_sample(w, layer_cache_bits, qs_bits, kn_bits, vn_bits):
-    """One stride period of ONE layer on the CPU oracle: 1 full step (+ rebuild) and stride-1 partial steps.
-
-    Returns seconds taken.  Inputs are the same bf16 bytes the GPU path consumes.
-    """
+def oracle_period_sample(w, layer_cache_bits, qs_bits, kn_bits, vn_bits, stride):
+    """One stride period of ONE layer and ONE sequence on the CPU oracle: 1 full step (+ rebuild) and
+    stride-1 partial steps.  Returns seconds taken.  Inputs are the same kind of bf16 bytes the GPU path consumes."""
     from oracle import rkv_oracle as O
     kf, vf = layer_cache_bits
     st = O.SequenceState(kf, vf, w.lens[0], w.k_small[0])
     t0 = time.perf_counter()
     st.full(qs_bits[0])
-    for t in range(1, STRIDE):
+    for t in range(1, stride):
         st.append(kn_bits[t], vn_bits[t])
         st.small(qs_bits[t])
     return time.perf_counter() - t0
 
 
-def cpu_inputs(w):
-    """Host copies (uint16 bf16 bits) of one layer of the workload for the oracle."""
-    import numpy as np
+def cpu_inputs(w, stride):
+    """Host copies (uint16 bf16 bits) of sequence 0 of one layer of the workload for the oracle."""
     import torch
     from paper_2411_05787_b200 import synth
-    cache = synth.fill_layer(w, 0, torch.device("cpu"), extra_cap=STRIDE + 1)
-    qs = synth.query_trajectory(synth.scaled(w, steps=STRIDE), 0)
-    synth.plant_heavy(w, cache, 0, qs[0])
-    kn, vn = synth.new_token_kv(synth.scaled(w, steps=STRIDE), 0)
+    w1 = synth.scaled(w, lens=[w.lens[0]], k_small=[w.k_small[0]], rho=[w.rho[0]] if w.rho else [], steps=stride)
+    cache = synth.fill_layer(w1, 0, torch.device("cpu"), extra_cap=stride + 1)
+    qs = synth.query_trajectory(w1, 0)
+    synth.plant_heavy(w1, cache, 0, qs[0])
+    kn, vn = synth.new_token_kv(w1, 0)
     cap = int(cache.cap[0])
     kf = synth.to_bits(cache.k).reshape(w.n_kv_heads, cap, 128)
     vf = synth.to_bits(cache.v).reshape(w.n_kv_heads, cap, 128)
-    qb = [synth.to_bits(qs[t, 0]) for t in range(STRIDE)]
-    knb = [synth.to_bits(kn[t, 0]) for t in range(STRIDE)]
-    vnb = [synth.to_bits(vn[t, 0]) for t in range(STRIDE)]
+    qb = [synth.to_bits(qs[t, 0]) for t in range(stride)]
+    knb = [synth.to_bits(kn[t, 0]) for t in range(stride)]
+    vnb = [synth.to_bits(vn[t, 0]) for t in range(stride)]
     return (kf, vf), qb, knb, vnb
 
 
@@ -144,39 +160,51 @@ def cpu_threads() -> int:
         return os.cpu_count() or 1
 
 
+def cpu_baseline(w, n_samples, warm):
+    """The oracle, as it stands, on the host cores: microseconds per token for all layers and sequences,
+    from samples of one stride period of one layer of sequence 0, scaled by the positions the other
+    sequences and layers hold."""
+    stride = w.stride
+    caches, qb, knb, vnb = cpu_inputs(w, stride)
+    for _ in range(warm):
+        oracle_period_sample(w, (caches[0].copy(), caches[1].copy()), qb, knb, vnb, stride)
+    t = [oracle_period_sample(w, (caches[0].copy(), caches[1].copy()), qb, knb, vnb, stride) for _ in range(n_samples)]
+    seq_scale = sum(w.lens) / float(w.lens[0])
+    per_token_us = statistics.mean(t) * w.n_layers * seq_scale / stride * 1e6
+    sample = (f"{n_samples} samples of one stride period (1 full step + rebuild + {stride - 1} partial steps) of sequence 0 "
+              f"in 1 of {w.n_layers} layers, scaled x{w.n_layers} layers x{seq_scale:.2f} (positions of all sequences) "
+              f"/ {stride} tokens")
+    return per_token_us, sample
+
+
 def run_reference(args):
-    """The oracle, as it stands, on the host cores: each step = one stride period of one layer, scaled to
-    all layers and divided by the stride to give microseconds per token."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    from paper_2411_05787_b200 import synth
-    w = synth.config2(n_layers=args.layers, ctx=args.ctx)
-    caches, qb, knb, vnb = cpu_inputs(w)
+    w = make_workload(args)
     steps = max(1, min(args.steps, 40))          # bounded: a period costs about a second of CPU time
     warm = max(1, min(args.warmup, 2))
-    for _ in range(warm):
-        oracle_period_sample(w, (caches[0].copy(), caches[1].copy()), qb, knb, vnb)
-    t = [oracle_period_sample(w, (caches[0].copy(), caches[1].copy()), qb, knb, vnb) for _ in range(steps)]
-    per_token_us = statistics.mean(t) * w.n_layers / STRIDE * 1e6
-    cores = cpu_threads()
-    sample = (f"{steps} samples of one stride period (1 full step + rebuild + {STRIDE - 1} partial steps) of 1 of "
-              f"{w.n_layers} layers, scaled x{w.n_layers} layers / {STRIDE} tokens")
+    per_token_us, sample = cpu_baseline(w, steps, warm)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": per_token_us, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warm, "ms_per_step": per_token_us / 1000.0, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w, args),
-        "cpu_baseline": {"value": per_token_us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": workload_config(w),
+        "cpu_baseline": {"value": per_token_us, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": per_token_us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def workload_config(w, args):
+def workload_config(w):
+    full_gb = sum(w.lens) * w.n_kv_heads * 512.0 * w.n_layers / 1e9
+    small_gb = sum(w.k_small) * w.n_kv_heads * 512.0 * w.n_layers / 1e9
     return {"workload": w.name, "layers": w.n_layers, "batch": w.batch, "q_heads": w.n_q_heads,
-            "kv_heads": w.n_kv_heads, "head_dim": 128, "context": w.lens[0], "k_small": w.k_small[0],
-            "stride": STRIDE, "schedule": "fixed", "l2_hygiene": "inputs larger than L2: every token walks all "
-            "layers' distinct caches (full 4.3 GB, small 0.27 GB)", "launch": "one CUDA graph replay per token"}
+            "kv_heads": w.n_kv_heads, "head_dim": 128, "context": max(w.lens), "context_min": min(w.lens),
+            "k_small": max(w.k_small), "stride": w.stride, "schedule": w.schedule,
+            "threshold": w.threshold if w.schedule == "dynamic" else None,
+            "l2_hygiene": f"inputs larger than L2: every token walks all layers' distinct caches "
+                          f"(full {full_gb:.1f} GB, small {small_gb:.2f} GB)",
+            "launch": "one CUDA graph replay per token"}
 
 
 # ----------------------------------------------------------------------------------------------- our arm
@@ -199,63 +227,84 @@ def run_ours(args):
     from paper_2411_05787_b200 import rkv, runner, synth
 
     dev = torch.device("cuda", torch.cuda.current_device())
-    n_tokens = args.steps + args.warmup
-    w = synth.config2(n_layers=args.layers, ctx=args.ctx)
-    # capacity for: warm-up + timed tokens of the main loop, the e2e loop, the always-full loop, profiling
-    total_tokens = 2 * n_tokens + 2 * 30 + 2 * STRIDE + 8
+    w = make_workload(args)
+    S, B, Hq, Hkv, NL = w.stride, w.batch, w.n_q_heads, w.n_kv_heads, w.n_layers
+    dynamic = w.schedule == "dynamic"
+    n_prof = 2 * S
+    # tokens decoded over all phases: main loop, e2e loop, always-full loop, small-only loop, profiling
+    total_tokens = 2 * (args.steps + args.warmup) + 10 + 23 + 2 * S + n_prof + 8
     wl = synth.scaled(w, steps=total_tokens)
-    L, K, Hq, Hkv = w.lens[0], w.k_small[0], w.n_q_heads, w.n_kv_heads
-    max_len = L + total_tokens + 1
-    ctx = rkv.Context(1, Hq, Hkv, max_len, K + STRIDE + 2)
+    k_max = max(w.k_small)
+    full_hint = max(w.lens) + total_tokens + 1
+    # a sequence that never refreshes keeps growing its small cache (dynamic schedule); fixed: at most S - 1 rows
+    small_extra = (total_tokens + 2) if dynamic else (S + 2)
+    small_hint = k_max + small_extra
+    ctx = rkv.Context(B, Hq, Hkv, full_hint, small_hint)
     if args.small_min_chunk:
         ctx.set_option(rkv.OPT_SMALL_MIN_CHUNK, args.small_min_chunk)
     if args.no_dependent_launch:
         ctx.set_option(rkv.OPT_DEPENDENT_LAUNCH, 0)
+    if args.no_small_cluster:
+        ctx.set_option(rkv.OPT_SMALL_CLUSTER, 0)
 
-    layers = []
-    q0 = synth.query_trajectory(synth.scaled(w, steps=1), 0).to(dev)
-    for l in range(w.n_layers):
-        cache = synth.fill_layer(wl, l, dev)
-        synth.plant_heavy(w, cache, l, q0[0])
-        layers.append(runner.LayerState(ctx, cache, [K], STRIDE + 2, Hq, Hkv))
-
-    # per-token inputs for all layers: [q | k_new | v_new] rows, one contiguous block per token
+    # per-token inputs: one contiguous block per token = all layers' q, then all k_new, then all v_new, so that
+    # one copy stages a token and the calls get contiguous views.  Queries follow the workload's AR(1) process
+    # per layer and sequence (the dynamic trigger depends on it).
+    n_in = min(total_tokens + 1, 320)             # distinct tokens kept; the loop cycles through them
+    win = synth.scaled(w, steps=n_in - 1)
+    nq, nk = NL * B * Hq * 128, NL * B * Hkv * 128
     row = (Hq + 2 * Hkv) * 128
-    n_in = 64                                     # distinct input blocks, cycled
-    g = torch.Generator(device="cpu"); g.manual_seed(1234)
-    inputs_host = torch.randn((n_in, w.n_layers, row), generator=g, dtype=torch.float32).to(torch.bfloat16).pin_memory()
+    inputs_host = torch.empty((n_in, nq + 2 * nk), dtype=torch.bfloat16).pin_memory()
+    for l in range(NL):
+        qs = synth.query_trajectory(win, l)                       # [n_in, B, Hq, 128]
+        kn, vn = synth.new_token_kv(win, l)                       # [n_in, B, Hkv, 128]
+        inputs_host[:, :nq].view(n_in, NL, B * Hq * 128)[:, l] = qs.reshape(n_in, -1)
+        inputs_host[:, nq: nq + nk].view(n_in, NL, B * Hkv * 128)[:, l] = kn.reshape(n_in, -1)
+        inputs_host[:, nq + nk:].view(n_in, NL, B * Hkv * 128)[:, l] = vn.reshape(n_in, -1)
     inputs_dev = inputs_host.to(dev)
-    stage = torch.zeros((w.n_layers, row), dtype=torch.bfloat16, device=dev)
-    outs = torch.zeros((w.n_layers, Hq * 128), dtype=torch.bfloat16, device=dev)
-    outs_host = torch.zeros((w.n_layers, Hq * 128), dtype=torch.bfloat16).pin_memory()
-    views = []
-    for l in range(w.n_layers):
-        q = stage[l, : Hq * 128].view(1, Hq, 128)
-        kn = stage[l, Hq * 128: (Hq + Hkv) * 128].view(1, Hkv, 128)
-        vn = stage[l, (Hq + Hkv) * 128:].view(1, Hkv, 128)
-        layers[l].out = outs[l].view(1, Hq, 128)
-        views.append((q, kn, vn))
+    stage = torch.zeros((nq + 2 * nk,), dtype=torch.bfloat16, device=dev)
+    q_stage = stage[:nq].view(NL, B, Hq, 128)
+    k_stage = stage[nq: nq + nk].view(NL, B, Hkv, 128)
+    v_stage = stage[nq + nk:].view(NL, B, Hkv, 128)
+    outs = torch.zeros((NL, B, Hq * 128), dtype=torch.bfloat16, device=dev)
+    outs_host = torch.zeros((NL, B, Hq * 128), dtype=torch.bfloat16).pin_memory()
+    flag_total = torch.zeros((NL, B), dtype=torch.int32, device=dev)
 
-    def token(full: bool):
+    stage.copy_(inputs_dev[0])
+    layers = []
+    for l in range(NL):
+        cache = synth.fill_layer(wl, l, dev)
+        synth.plant_heavy(w, cache, l, q_stage[l])
+        st = runner.LayerState(ctx, cache, list(w.k_small), small_extra, Hq, Hkv)
+        st.out = outs[l].view(B, Hq, 128)
+        layers.append(st)
+
+    def token(kind: str):
         for l, st in enumerate(layers):
-            q, kn, vn = views[l]
-            if full:
+            q, kn, vn = q_stage[l], k_stage[l], v_stage[l]
+            if kind == "full":
                 st.append(kn, vn)
-                st.refresh(q, max_len_hint=max_len)
-            else:      # append + partial step in one call (one launch)
-                st.append_partial(q, kn, vn, max_len_hint=K + STRIDE + 1)
+                st.refresh(q, max_len_hint=full_hint)
+            elif kind == "small":      # append + partial step in one call (one launch)
+                st.append_partial(q, kn, vn, max_len_hint=small_hint)
+            else:                      # check: the trigger decides per sequence; both branches run under its masks
+                st.check_trigger(q, w.threshold)
+                st.append_partial(q, kn, vn, active=st.not_flag, max_len_hint=small_hint)
+                st.refresh(q, active=st.flag, max_len_hint=full_hint)
+                flag_total[l].add_(st.flag)
 
     # initial small caches + eager warm-up of every kernel (also creates the tensor maps)
-    stage.copy_(inputs_dev[0])
-    for st, (q, _, _) in zip(layers, views):
-        st.refresh(q, max_len_hint=max_len)
-    token(False); token(True)
+    for l, st in enumerate(layers):
+        st.refresh(q_stage[l], max_len_hint=full_hint)
+    kinds = ["small", "full"] + (["check"] if dynamic else [])
+    for kind in kinds:
+        token(kind)
     torch.cuda.synchronize()
 
     # capture one graph per kind of token
     side = torch.cuda.Stream()
     graphs, launches_per = {}, {}
-    for kind in (False, True):
+    for kind in kinds:
         gr = torch.cuda.CUDAGraph()
         before = ctx.launch_count
         with torch.cuda.stream(side):
@@ -267,19 +316,28 @@ def run_ours(args):
 
     tok_counter = [1]
 
+    def kind_of(t, always_full, force_small):
+        if force_small:
+            return "small"
+        if always_full:
+            return "full"
+        if t % S != 0:
+            return "small"
+        return "check" if dynamic else "full"
+
     def run_tokens(n, e2e=False, always_full=False, force_small=False):
-        """Enqueue n decode tokens; returns (#full tokens, #small tokens)."""
-        nf = ns = 0
+        """Enqueue n decode tokens; returns the count of each kind."""
+        cnt = {k: 0 for k in kinds}
         for _ in range(n):
             t = tok_counter[0]; tok_counter[0] += 1
             src = inputs_host if e2e else inputs_dev
             stage.copy_(src[t % n_in], non_blocking=True)
-            full = (always_full or (t % STRIDE == 0)) and not force_small
-            graphs[full].replay()
+            kind = kind_of(t, always_full, force_small)
+            graphs[kind].replay()
             if e2e:
                 outs_host.copy_(outs, non_blocking=True)
-            nf += int(full); ns += int(not full)
-        return nf, ns
+            cnt[kind] += 1
+        return cnt
 
     def timed(n, **kw):
         if world > 1:
@@ -287,7 +345,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        nf, ns = run_tokens(n, **kw)
+        cnt = run_tokens(n, **kw)
         e1.record()
         torch.cuda.synchronize()
         if world > 1:
@@ -297,41 +355,45 @@ def run_ours(args):
             tt = torch.tensor([ms], device=dev)
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             ms = float(tt.item())
-        return ms, nf, ns
+        return ms, cnt
 
     # ---- main measurement: inputs resident in HBM.  The token counter runs on through all phases, so a
-    # refresh comes at least every STRIDE tokens and the small caches never outgrow their capacity.
+    # refresh (or a check) comes every S tokens and the small caches never outgrow their capacity.
     run_tokens(args.warmup)
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else 0)
     if rank == 0:
         sampler.start()
-    ms, nf, ns = timed(args.steps)
+    torch.cuda.synchronize()
+    flag_total.zero_()
+    ms, cnt = timed(args.steps)
     clocks = sampler.stop() if rank == 0 else {}
     us_per_token = ms * 1000.0 / (args.steps * world)
-    launches = nf * launches_per[True] + ns * launches_per[False]
+    launches = sum(cnt[k] * launches_per[k] for k in kinds)
+    refreshed = int(flag_total.sum().item()) if dynamic else cnt["full"] * NL * B
+    checks = cnt.get("check", 0)
 
     # ---- end to end: inputs from pinned host memory, outputs back to the host, every token
     run_tokens(min(args.warmup, 10), e2e=True)
-    ms_e2e, _, _ = timed(args.steps, e2e=True)
+    ms_e2e, _ = timed(args.steps, e2e=True)
     e2e_us = ms_e2e * 1000.0 / (args.steps * world)
 
-    # ---- always-full attention (the vanilla comparator) on the same caches
+    # ---- always-full attention (the vanilla comparator) on the same caches, then partial steps only
     run_tokens(3, always_full=True)
-    ms_full, nff, _ = timed(20, always_full=True)
+    ms_full, _ = timed(20, always_full=True)
     full_token_us = ms_full * 1000.0 / (20 * world)
-    ms_small, _, nss = timed(STRIDE - 1, force_small=True)   # right after a full token: K .. K+8 rows
+    ms_small, _ = timed(S - 1, force_small=True)   # right after a full token: K .. K+S-2 rows
     run_tokens(1, always_full=True)
-    # ---- per-kernel device time: every launch bracketed by CUDA events on its stream (same schedule, two
-    # periods).  A spin kernel first keeps the GPU busy while the host enqueues, so that the launches sit
-    # back to back in the queue and an event pair measures the kernel, not the host's launch latency.
+    # ---- per-kernel device time: every launch bracketed by CUDA events on its stream (fixed-stride schedule,
+    # two periods, every sequence active).  A spin kernel first keeps the GPU busy while the host enqueues, so
+    # that the launches sit back to back in the queue and an event pair measures the kernel, not the host.
     torch.cuda.synchronize()
     ctx.set_profiling(True)
     ctx.get_profile()
     torch.cuda._sleep(int(8e7))
-    for _ in range(2 * STRIDE):
+    for i in range(n_prof):
         t = tok_counter[0]; tok_counter[0] += 1
         stage.copy_(inputs_dev[t % n_in])
-        token(t % STRIDE == 0)
+        token("full" if i % S == 0 else "small")
     torch.cuda.synchronize()
     prof = ctx.get_profile()
     ctx.set_profiling(False)
@@ -343,57 +405,56 @@ def run_ours(args):
         return
 
     peak, peak_src = load_peaks()
-    len_avg = L + total_tokens / 2.0
-    kv_bytes_full = len_avg * Hkv * 512.0                       # K+V bytes one full-step launch must read
-    kv_bytes_small = (K + STRIDE / 2.0) * Hkv * 512.0
+    pos_full = sum(w.lens) + B * (total_tokens / 2.0)           # positions one full-step launch streams (all sequences)
+    pos_small = sum(w.k_small) + B * (S / 2.0)
+    kv_bytes_full = pos_full * Hkv * 512.0                      # K+V bytes one full-step launch must read
+    kv_bytes_small = pos_small * Hkv * 512.0
     kern = {}
-    for name, (us, cnt) in prof.items():
-        if cnt:
-            kern[name] = {"launches": cnt, "avg_us": us / cnt}
+    for name, (us, c) in prof.items():
+        if c:
+            kern[name] = {"launches": c, "avg_us": us / c}
     attn_us = kern["attn_full"]["avg_us"]
     achieved = kv_bytes_full / (attn_us * 1e-6) / 1e9
     small_us = kern["attn_small"]["avg_us"]
     kern["attn_full"]["gbs"] = achieved
     kern["attn_small"]["gbs"] = kv_bytes_small / (small_us * 1e-6) / 1e9
-    kern["gather"]["gbs"] = 2 * K * Hkv * 512.0 / (kern["gather"]["avg_us"] * 1e-6) / 1e9
+    kern["gather"]["gbs"] = 2 * sum(w.k_small) * Hkv * 512.0 / (kern["gather"]["avg_us"] * 1e-6) / 1e9
     full_step_us = attn_us + kern["select"]["avg_us"]
 
     result = {
         "metric": METRIC, "value": us_per_token, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in / fp32 accumulate", "data": "synthetic",
-        "config": workload_config(w, args),
+        "config": workload_config(w),
         "clocks": clocks,
-        "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": w.n_layers * row * 2,
-                "d2h_bytes_per_step": w.n_layers * Hq * 128 * 2},
+        "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": NL * B * row * 2,
+                "d2h_bytes_per_step": NL * B * Hq * 128 * 2},
         "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "attn_kernel<logits> (full-cache attention + score logits)",
+        "roofline": {"bound": "hbm", "kernel": "attn_kernel<full> (full-cache attention + score logits)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": peak_src, "traffic": None,
                      "algorithmic_bytes_per_launch": kv_bytes_full},
         "detail": {
             "always_full_us_per_token": full_token_us,
             "refresh_speedup_vs_always_full": full_token_us / us_per_token,
-            "small_only_us_per_token": ms_small * 1000.0 / ((STRIDE - 1) * world),
+            "small_only_us_per_token": ms_small * 1000.0 / ((S - 1) * world),
+            "full_steps_in_timed_region": {"sequence_layer_refreshes": refreshed, "check_tokens": checks,
+                                           "of_possible": args.steps * NL * B},
             "per_layer_kernel_us": kern,
             "full_step_attn_plus_select_us": full_step_us,
             "full_step_frac_of_8TBs": kv_bytes_full / (full_step_us * 1e-6) / 8e12,
             "small_step_frac_of_8TBs": kv_bytes_small / (small_us * 1e-6) / 8e12,
             "attn_full_frac_of_8TBs": achieved / 8000.0,
+            "in_graph_us_per_layer": {"full_token": full_token_us / NL,
+                                      "small_token": ms_small * 1000.0 / ((S - 1) * world) / NL},
             "device_status": status,
-            "graph_launches": {"full_token": launches_per[True], "small_token": launches_per[False]},
+            "graph_launches": launches_per,
         },
     }
     if not args.no_cpu_baseline and world == 1:
-        caches, qb, knb, vnb = cpu_inputs(w)
-        oracle_period_sample(w, (caches[0].copy(), caches[1].copy()), qb, knb, vnb)
-        n_s = 8
-        t = [oracle_period_sample(w, (caches[0].copy(), caches[1].copy()), qb, knb, vnb) for _ in range(n_s)]
-        per_token_us = statistics.mean(t) * w.n_layers / STRIDE * 1e6
-        result["cpu_baseline"] = {
-            "value": per_token_us, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-            "sample": f"{n_s} samples of one stride period (1 full + {STRIDE - 1} partial steps) of 1 of "
-                      f"{w.n_layers} layers, scaled x{w.n_layers} / {STRIDE} tokens"}
+        per_token_us, sample = cpu_baseline(w, 8, 1)
+        result["cpu_baseline"] = {"value": per_token_us, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                  "sample": sample}
     print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()

@@ -177,10 +177,12 @@ rkv_status rkv_append_small_step(rkv_ctx* ctx, const void* q, const void* k_new,
  *   sim   = <qbar, qbar'> / (|qbar| |qbar'|)          (fp32)
  *   flag[b] = 0 (partial step) if sim > threshold, else 1 (full step);
  *   equality and NaN (a zero mean vector) give 1.
- *   q_now, q_last_full  bf16 [B][Hq][128];  flag int32 [B];  sim fp32 [B] or NULL
+ *   keep[b] = 1 - flag[b]: the mask of the sequences that stay on the partial cache, ready to be
+ *   passed as `active` to rkv_small_step / rkv_append_small_step while flag goes to rkv_full_step.
+ *   q_now, q_last_full  bf16 [B][Hq][128];  flag int32 [B];  keep int32 [B] or NULL;  sim fp32 [B] or NULL
  */
 rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_last_full,
-                              float threshold, int32_t* flag, float* sim, void* stream);
+                              float threshold, int32_t* flag, int32_t* keep, float* sim, void* stream);
 
 /*
  * Partial step without a context and without any allocation (the paper has no counterpart: this

@@ -392,12 +392,12 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const 
 }
 
 rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_last_full, float threshold,
-                              int32_t* flag, float* sim, void* stream) {
+                              int32_t* flag, int32_t* keep, float* sim, void* stream) {
   if (!ctx || !q_now || !q_last_full || !flag) return RKV_ERR_INVALID_ARG;
   cudaError_t e;
   {
     LaunchScope scope(ctx, static_cast<cudaStream_t>(stream), RKV_KERNEL_TRIGGER);
-    e = rkv::launch_trigger(q_now, q_last_full, threshold, flag, sim, ctx->cfg.n_seq, ctx->cfg.n_q_heads,
+    e = rkv::launch_trigger(q_now, q_last_full, threshold, flag, keep, sim, ctx->cfg.n_seq, ctx->cfg.n_q_heads,
                             static_cast<cudaStream_t>(stream));
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "trigger launch");

@@ -97,7 +97,7 @@ cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k
 cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, CacheDev small_cache,
                           bool has_full, bool has_small, int n_seq, int n_kv_heads, int32_t* status,
                           cudaStream_t st);
-cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag,
+cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, int32_t* keep,
                            float* sim, int n_seq, int n_q_heads, cudaStream_t st);
 // Launch with optional programmatic dependent launch (the kernel may start while its predecessor on
 // the stream drains; every kernel waits with pdl_wait() before touching global memory) and an

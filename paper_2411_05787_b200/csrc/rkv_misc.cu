@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(128) append_kernel(const uint4* __restrict__ k
 // one block of 128 threads per sequence: thread d owns channel d of the head-averaged queries
 __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __restrict__ q_now,
                                                       const __nv_bfloat16* __restrict__ q_last, float threshold,
-                                                      int32_t* flag, float* sim, int n_q_heads) {
+                                                      int32_t* flag, int32_t* keep, float* sim, int n_q_heads) {
   const int b = blockIdx.x, d = threadIdx.x;
   pdl_launch();
   pdl_wait();
@@ -130,7 +130,9 @@ __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __res
     const float n1 = (red[1][0] + red[1][1]) + (red[1][2] + red[1][3]);
     const float n2 = (red[2][0] + red[2][1]) + (red[2][2] + red[2][3]);
     const float cs = dt / (sqrtf(n1) * sqrtf(n2));  // 0/0 -> NaN -> not "higher" -> refresh
-    flag[b] = (cs > threshold) ? 0 : 1;
+    const int refresh = (cs > threshold) ? 0 : 1;
+    flag[b] = refresh;
+    if (keep != nullptr) keep[b] = 1 - refresh;
     if (sim != nullptr) sim[b] = cs;
   }
 }
@@ -156,10 +158,10 @@ cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, C
                    n_kv_heads, status);
 }
 
-cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, float* sim,
-                           int n_seq, int n_q_heads, cudaStream_t st) {
+cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, int32_t* keep,
+                           float* sim, int n_seq, int n_q_heads, cudaStream_t st) {
   return launch_ex(trigger_kernel, dim3(n_seq), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(q_now),
-                   static_cast<const __nv_bfloat16*>(q_last), threshold, flag, sim, n_q_heads);
+                   static_cast<const __nv_bfloat16*>(q_last), threshold, flag, keep, sim, n_q_heads);
 }
 
 }  // namespace rkv

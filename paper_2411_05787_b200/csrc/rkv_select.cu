@@ -232,18 +232,18 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   }
   __nv_bfloat16 qv = __float2bfloat16(0.f);
   if (p.q_last_full != nullptr && sgrp == 0 && o_on) qv = static_cast<const __nv_bfloat16*>(p.q)[hrow0 + o_flat];
-  float4 v[U][GP / 4];
-  auto load_round = [&](int i0) {
+  float4 v[U][GP / 4], vnext[U][GP / 4];     // the round being turned into keys, and the one in flight behind it
+  auto load_round = [&](float4 (&dst)[U][GP / 4], int i0) {
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int i = i0 + u * NT + tid;
       const bool on = i < per && lo + i < p.logit_stride;
 #pragma unroll
       for (int c = 0; c < GP / 4; ++c)
-        v[u][c] = on ? __ldcg(reinterpret_cast<const float4*>(lg + (int64_t)i * GP) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        dst[u][c] = on ? __ldcg(reinterpret_cast<const float4*>(lg + (int64_t)i * GP) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
-  load_round(0);
+  load_round(v, 0);
 
   if (act == 0) return;   // same decision in all CTAs of the cluster
   {
@@ -331,7 +331,8 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
     const float inv_g = 1.f / (float)G;
     bool bad = false;
     for (int i0 = 0; i0 < cnt_pad; i0 += U * NT) {
-      if (i0 > 0) load_round(i0);
+      const bool more = i0 + U * NT < cnt_pad;
+      if (more) load_round(vnext, i0 + U * NT);   // overlaps the arithmetic below
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int i = i0 + u * NT + tid;
@@ -365,6 +366,12 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
           if (!all_selected) atomicAdd(&sh->hist[0][bin >> 1], 1u << ((bin & 1u) << 4));
         }
         keys[i] = key;
+      }
+      if (more) {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+          for (int c = 0; c < GP / 4; ++c) v[u][c] = vnext[u][c];
       }
     }
     if (bad) sh->bad = 1u;

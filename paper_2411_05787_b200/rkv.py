@@ -55,7 +55,7 @@ def _load() -> ctypes.CDLL:
     lib.rkv_append.argtypes = [vp, vp, vp, cachep, cachep, vp]
     lib.rkv_append_small_step.argtypes = [vp, vp, vp, vp, cachep, cachep, vp, vp, i32, vp]
     lib.rkv_append_small_step.restype = i32
-    lib.rkv_should_refresh.argtypes = [vp, vp, vp, f32, vp, vp, vp]
+    lib.rkv_should_refresh.argtypes = [vp, vp, vp, f32, vp, vp, vp, vp]
     lib.rkv_get_device_status.argtypes = [vp, ctypes.POINTER(i32), vp]
     lib.rkv_status_string.argtypes = [i32]
     lib.rkv_status_string.restype = ctypes.c_char_p
@@ -184,9 +184,9 @@ class Context:
                                               ctypes.byref(full) if full is not None else None, ctypes.byref(small),
                                               _ptr(active), _ptr(out), max_len_hint, _stream(stream)))
 
-    def should_refresh(self, q_now, q_last_full, threshold, flag, sim=None, stream=None):
+    def should_refresh(self, q_now, q_last_full, threshold, flag, sim=None, keep=None, stream=None):
         self._check(lib.rkv_should_refresh(self._h, _ptr(q_now), _ptr(q_last_full), float(threshold), _ptr(flag),
-                                           _ptr(sim), _stream(stream)))
+                                           _ptr(keep), _ptr(sim), _stream(stream)))
 
     def set_option(self, option: int, value: int):
         self._check(lib.rkv_set_option(self._h, option, value))

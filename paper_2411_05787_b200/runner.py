@@ -58,5 +58,5 @@ class LayerState:
         self.ctx.append(k_new, v_new, self.full_c, self.small_c)
 
     def check_trigger(self, q, threshold):
-        self.ctx.should_refresh(q, self.q_last_full, threshold, self.flag, self.sim)
+        self.ctx.should_refresh(q, self.q_last_full, threshold, self.flag, self.sim, keep=self.not_flag)
         return self.flag

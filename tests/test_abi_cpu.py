@@ -53,4 +53,4 @@ def test_null_arguments_are_rejected_before_any_launch(lib):
     assert lib.lib.rkv_launch_count(None) == 0
     assert lib.lib.rkv_small_step(None, None, None, None, None, 0, None) == 1
     assert lib.lib.rkv_append(None, None, None, None, None, None) == 1
-    assert lib.lib.rkv_should_refresh(None, None, None, 0.5, None, None, None) == 1
+    assert lib.lib.rkv_should_refresh(None, None, None, 0.5, None, None, None, None) == 1

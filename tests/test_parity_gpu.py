@@ -278,7 +278,9 @@ def test_trigger_flags_and_similarity(mods):
     flag = torch.full((n_seq,), -7, dtype=torch.int32, device="cuda")
     sim = torch.zeros((n_seq,), dtype=torch.float32, device="cuda")
     thr = 0.9
-    ctx.should_refresh(now, last, thr, flag, sim)
+    keep = torch.full((n_seq,), -7, dtype=torch.int32, device="cuda")
+    ctx.should_refresh(now, last, thr, flag, sim, keep=keep)
+    assert torch.equal(keep, 1 - flag)
     flag_h, sim_h = flag.cpu().numpy(), sim.cpu().numpy()
     near = 0
     for b in range(n_seq):
@@ -408,7 +410,7 @@ def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False):
             if t % w.stride == 0:
                 st.check_trigger(qs[t], w.threshold)
                 flags = st.flag.cpu().numpy()
-                st.not_flag.copy_(1 - st.flag)
+                assert torch.equal(st.not_flag, 1 - st.flag)      # the trigger wrote both masks
                 if fused:      # appends for every sequence, attends for those that keep the partial cache
                     st.append_partial(qs[t], kn[t], vn[t], active=st.not_flag)
                     st.refresh(qs[t], active=st.flag)
