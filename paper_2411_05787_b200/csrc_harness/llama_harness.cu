@@ -1,0 +1,245 @@
+// Batch-1 decoder kernels around the attention calls (see include/rkv_harness.h).
+// All of them are bound by streaming bf16 weights once per token; the matrix-vector kernels keep
+// 64 bytes per lane in flight and reduce inside a warp.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rkv_harness.h"
+
+namespace {
+
+constexpr int kGemvThreads = 256;
+constexpr int kMaxIn = 16384;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 t = __bfloat1622float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+// <row, x> for one weight row: lane l takes 16-byte chunks l, l+32, ...; x sits in shared memory as fp32
+__device__ __forceinline__ float row_dot(const uint4* __restrict__ row, const float* xs, int n_chunks, int lane) {
+  float acc = 0.f;
+  for (int c0 = lane; c0 < n_chunks; c0 += 128) {   // four chunks (64 bytes) per lane in flight
+    uint4 u[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int c = c0 + 32 * k;
+      u[k] = (c < n_chunks) ? __ldcs(row + c) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int c = c0 + 32 * k;
+      if (c < n_chunks) {
+        float f[8];
+        unpack8(u[k], f);
+        const float4 x0 = *reinterpret_cast<const float4*>(xs + 8 * c);
+        const float4 x1 = *reinterpret_cast<const float4*>(xs + 8 * c + 4);
+        acc = fmaf(f[0], x0.x, acc); acc = fmaf(f[1], x0.y, acc); acc = fmaf(f[2], x0.z, acc); acc = fmaf(f[3], x0.w, acc);
+        acc = fmaf(f[4], x1.x, acc); acc = fmaf(f[5], x1.y, acc); acc = fmaf(f[6], x1.z, acc); acc = fmaf(f[7], x1.w, acc);
+      }
+    }
+  }
+  return warp_sum(acc);
+}
+__device__ __forceinline__ void stage_x(const void* x, int x_is_bf16, float* xs, int n_in) {
+  if (x_is_bf16) {
+    const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+    for (int i = threadIdx.x; i < n_in; i += blockDim.x) xs[i] = __bfloat162float(xb[i]);
+  } else {
+    const float* xf = static_cast<const float*>(x);
+    for (int i = threadIdx.x; i < n_in; i += blockDim.x) xs[i] = xf[i];
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const uint4* __restrict__ w, const void* x, int x_is_bf16,
+                                                            const float* residual, float* y, int n_out, int n_in) {
+  extern __shared__ float xs[];
+  stage_x(x, x_is_bf16, xs, n_in);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = kGemvThreads / 32;
+  const int n_chunks = n_in / 8;
+  for (int o = blockIdx.x * wpb + warp; o < n_out; o += gridDim.x * wpb) {
+    const float d = row_dot(w + (int64_t)o * n_chunks, xs, n_chunks, lane);
+    if (lane == 0) y[o] = d + (residual != nullptr ? residual[o] : 0.f);
+  }
+}
+
+__global__ void __launch_bounds__(kGemvThreads) gemv_swiglu_kernel(const uint4* __restrict__ w, const float* x, float* y,
+                                                                   int n_ff, int n_in) {
+  extern __shared__ float xs[];
+  stage_x(x, 0, xs, n_in);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = kGemvThreads / 32;
+  const int n_chunks = n_in / 8;
+  for (int f = blockIdx.x * wpb + warp; f < n_ff; f += gridDim.x * wpb) {
+    const float g = row_dot(w + (int64_t)f * n_chunks, xs, n_chunks, lane);
+    const float u = row_dot(w + (int64_t)(f + n_ff) * n_chunks, xs, n_chunks, lane);
+    if (lane == 0) y[f] = g / (1.f + __expf(-g)) * u;
+  }
+}
+
+__global__ void __launch_bounds__(1024) rmsnorm_kernel(const float* x, const __nv_bfloat16* w, float eps, float* y, int n) {
+  __shared__ float red[32];
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) ss = fmaf(x[i], x[i], ss);
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int i = 0; i < (int)(blockDim.x >> 5); ++i) tot += red[i];
+  const float r = rsqrtf(tot / (float)n + eps);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) y[i] = x[i] * r * __bfloat162float(w[i]);
+}
+
+// one thread per (head, channel pair c, c + 64); v heads are copied
+__global__ void __launch_bounds__(256) rope_split_kernel(const float* qkv, const int32_t* pos, float theta, __nv_bfloat16* q,
+                                                         __nv_bfloat16* k, __nv_bfloat16* v, int n_q, int n_kv) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n_rot = (n_q + n_kv) * 64;
+  if (t < n_rot) {
+    const int head = t >> 6, c = t & 63;
+    // the angle reaches tens of thousands of radians: form it and its sine / cosine in double
+    const double ang = (double)pos[0] * pow((double)theta, -(double)c / 64.0);
+    double snd, csd;
+    sincos(ang, &snd, &csd);
+    const float sn = (float)snd, cs = (float)csd;
+    const float a = qkv[head * 128 + c], b = qkv[head * 128 + c + 64];
+    __nv_bfloat16* dst = head < n_q ? q + head * 128 : k + (head - n_q) * 128;
+    dst[c] = __float2bfloat16(a * cs - b * sn);
+    dst[c + 64] = __float2bfloat16(b * cs + a * sn);
+  } else if (t < n_rot + n_kv * 128) {
+    const int i = t - n_rot;
+    v[i] = __float2bfloat16(qkv[(n_q + n_kv) * 128 + i]);
+  }
+}
+
+__global__ void __launch_bounds__(256) embed_kernel(const __nv_bfloat16* table, const int32_t* token, float* x, int hidden,
+                                                    int vocab) {
+  int tok = token[0];
+  tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < hidden; i += gridDim.x * blockDim.x)
+    x[i] = __bfloat162float(table[(int64_t)tok * hidden + i]);
+}
+
+__global__ void __launch_bounds__(1024) argmax_kernel(const float* logits, int n, int32_t* token) {
+  __shared__ float bv[32];
+  __shared__ int bi[32];
+  float best = -INFINITY;
+  int idx = 0x7fffffff;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {   // indices ascend, so a strict compare keeps the lowest
+    const float vv = logits[i];
+    if (vv > best || idx == 0x7fffffff) {
+      best = vv;
+      idx = i;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+    if (ov > best || (ov == best && oi < idx)) {
+      best = ov;
+      idx = oi;
+    }
+  }
+  if ((threadIdx.x & 31) == 0) {
+    bv[threadIdx.x >> 5] = best;
+    bi[threadIdx.x >> 5] = idx;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w2 = 1; w2 < (int)(blockDim.x >> 5); ++w2)
+      if (bv[w2] > best || (bv[w2] == best && bi[w2] < idx)) {
+        best = bv[w2];
+        idx = bi[w2];
+      }
+    token[0] = idx == 0x7fffffff ? 0 : idx;
+  }
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+bool g_attr_set = false;
+int ensure_attrs() {
+  if (g_attr_set) return 0;
+  cudaError_t e = cudaFuncSetAttribute(gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_swiglu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
+  if (e != cudaSuccess) return (int)e;
+  g_attr_set = true;
+  return 0;
+}
+int gemv_grid(int n_rows) {
+  const int per_block = kGemvThreads / 32;
+  int blocks = (n_rows + per_block - 1) / per_block;
+  const int cap = sm_count() * 8;
+  return blocks < cap ? (blocks < 1 ? 1 : blocks) : cap;
+}
+
+}  // namespace
+
+extern "C" {
+
+int llh_rmsnorm(const float* x, const void* w, float eps, float* y, int32_t n, void* stream) {
+  if (!x || !w || !y || n < 4 || n > kMaxIn || n % 4) return -1;
+  rmsnorm_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(x, static_cast<const __nv_bfloat16*>(w), eps, y, n);
+  return (int)cudaGetLastError();
+}
+
+int llh_gemv(const void* w, const void* x, int32_t x_is_bf16, const float* residual, float* y, int32_t n_out,
+             int32_t n_in, void* stream) {
+  if (!w || !x || !y || n_out < 1 || n_in < 256 || n_in > kMaxIn || n_in % 256) return -1;
+  if (int e = ensure_attrs()) return e;
+  gemv_kernel<<<gemv_grid(n_out), kGemvThreads, (size_t)n_in * 4, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4*>(w), x, x_is_bf16, residual, y, n_out, n_in);
+  return (int)cudaGetLastError();
+}
+
+int llh_gemv_swiglu(const void* w_gate_up, const float* x, float* y, int32_t n_ff, int32_t n_in, void* stream) {
+  if (!w_gate_up || !x || !y || n_ff < 1 || n_in < 256 || n_in > kMaxIn || n_in % 256) return -1;
+  if (int e = ensure_attrs()) return e;
+  gemv_swiglu_kernel<<<gemv_grid(n_ff), kGemvThreads, (size_t)n_in * 4, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4*>(w_gate_up), x, y, n_ff, n_in);
+  return (int)cudaGetLastError();
+}
+
+int llh_rope_split(const float* qkv, const int32_t* pos, float theta, void* q, void* k, void* v, int32_t n_q,
+                   int32_t n_kv, void* stream) {
+  if (!qkv || !pos || !q || !k || !v || n_q < 1 || n_kv < 1 || !(theta > 1.f)) return -1;
+  const int n = (n_q + n_kv) * 64 + n_kv * 128;
+  rope_split_kernel<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      qkv, pos, theta, static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k), static_cast<__nv_bfloat16*>(v), n_q,
+      n_kv);
+  return (int)cudaGetLastError();
+}
+
+int llh_embed(const void* table, const int32_t* token, float* x, int32_t hidden, int32_t vocab, void* stream) {
+  if (!table || !token || !x || hidden < 1 || vocab < 1) return -1;
+  embed_kernel<<<(hidden + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(table), token, x, hidden, vocab);
+  return (int)cudaGetLastError();
+}
+
+int llh_argmax(const float* logits, int32_t n, int32_t* token, void* stream) {
+  if (!logits || !token || n < 1) return -1;
+  argmax_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(logits, n, token);
+  return (int)cudaGetLastError();
+}
+
+}  // extern "C"

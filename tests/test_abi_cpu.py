@@ -54,3 +54,18 @@ def test_null_arguments_are_rejected_before_any_launch(lib):
     assert lib.lib.rkv_small_step(None, None, None, None, None, 0, None) == 1
     assert lib.lib.rkv_append(None, None, None, None, None, None) == 1
     assert lib.lib.rkv_should_refresh(None, None, None, 0.5, None, None, None, None) == 1
+
+
+def test_harness_library_exports_every_declared_symbol():
+    """libllama_harness.so (decoder kernels of the end-to-end workload) against include/rkv_harness.h."""
+    from paper_2411_05787_b200 import build
+    build.build()
+    from paper_2411_05787_b200 import harness
+    with open(os.path.join(ROOT, "include", "rkv_harness.h")) as f:
+        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    names = sorted(set(re.findall(r"\b(llh_[a-z_]+)\s*\(", text)))
+    assert len(names) == 6 and sorted(harness.EXPORTS) == names
+    for n in names:
+        assert hasattr(harness.lib, n), n
+    assert harness.lib.llh_gemv(None, None, 0, None, None, 8, 256, None) == -1      # null pointers: rejected on the host
+    assert harness.lib.llh_rmsnorm(None, None, 1e-5, None, 4096, None) == -1
