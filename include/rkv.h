@@ -71,7 +71,8 @@ typedef struct {
   int32_t max_len;       /* largest full-cache length any call will see                */
   int32_t max_small;     /* largest small-cache length any call will see               */
   int32_t agg;           /* rkv_agg; RKV_AGG_MAX is the paper's rule                   */
-  int32_t pool_kernel;   /* 1 = no pooling; odd w > 1 = max-pool of width w (App. A.1) */
+  int32_t pool_kernel;   /* 1 = no pooling; odd w in 3..31 = the scores are max-pooled over w neighbouring
+                            positions before the top-K (App. A.1: 7); then max_len <= 163840          */
   float softmax_scale;   /* 0 -> 1/sqrt(head_dim)                                      */
 } rkv_config;
 
@@ -99,7 +100,9 @@ size_t rkv_workspace_bytes(const rkv_config* cfg /*host*/);
  *   s[h][j]   = scale * <q[b][h], K[b][h/G][j]>               j < n
  *   p[h][j]   = softmax_j(s[h][:])
  *   out[b][h] = sum_j p[h][j] V[b][h/G][j]                     (bf16)
- *   score[b][g][j] = agg_{h in group g} p[h][j]                (fp32, optional output)
+ *   score[b][g][j] = agg_{h in group g} p[h][j]                (fp32, optional output);
+ *       with cfg.pool_kernel = w > 1:  score[j] <- max over |i - j| <= (w-1)/2, 0 <= i < n  (Sec. 2.2
+ *       "Prefilling stage": max pooling over the scores of surrounding tokens)
  *   topk_idx[b][g][0..m) = the m = min(k_small[b], n) positions of largest
  *       score, ties to the lower position, listed in ASCENDING position
  *       order; entries m..k_max-1 are -1.

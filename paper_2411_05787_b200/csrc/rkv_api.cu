@@ -24,7 +24,9 @@ bool config_ok(const rkv_config* c, rkv_status* why) {
   if (c->n_seq < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_len < 1 || c->max_small < 1 ||
       c->n_q_heads % c->n_kv_heads != 0) { *why = RKV_ERR_INVALID_ARG; return false; }
   if (c->head_dim != rkv::kHeadDim || c->n_q_heads / c->n_kv_heads > rkv::kMaxGroup ||
-      c->agg < RKV_AGG_MAX || c->agg > RKV_AGG_FIRST || c->pool_kernel != 1 ||
+      c->agg < RKV_AGG_MAX || c->agg > RKV_AGG_FIRST || c->pool_kernel < 1 || c->pool_kernel > 31 ||
+      c->pool_kernel % 2 == 0 ||
+      (c->pool_kernel > 1 && (int64_t)c->max_len > (int64_t)rkv::kSelectCluster * rkv::kSelectMaxKeysPerCtaPooled) ||
       (int64_t)c->max_len > (int64_t)rkv::kSelectCluster * rkv::kSelectMaxKeysPerCta ||
       (int64_t)c->n_seq * c->n_kv_heads > 65535 * 8) { *why = RKV_ERR_UNSUPPORTED; return false; }
   if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) { *why = RKV_ERR_INVALID_ARG; return false; }
@@ -322,6 +324,8 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, con
   const int per = (n_max + rkv::kSelectCluster - 1) / rkv::kSelectCluster;
   sp.per_cta = (per + 3) & ~3;
   sp.grid_splits = gx;
+  sp.pool_half = (ctx->cfg.pool_kernel - 1) / 2;
+  sp.keys_cap = rkv::select_keys_cap(sp.per_cta);
   cudaError_t e;
   {
     LaunchScope scope(ctx, st, RKV_KERNEL_SELECT);

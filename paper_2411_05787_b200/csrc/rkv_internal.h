@@ -77,6 +77,8 @@ struct SelectParams {
   int32_t per_cta;            // positions per CTA of the cluster (from the host's length bound; multiple of 4)
   int32_t chunk, max_splits;  // split geometry of the attention launch that produced the partials
   int32_t grid_splits;        // CTAs per (sequence, KV head) that launch had
+  int32_t pool_half;          // (pool_kernel - 1) / 2
+  int32_t keys_cap;           // padded key capacity of a CTA (offset of the unpooled keys in shared memory)
 };
 
 struct CacheDev {
@@ -140,7 +142,9 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 cudaError_t prepare_attention();  // one-time function attributes (dynamic shared memory sizes)
 cudaError_t prepare_select();
 size_t attention_smem_bytes();
-size_t select_smem_bytes(int keys_per_cta);
+size_t select_smem_bytes(int keys_per_cta, int pool_half);
+int select_keys_cap(int keys_per_cta);
+constexpr int kSelectMaxKeysPerCtaPooled = 20480;   // with pooling a CTA keeps two key arrays
 
 }  // namespace rkv
 

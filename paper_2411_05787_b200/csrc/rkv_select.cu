@@ -16,7 +16,8 @@
 // position).  The kernel is a chain of latencies, so it is laid out to have few links:
 //   1  one round trip fetches the per-sequence sizes, the split weights, this CTA's
 //      slice of the partial outputs and its first logits, all at once;
-//   2  keys + a 2048-bin histogram (1/64 nat per bin) in shared memory;
+//   2  keys + a 2048-bin histogram (1/64 nat per bin) in shared memory (with neighbour max-pooling
+//      of the scores, App. A.1, the keys of a window are min-reduced first);
 //   3  cluster barrier; the eight histograms are merged through distributed shared
 //      memory and the bin T that holds the K-th key is located (while T holds more
 //      than 256 keys, a finer histogram over T's key range repeats this step);
@@ -200,7 +201,10 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   const int per = p.per_cta;                  // positions per CTA, fixed by the host from its length bound
   const int lo = rank * per;
   const float* pbase = p.partials + (int64_t)bg * p.max_splits * PartialLayout::kFloats;
-  const float* lg = p.logits + ((int64_t)bg * p.logit_stride + lo) * GP;
+  const int half = p.pool_half;               // neighbour max-pooling of the scores over 2*half+1 positions (0: none)
+  // keys are made for positions lo-half .. lo+per+half-1 (the pooling window reaches into the neighbours' slices)
+  const float* lg = p.logits + ((int64_t)bg * p.logit_stride + lo - half) * GP;
+  uint32_t* raw = half > 0 ? keys + p.keys_cap : keys;   // unpooled keys; the same array when there is no pooling
   constexpr int U = 32 / GP;                  // positions per thread per round: all their loads are in flight together
   const int gx = p.grid_splits;               // splits the attention launch had room for (>= the sequence's own count)
   // slice of out[] this CTA folds: 16*G consecutive (head, channel) pairs of the group
@@ -237,7 +241,8 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int i = i0 + u * NT + tid;
-      const bool on = i < per && lo + i < p.logit_stride;
+      const int pos = lo - half + i;
+      const bool on = i < per + 2 * half && pos >= 0 && pos < p.logit_stride;
 #pragma unroll
       for (int c = 0; c < GP / 4; ++c)
         dst[u][c] = on ? __ldcg(reinterpret_cast<const float4*>(lg + (int64_t)i * GP) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -330,13 +335,14 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
     const int agg = p.agg;
     const float inv_g = 1.f / (float)G;
     bool bad = false;
-    for (int i0 = 0; i0 < cnt_pad; i0 += U * NT) {
-      const bool more = i0 + U * NT < cnt_pad;
+    const int n_raw = half > 0 ? (cnt > 0 ? cnt + 2 * half : 0) : cnt_pad;   // without pooling the padding is written here too
+    for (int i0 = 0; i0 < n_raw; i0 += U * NT) {
+      const bool more = i0 + U * NT < n_raw;
       if (more) load_round(vnext, i0 + U * NT);   // overlaps the arithmetic below
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int i = i0 + u * NT + tid;
-        if (i >= cnt_pad) continue;
+        if (i >= n_raw) continue;
         const float* x = reinterpret_cast<const float*>(&v[u][0]);
         float ell;
         if (agg == RKV_AGG_MAX) {   // heads >= G carry LSE = +inf and drop out of the max
@@ -352,7 +358,8 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
           ell = x[0] - lse_r[0];
         }
         uint32_t key = kPadKey;
-        if (i < cnt) {
+        const int pos = lo - half + i;
+        if (i < cnt + 2 * half && pos >= 0 && pos < n) {
           uint32_t bin;
           if (ell != ell) {
             bad = true;
@@ -363,9 +370,9 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
             key = __float_as_uint(nl) & 0x7fffffffu;
             bin = __float2uint_rz(fminf(nl * 64.f, (float)(kBins - 1)));
           }
-          if (!all_selected) atomicAdd(&sh->hist[0][bin >> 1], 1u << ((bin & 1u) << 4));
+          if (!all_selected && half == 0) atomicAdd(&sh->hist[0][bin >> 1], 1u << ((bin & 1u) << 4));
         }
-        keys[i] = key;
+        raw[i] = key;
       }
       if (more) {
 #pragma unroll
@@ -375,6 +382,19 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
       }
     }
     if (bad) sh->bad = 1u;
+    if (half > 0) {
+      // pooled score = max over the window = smallest key of the window (App. A.1: kernel size 7 in the paper)
+      __syncthreads();
+      for (int i = tid; i < cnt_pad; i += NT) {
+        uint32_t key = kPadKey;
+        if (i < cnt) {
+          for (int d = 0; d <= 2 * half; ++d) key = min(key, raw[i + d]);
+          const uint32_t bin = __float2uint_rz(fminf(__uint_as_float(key) * 64.f, (float)(kBins - 1)));
+          if (!all_selected) atomicAdd(&sh->hist[0][bin >> 1], 1u << ((bin & 1u) << 4));
+        }
+        keys[i] = key;
+      }
+    }
   }
 
   if (all_selected || kk == 0) {   // uniform over the cluster: nothing to choose
@@ -556,24 +576,29 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
 
 }  // namespace
 
-size_t select_smem_bytes(int keys_per_cta) {
-  const size_t padded = ((size_t)keys_per_cta + 4 * NT - 1) / (4 * NT) * (4 * NT);   // R * NT keys, R a multiple of 4
-  return ((sizeof(SelectShared) + 15) & ~size_t(15)) + padded * 4;
+int select_keys_cap(int keys_per_cta) {   // R * NT keys, R a multiple of 4
+  return (int)(((size_t)keys_per_cta + 4 * NT - 1) / (4 * NT) * (4 * NT));
+}
+
+size_t select_smem_bytes(int keys_per_cta, int pool_half) {
+  const size_t padded = (size_t)select_keys_cap(keys_per_cta);
+  const size_t raw = pool_half > 0 ? padded + 2 * (size_t)pool_half + 4 : 0;   // unpooled keys with their halo
+  return ((sizeof(SelectShared) + 15) & ~size_t(15)) + (padded + raw) * 4;
 }
 
 cudaError_t prepare_select() {
   cudaError_t e = cudaFuncSetAttribute(select_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)select_smem_bytes(kSelectMaxKeysPerCta));
+                                       (int)select_smem_bytes(kSelectMaxKeysPerCta, 0));
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)select_smem_bytes(kSelectMaxKeysPerCta));
+                              (int)select_smem_bytes(kSelectMaxKeysPerCta, 0));
 }
 
 cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st) {
   const dim3 grid(kSelectCluster, p.n_kv_heads, n_seq);
   if (p.group <= 4)
-    return launch_ex(select_kernel<4>, grid, dim3(NT), select_smem_bytes(p.per_cta), st, kSelectCluster, p);
-  return launch_ex(select_kernel<8>, grid, dim3(NT), select_smem_bytes(p.per_cta), st, kSelectCluster, p);
+    return launch_ex(select_kernel<4>, grid, dim3(NT), select_smem_bytes(p.per_cta, p.pool_half), st, kSelectCluster, p);
+  return launch_ex(select_kernel<8>, grid, dim3(NT), select_smem_bytes(p.per_cta, p.pool_half), st, kSelectCluster, p);
 }
 
 }  // namespace rkv

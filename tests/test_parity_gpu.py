@@ -46,7 +46,8 @@ def host_heads(cache, b, n_kv, which):
     return bits(t[off: off + n_kv * cap]).reshape(n_kv, cap, 128)
 
 
-def make_layer(mods, lens, k_small, n_q, n_kv, extra=8, seed=0, scale=1.0, agg=0, want_scores=True, poison=False):
+def make_layer(mods, lens, k_small, n_q, n_kv, extra=8, seed=0, scale=1.0, agg=0, want_scores=True, poison=False,
+               pool=1):
     rkv, runner, synth = mods
     dev = torch.device("cuda")
     caps = [l + extra for l in lens]
@@ -60,24 +61,24 @@ def make_layer(mods, lens, k_small, n_q, n_kv, extra=8, seed=0, scale=1.0, agg=0
                 r0 = int(cache.row_offset[b]) + h * caps[b]
                 cache.k[r0 + n: r0 + caps[b]] = float("nan")
                 cache.v[r0 + n: r0 + caps[b]] = float("nan")
-    ctx = rkv.Context(len(lens), n_q, n_kv, max(caps), max(max(k_small), 1) + extra, agg=agg)
+    ctx = rkv.Context(len(lens), n_q, n_kv, max(caps), max(max(k_small), 1) + extra, agg=agg, pool_kernel=pool)
     st = runner.LayerState(ctx, cache, k_small, extra, n_q, n_kv, want_scores=want_scores)
     q = (torch.randn((len(lens), n_q, 128), generator=g, device=dev)).to(torch.bfloat16)
     return ctx, st, cache, q
 
 
-def oracle_full(cache, b, n, q_b, n_kv, k_small, agg="max"):
+def oracle_full(cache, b, n, q_b, n_kv, k_small, agg="max", pool=1):
     k = O.bf16_bits_to_f64(host_heads(cache, b, n_kv, "k")[:, :n])
     v = O.bf16_bits_to_f64(host_heads(cache, b, n_kv, "v")[:, :n])
-    return O.full_step(O.bf16_bits_to_f64(bits(q_b)), k, v, k_small, agg=agg)
+    return O.full_step(O.bf16_bits_to_f64(bits(q_b)), k, v, k_small, agg=agg, pool=pool)
 
 
-def check_full_against_oracle(st, cache, q, lens, k_small, n_kv, agg="max", seqs=None):
+def check_full_against_oracle(st, cache, q, lens, k_small, n_kv, agg="max", seqs=None, pool=1):
     idx_host = st.topk_idx.cpu().numpy()
     scores = st.scores.cpu().numpy() if st.scores is not None else None
     for b in (range(len(lens)) if seqs is None else seqs):
         n = lens[b]
-        out, score, idx, _ = oracle_full(cache, b, n, q[b], n_kv, k_small[b], agg)
+        out, score, idx, _ = oracle_full(cache, b, n, q[b], n_kv, k_small[b], agg, pool)
         check_out(st.out[b], out, f"seq {b}")
         take = min(k_small[b], n)
         for g in range(n_kv):
@@ -129,6 +130,18 @@ def test_aggregation_modes(mods, agg, name):
     ctx, st, cache, q = make_layer(mods, lens, k_small, 16, 4, seed=5, agg=agg)
     st.refresh(q)
     check_full_against_oracle(st, cache, q, lens, k_small, 4, agg=name)
+
+
+@pytest.mark.parametrize("pool,agg,name", [(7, 0, "max"), (3, 0, "max"), (7, 1, "mean"), (31, 0, "max")])
+@pytest.mark.parametrize("lens,k_small,n_q,n_kv", [([1], [1], 4, 1), ([5, 64, 2049], [2, 16, 300], 28, 4),
+                                                  ([4096 + 37], [512], 8, 1), ([1000, 33], [100, 40], 32, 8)])
+def test_full_step_with_neighbour_max_pooling(mods, lens, k_small, n_q, n_kv, pool, agg, name):
+    """Scores max-pooled over `pool` neighbouring positions before the top-K (the paper's kernel size is 7):
+    windows clipped at both ends of the sequence and reaching across the slices of the selection cluster."""
+    ctx, st, cache, q = make_layer(mods, lens, k_small, n_q, n_kv, seed=7 * pool + n_q, agg=agg, pool=pool, poison=True)
+    st.refresh(q)
+    assert ctx.device_status() == 0
+    check_full_against_oracle(st, cache, q, lens, k_small, n_kv, agg=name, pool=pool)
 
 
 @pytest.mark.parametrize("cluster", [1, 0])
@@ -360,6 +373,10 @@ def test_host_side_argument_errors(mods):
         ctx.full_step(q, st.full_c, st.k_small, st.k_max, st.out, st.topk_idx, max_len_hint=10 ** 7)
     with pytest.raises(rkv.RkvError):
         rkv.Context(1, 8, 2, 100, 10, pool_kernel=4)
+    with pytest.raises(rkv.RkvError):
+        rkv.Context(1, 8, 2, 100, 10, pool_kernel=33)
+    with pytest.raises(rkv.RkvError):
+        rkv.Context(1, 8, 2, 200000, 10, pool_kernel=7)      # with pooling the length limit is 163840
 
 
 # ----------------------------------------------------------------------------- the five workload configs
