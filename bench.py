@@ -29,6 +29,11 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# DRAM traffic of one full-step attention launch per algorithmic K/V byte, from the ncu capture of the cfg-2
+# launch summarised in profiles/attn_kernel_full_step_cfg2_L32768.md (134.26 MB read + 4.88 MB written for
+# 134.22 MB of K/V); traffic grows with the positions streamed.  Set to None when the kernel changes.
+ATTN_FULL_TRAFFIC_PER_KV_BYTE = 139.14 / 134.22
+
 METRIC = "decode attention us/token (all layers, refresh schedule of the workload; full step and small step also reported)"
 UNIT = "us/token"
 
@@ -432,7 +437,9 @@ def run_ours(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": "attn_kernel<full> (full-cache attention + score logits)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_source": peak_src, "traffic": None,
+                     "peak_source": peak_src,
+                     "traffic": (kv_bytes_full * ATTN_FULL_TRAFFIC_PER_KV_BYTE
+                                 if ATTN_FULL_TRAFFIC_PER_KV_BYTE and args.workload == "cfg2" else None),
                      "algorithmic_bytes_per_launch": kv_bytes_full},
         "detail": {
             "always_full_us_per_token": full_token_us,
