@@ -324,12 +324,13 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, con
   const int per = (n_max + rkv::kSelectCluster - 1) / rkv::kSelectCluster;
   sp.per_cta = (per + 3) & ~3;
   sp.grid_splits = gx;
+  sp.per_fixed = ctx->cfg.n_seq == 1 ? 1 : 0;
   sp.pool_half = (ctx->cfg.pool_kernel - 1) / 2;
   sp.keys_cap = rkv::select_keys_cap(sp.per_cta);
   cudaError_t e;
   {
     LaunchScope scope(ctx, st, RKV_KERNEL_SELECT);
-    e = rkv::launch_select(sp, ctx->cfg.n_seq, st);
+    e = rkv::launch_select(sp, ctx->cfg.n_seq, ctx->sm_count, st);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
   ctx->launches += 1;

@@ -77,6 +77,7 @@ struct SelectParams {
   int32_t per_cta;            // positions per CTA of the cluster (from the host's length bound; multiple of 4)
   int32_t chunk, max_splits;  // split geometry of the attention launch that produced the partials
   int32_t grid_splits;        // CTAs per (sequence, KV head) that launch had
+  int32_t per_fixed;          // 1: slices are rank * per_cta (one sequence); 0: cut by each sequence's own length
   int32_t pool_half;          // (pool_kernel - 1) / 2
   int32_t keys_cap;           // padded key capacity of a CTA (offset of the unpooled keys in shared memory)
 };
@@ -92,7 +93,7 @@ cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_
                                      int n_seq, int cluster, cudaStream_t st);
 cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                             int n_seq, int cluster, cudaStream_t st);
-cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st);
+cudaError_t launch_select(const SelectParams& p, int n_seq, int sm_count, cudaStream_t st);
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
                           int32_t* status, cudaStream_t st);

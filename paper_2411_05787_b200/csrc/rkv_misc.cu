@@ -37,17 +37,36 @@ __global__ void __launch_bounds__(256) gather_kernel(const int32_t* __restrict__
   uint4* sk = static_cast<uint4*>(small_cache.k);
   uint4* sv = static_cast<uint4*>(small_cache.v);
   const int sub = threadIdx.x & 15;
-  for (int r = blockIdx.x * 16 + (threadIdx.x >> 4); r < m; r += gridDim.x * 16) {
-    const int j = idx[r];
-    if (j < 0) continue;
-    if (j >= n) {
-      if (sub == 0) atomicOr(status, RKV_DEV_BAD_INDEX);
-      continue;
+  // four rows per thread and round: first all indices, then all eight 16-byte loads, then the stores, so that a
+  // round costs two memory round trips however many rows it moves
+  const int stride = gridDim.x * 16;
+  for (int r0 = blockIdx.x * 16 + (threadIdx.x >> 4); r0 < m; r0 += 4 * stride) {
+    int j[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + u * stride;
+      j[u] = (r < m) ? idx[r] : -1;
     }
-    const uint4 kv = __ldcs(fk + (src0 + j) * 16 + sub);
-    const uint4 vv = __ldcs(fv + (src0 + j) * 16 + sub);
-    sk[(dst0 + r) * 16 + sub] = kv;
-    sv[(dst0 + r) * 16 + sub] = vv;
+    uint4 kv[4], vv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (j[u] >= n) {
+        if (sub == 0) atomicOr(status, RKV_DEV_BAD_INDEX);
+        j[u] = -1;
+      }
+      if (j[u] >= 0) {
+        kv[u] = __ldcs(fk + (src0 + j[u]) * 16 + sub);
+        vv[u] = __ldcs(fv + (src0 + j[u]) * 16 + sub);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (j[u] >= 0) {
+        const int r = r0 + u * stride;
+        sk[(dst0 + r) * 16 + sub] = kv[u];
+        sv[(dst0 + r) * 16 + sub] = vv[u];
+      }
+    }
   }
 }
 
@@ -142,7 +161,7 @@ __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __res
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
                           int32_t* status, cudaStream_t st) {
-  int gx = (k_max + 15) / 16;
+  int gx = (k_max + 63) / 64;   // a thread moves up to four rows per round
   if (gx > 64) gx = 64;
   if (gx < 1) gx = 1;
   dim3 grid(gx, n_kv_heads, n_seq);

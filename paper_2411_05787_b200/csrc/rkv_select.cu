@@ -181,8 +181,10 @@ __device__ __forceinline__ void merge_locate(SelectShared* sh, int buf, uint32_t
   __syncthreads();
 }
 
-template <int GP>   // floats per position in the logit scratch: 4 (G <= 4) or 8
-__global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
+// GP: floats per position in the logit scratch, 4 (G <= 4) or 8.  kMinBlocks = 2 trades a few spilled
+// registers for two resident CTAs per SM: with more clusters than one wave holds, their latency chains overlap.
+template <int GP, int kMinBlocks>
+__global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int rank = (int)cluster_rank();
   const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -198,12 +200,16 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   }
   const int G = p.group;
   const int bg = b * p.n_kv_heads + g;
-  const int per = p.per_cta;                  // positions per CTA, fixed by the host from its length bound
-  const int lo = rank * per;
+  // Positions per CTA: with one sequence the host fixes the slices from its length bound, so the first logits
+  // can be requested before the length arrives; with a batch (ragged lengths) each sequence is cut in eight
+  // by its own length once that is known, so that short sequences still use the whole cluster.
+  const bool per_fixed = p.per_fixed != 0;
+  int per = p.per_cta;
+  int lo = rank * per;
   const float* pbase = p.partials + (int64_t)bg * p.max_splits * PartialLayout::kFloats;
   const int half = p.pool_half;               // neighbour max-pooling of the scores over 2*half+1 positions (0: none)
   // keys are made for positions lo-half .. lo+per+half-1 (the pooling window reaches into the neighbours' slices)
-  const float* lg = p.logits + ((int64_t)bg * p.logit_stride + lo - half) * GP;
+  const float* lg = p.logits + ((int64_t)bg * p.logit_stride + lo - half) * GP;   // re-based below if the slices move
   uint32_t* raw = half > 0 ? keys + p.keys_cap : keys;   // unpooled keys; the same array when there is no pooling
   constexpr int U = 32 / GP;                  // positions per thread per round: all their loads are in flight together
   const int gx = p.grid_splits;               // splits the attention launch had room for (>= the sequence's own count)
@@ -248,7 +254,7 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
         dst[u][c] = on ? __ldcg(reinterpret_cast<const float4*>(lg + (int64_t)i * GP) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
-  load_round(v, 0);
+  if (per_fixed) load_round(v, 0);
 
   if (act == 0) return;   // same decision in all CTAs of the cluster
   {
@@ -263,6 +269,12 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   if (n == 0) {   // the attention kernel has zeroed out[]
     for (int i = rank * NT + tid; i < p.k_max; i += kSelectCluster * NT) idx_out[i] = -1;
     return;
+  }
+  if (!per_fixed) {
+    per = (((n + kSelectCluster - 1) / kSelectCluster) + 3) & ~3;   // never above the host's per_cta (n <= its bound)
+    lo = rank * per;
+    lg = p.logits + ((int64_t)bg * p.logit_stride + lo - half) * GP;
+    load_round(v, 0);
   }
   const int cnt = (n - lo < 0) ? 0 : (n - lo < per ? n - lo : per);
   const int R = (((cnt + NT - 1) / NT) + 3) & ~3;   // keys per thread in the ordered phases (multiple of 4)
@@ -587,18 +599,25 @@ size_t select_smem_bytes(int keys_per_cta, int pool_half) {
 }
 
 cudaError_t prepare_select() {
-  cudaError_t e = cudaFuncSetAttribute(select_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)select_smem_bytes(kSelectMaxKeysPerCta, 0));
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)select_smem_bytes(kSelectMaxKeysPerCta, 0));
+  const int bytes = (int)select_smem_bytes(kSelectMaxKeysPerCta, 0);
+  cudaError_t e = cudaFuncSetAttribute(select_kernel<4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  return e;
 }
 
-cudaError_t launch_select(const SelectParams& p, int n_seq, cudaStream_t st) {
+cudaError_t launch_select(const SelectParams& p, int n_seq, int sm_count, cudaStream_t st) {
   const dim3 grid(kSelectCluster, p.n_kv_heads, n_seq);
-  if (p.group <= 4)
-    return launch_ex(select_kernel<4>, grid, dim3(NT), select_smem_bytes(p.per_cta, p.pool_half), st, kSelectCluster, p);
-  return launch_ex(select_kernel<8>, grid, dim3(NT), select_smem_bytes(p.per_cta, p.pool_half), st, kSelectCluster, p);
+  const size_t smem = select_smem_bytes(p.per_cta, p.pool_half);
+  // two CTAs per SM when one wave cannot hold every cluster and two CTAs' shared memory fits
+  const bool dense = (int64_t)kSelectCluster * p.n_kv_heads * n_seq > sm_count && 2 * (smem + 1024) <= 227 * 1024;
+  if (p.group <= 4) {
+    if (dense) return launch_ex(select_kernel<4, 2>, grid, dim3(NT), smem, st, kSelectCluster, p);
+    return launch_ex(select_kernel<4, 1>, grid, dim3(NT), smem, st, kSelectCluster, p);
+  }
+  if (dense) return launch_ex(select_kernel<8, 2>, grid, dim3(NT), smem, st, kSelectCluster, p);
+  return launch_ex(select_kernel<8, 1>, grid, dim3(NT), smem, st, kSelectCluster, p);
 }
 
 }  // namespace rkv
