@@ -237,7 +237,7 @@ def run_ours(args):
     dynamic = w.schedule == "dynamic"
     n_prof = 2 * S
     # tokens decoded over all phases: main loop, e2e loop, always-full loop, small-only loop, profiling
-    total_tokens = 2 * (args.steps + args.warmup) + 10 + 23 + 2 * S + n_prof + 8
+    total_tokens = 2 * (args.steps + args.warmup) + 10 + 23 + 21 + 2 * S + n_prof + 8
     wl = synth.scaled(w, steps=total_tokens)
     k_max = max(w.k_small)
     full_hint = max(w.lens) + total_tokens + 1
@@ -290,6 +290,9 @@ def run_ours(args):
             if kind == "full":
                 st.append(kn, vn)
                 st.refresh(q, max_len_hint=full_hint)
+            elif kind == "score":      # score-only refresh: K-only pass + top-K, rebuild, attention over the new small cache
+                st.append(kn, vn)
+                st.refresh_scores_only(q, max_len_hint=full_hint, small_hint=small_hint)
             elif kind == "small":      # append + partial step in one call (one launch)
                 st.append_partial(q, kn, vn, max_len_hint=small_hint)
             else:                      # check: the trigger decides per sequence; both branches run under its masks
@@ -301,7 +304,7 @@ def run_ours(args):
     # initial small caches + eager warm-up of every kernel (also creates the tensor maps)
     for l, st in enumerate(layers):
         st.refresh(q_stage[l], max_len_hint=full_hint)
-    kinds = ["small", "full"] + (["check"] if dynamic else [])
+    kinds = ["small", "full", "score"] + (["check"] if dynamic else [])
     for kind in kinds:
         token(kind)
     torch.cuda.synchronize()
@@ -321,7 +324,9 @@ def run_ours(args):
 
     tok_counter = [1]
 
-    def kind_of(t, always_full, force_small):
+    def kind_of(t, always_full, force_small, force_kind=None):
+        if force_kind:
+            return force_kind
         if force_small:
             return "small"
         if always_full:
@@ -330,14 +335,14 @@ def run_ours(args):
             return "small"
         return "check" if dynamic else "full"
 
-    def run_tokens(n, e2e=False, always_full=False, force_small=False):
+    def run_tokens(n, e2e=False, always_full=False, force_small=False, force_kind=None):
         """Enqueue n decode tokens; returns the count of each kind."""
         cnt = {k: 0 for k in kinds}
         for _ in range(n):
             t = tok_counter[0]; tok_counter[0] += 1
             src = inputs_host if e2e else inputs_dev
             stage.copy_(src[t % n_in], non_blocking=True)
-            kind = kind_of(t, always_full, force_small)
+            kind = kind_of(t, always_full, force_small, force_kind)
             graphs[kind].replay()
             if e2e:
                 outs_host.copy_(outs, non_blocking=True)
@@ -386,6 +391,8 @@ def run_ours(args):
     run_tokens(3, always_full=True)
     ms_full, _ = timed(20, always_full=True)
     full_token_us = ms_full * 1000.0 / (20 * world)
+    ms_score, _ = timed(20, force_kind="score")    # every token refreshes from scores alone (K half of the cache)
+    run_tokens(1, always_full=True)
     ms_small, _ = timed(S - 1, force_small=True)   # right after a full token: K .. K+S-2 rows
     run_tokens(1, always_full=True)
     # ---- per-kernel device time: every launch bracketed by CUDA events on its stream (fixed-stride schedule,
@@ -453,6 +460,7 @@ def run_ours(args):
             "small_step_frac_of_8TBs": kv_bytes_small / (small_us * 1e-6) / 8e12,
             "attn_full_frac_of_8TBs": achieved / 8000.0,
             "in_graph_us_per_layer": {"full_token": full_token_us / NL,
+                                      "score_only_refresh_token": ms_score * 1000.0 / (20 * world) / NL,
                                       "small_token": ms_small * 1000.0 / ((S - 1) * world) / NL},
             "device_status": status,
             "graph_launches": launches_per,

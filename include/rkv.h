@@ -126,6 +126,19 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*ho
                          void* q_last_full, int32_t max_len_hint, void* stream);
 
 /*
+ * Score-only refresh step (Sec. 4.2 "Impact of full attention steps", the "w/o full attention" setting:
+ * at the stride the attention scores over the entire cache update the partial cache, and the step then
+ * attends to the UPDATED partial cache instead of the full one; the paper reports the same quality as
+ * the regular method).  Computes exactly the scores / topk_idx / q_last_full of rkv_full_step but reads
+ * the K half of C_f only and produces no attention output: half the bytes of a full step.  The caller
+ * follows it with rkv_gather_small and rkv_small_step.  Arguments as in rkv_full_step (without out).
+ */
+rkv_status rkv_score_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
+                          const int32_t* k_small, int32_t k_max, const int32_t* active, float* scores,
+                          int64_t score_stride, int32_t* topk_idx, void* q_last_full, int32_t max_len_hint,
+                          void* stream);
+
+/*
  * Rebuild C_p from the selected positions (Sec. 2.2 "refresh the partial
  * cache").  For active b, KV head g, r < m = min(k_small[b], full->len[b]):
  *   small.K[b][g][r] = full.K[b][g][topk_idx[b][g][r]]   (same for V; bit copy)

@@ -179,6 +179,18 @@ def full_step(q, k, v, k_small_size, *, agg="max", pool=1, scale=None):
     return out, score, idx, lse
 
 
+def score_only_step(q, k, v, k_small_size, *, agg="max", pool=1, scale=None):
+    """The "w/o full attention" refresh of Sec. 4.2: scores over the whole cache pick the top-K positions,
+    and the step's output is attention over those K positions only.  Returns (out, score, idx)."""
+    _, score, idx, _ = full_step(q, k, v, k_small_size, agg=agg, pool=pool, scale=scale)
+    v = np.asarray(v, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    ks = np.stack([k[g, idx[g]] for g in range(k.shape[0])])
+    vs = np.stack([v[g, idx[g]] for g in range(k.shape[0])])
+    out, _, _ = decode_attention(q, ks, vs, scale)
+    return out, score, idx
+
+
 def gather_rows(cache: np.ndarray, idx: list[np.ndarray]) -> list[np.ndarray]:
     """small[g][r] = cache[g, idx[g][r]] (bit copy; works on uint16 or float arrays)."""
     return [cache[g, idx[g]] for g in range(cache.shape[0])]

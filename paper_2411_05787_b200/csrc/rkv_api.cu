@@ -153,7 +153,7 @@ bool cluster_eligible(const rkv_ctx* ctx, int n_max) { return ctx->small_cluster
 
 rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
                          int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out, int* gx_out,
-                         const AppendArgs* app = nullptr) {
+                         const AppendArgs* app = nullptr, bool score_only = false) {
   CUtensorMap tm_k, tm_v;
   rkv_status s = tensor_map(ctx, cache->k, cache->n_rows, &tm_k);
   if (s != RKV_OK) return s;
@@ -211,6 +211,7 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   {
     LaunchScope scope(ctx, st, logits ? RKV_KERNEL_ATTN_FULL : RKV_KERNEL_ATTN_SMALL);
     e = app != nullptr ? rkv::launch_attention_cluster_append(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
+        : score_only   ? rkv::launch_attention_scores(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
         : cluster      ? rkv::launch_attention_cluster(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
                        : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
   }
@@ -285,17 +286,18 @@ rkv_status rkv_destroy(rkv_ctx* ctx) {
   return e == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 
-rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
-                         const int32_t* active, void* out, float* scores, int64_t score_stride, int32_t* topk_idx,
-                         void* q_last_full, int32_t max_len_hint, void* stream) {
-  if (!ctx || !q || !cache_ok(full) || !k_small || !out || !topk_idx) return RKV_ERR_INVALID_ARG;
+static rkv_status full_step_impl(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small,
+                                 int32_t k_max, const int32_t* active, void* out, float* scores, int64_t score_stride,
+                                 int32_t* topk_idx, void* q_last_full, int32_t max_len_hint, void* stream,
+                                 bool score_only) {
+  if (!ctx || !q || !cache_ok(full) || !k_small || (!out && !score_only) || !topk_idx) return RKV_ERR_INVALID_ARG;
   if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
   int n_max = max_len_hint == 0 ? ctx->cfg.max_len : max_len_hint;
   if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
   if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int chunk = 0, gx = 1;
-  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx);
+  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, nullptr, score_only);
   if (s != RKV_OK) return s;
   SelectParams sp;
   memset(&sp, 0, sizeof(sp));
@@ -335,6 +337,20 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, con
   if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
   ctx->launches += 1;
   return RKV_OK;
+}
+
+rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
+                         const int32_t* active, void* out, float* scores, int64_t score_stride, int32_t* topk_idx,
+                         void* q_last_full, int32_t max_len_hint, void* stream) {
+  return full_step_impl(ctx, q, full, k_small, k_max, active, out, scores, score_stride, topk_idx, q_last_full,
+                        max_len_hint, stream, false);
+}
+
+rkv_status rkv_score_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
+                          const int32_t* active, float* scores, int64_t score_stride, int32_t* topk_idx,
+                          void* q_last_full, int32_t max_len_hint, void* stream) {
+  return full_step_impl(ctx, q, full, k_small, k_max, active, nullptr, scores, score_stride, topk_idx, q_last_full,
+                        max_len_hint, stream, true);
 }
 
 rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t* k_small, int32_t k_max,

@@ -15,7 +15,8 @@
 // O^T += V^T P^T with m16n8k16 bf16 tensor-core MMAs (fp32 accumulate), where
 // the N=8 dimension holds all query heads of the group, so K/V are read once
 // per group.  Online softmax lives in registers.  Three ways to merge the splits:
-//   full step      partials go to the workspace, the selection kernel folds them;
+//   full step      partials go to the workspace, the selection kernel folds them (the score-only
+//                  variant of the full step streams K alone: logits and softmax statistics, no output);
 //   partial step   (a) the CTAs of one (sequence, KV head) form a thread-block cluster:
 //                  each pushes its slice of the partial output into the peer that owns
 //                  that slice through distributed shared memory, one cluster barrier,
@@ -41,7 +42,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kOPad = 132;  // floats per head row in the merge buffer (bank spread)
 constexpr int kRecvFloats = kMaxGroup * kHeadDim + kAttnCluster * kMaxGroup * 2;   // pushed slices + (m, l) pairs
 
-enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2, kModeClusterAppend = 3 };
+enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2, kModeClusterAppend = 3, kModeScore = 4 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -135,7 +136,8 @@ template <int kMode>
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
             const AttnParams p) {
-  constexpr bool kLogits = (kMode == kModeFull);
+  constexpr bool kLogits = (kMode == kModeFull || kMode == kModeScore);
+  constexpr bool kScoreOnly = (kMode == kModeScore);   // logits and softmax statistics only: V is never read
   constexpr bool kCluster = (kMode == kModeCluster || kMode == kModeClusterAppend);
   constexpr bool kAppend = (kMode == kModeClusterAppend);
   extern __shared__ uint8_t smem_raw[];
@@ -278,11 +280,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         const uint32_t dst = smem_base + s * kStageBytes;
         const uint32_t bar = bar_full + 8 * s;
         const int y = (int)(row0 + (int64_t)t * kTile);
-        mbar_expect_tx(bar, kStageBytes);
+        mbar_expect_tx(bar, kScoreOnly ? 2 * kHalfBytes : kStageBytes);
         tma_load_2d(dst, &tm_k, 0, y, bar, policy);
         tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar, policy);
-        tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
-        tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
+        if (!kScoreOnly) {
+          tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
+          tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
+        }
       }
     }
     if (kCluster) {   // stay until the peers have pushed: every warp of the cluster meets at one barrier
@@ -376,6 +380,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       const float p2 = ex2(fmaf(s2, kLog2e, nm0)), p3 = ex2(fmaf(s3, kLog2e, nm1));
       l0 += p0 + p2;
       l1 += p1 + p3;
+      if (!kScoreOnly) {
       // P^T as the B operand: transpose the two 8x8 [position][head] blocks inside the warp
       const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1));
       const uint32_t pb1 = movmatrix_t(pack_bf16(p2, p3));
@@ -399,6 +404,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
           a[3] &= mk1;
         }
         mma_bf16(o[mt], a, pb0, pb1);
+      }
       }
     }
     __syncwarp();
@@ -503,9 +509,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   const bool single = (kMode == kModeTicket) && n_splits == 1;   // the full step always leaves its partials to the selector
   if (!single) {
     float* part = p.partials + ((int64_t)bg * p.max_splits + split) * PartialLayout::kFloats;
+    if (!kScoreOnly) {
 #pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h)
-      if (h < G) part[h * kHeadDim + d] = accO[h];
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h < G) part[h * kHeadDim + d] = accO[h];
+    }
     if (d < kMaxGroup) {
       float Md = ninf, Ld = 0.f;
 #pragma unroll
@@ -563,6 +571,8 @@ cudaError_t prepare_attention() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_kernel<kModeTicket>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_kernel<kModeScore>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_kernel<kModeCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(attn_kernel<kModeClusterAppend>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
@@ -574,6 +584,12 @@ cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const
   if (write_logits)
     return launch_ex(attn_kernel<kModeFull>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
   return launch_ex(attn_kernel<kModeTicket>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
+}
+
+cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                    int n_seq, int grid_x, cudaStream_t st) {
+  dim3 grid(grid_x, p.n_kv_heads, n_seq);
+  return launch_ex(attn_kernel<kModeScore>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
 }
 
 cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,

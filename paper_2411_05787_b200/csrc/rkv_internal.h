@@ -91,6 +91,8 @@ cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const
                              int n_seq, int grid_x, bool write_logits, cudaStream_t st);
 cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                      int n_seq, int cluster, cudaStream_t st);
+cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                    int n_seq, int grid_x, cudaStream_t st);
 cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                             int n_seq, int cluster, cudaStream_t st);
 cudaError_t launch_select(const SelectParams& p, int n_seq, int sm_count, cudaStream_t st);

@@ -216,6 +216,7 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
   // slice of out[] this CTA folds: 16*G consecutive (head, channel) pairs of the group
   const int o_local = tid & 127, sgrp = tid >> 7;
   const bool o_on = o_local < 16 * G;
+  const bool fold_on = o_on && p.out != nullptr;   // the score-only step has no attention output to fold
   const int o_flat = rank * 16 * G + o_local;
   const int64_t hrow0 = ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
   pdl_wait();
@@ -238,7 +239,7 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
 #pragma unroll
   for (int k = 0; k < kOPre; ++k) {
     const int s = sgrp + 4 * k;
-    opre[k] = (o_on && s < gx) ? __ldcg(pbase + (int64_t)s * PartialLayout::kFloats + o_flat) : 0.f;
+    opre[k] = (fold_on && s < gx) ? __ldcg(pbase + (int64_t)s * PartialLayout::kFloats + o_flat) : 0.f;
   }
   __nv_bfloat16 qv = __float2bfloat16(0.f);
   if (p.q_last_full != nullptr && sgrp == 0 && o_on) qv = static_cast<const __nv_bfloat16*>(p.q)[hrow0 + o_flat];
@@ -312,7 +313,7 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
   auto fold_slice = [&] {
     const int h = o_flat >> 7;
     float acc = 0.f;
-    if (o_on) {
+    if (fold_on) {
 #pragma unroll
       for (int k = 0; k < kOPre; ++k) {
         const int s = sgrp + 4 * k;
@@ -325,7 +326,7 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
     __syncthreads();
     if (sgrp == 0 && o_on) {
       const float o = (sh->red[0][o_local] + sh->red[1][o_local]) + (sh->red[2][o_local] + sh->red[3][o_local]);
-      static_cast<__nv_bfloat16*>(p.out)[hrow0 + o_flat] = __float2bfloat16(o * sh->linv[h]);
+      if (fold_on) static_cast<__nv_bfloat16*>(p.out)[hrow0 + o_flat] = __float2bfloat16(o * sh->linv[h]);
       if (p.q_last_full != nullptr) static_cast<__nv_bfloat16*>(p.q_last_full)[hrow0 + o_flat] = qv;
     }
     for (int i = kk + rank * NT + tid; i < p.k_max; i += kSelectCluster * NT) idx_out[i] = -1;   // padding

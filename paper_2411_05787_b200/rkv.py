@@ -21,7 +21,7 @@ DEV_APPEND_OVERFLOW, DEV_LEN_CLAMPED, DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT 
 EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", "rkv_gather_small",
            "rkv_small_step", "rkv_append", "rkv_should_refresh", "rkv_get_device_status",
            "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
-           "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step"]
+           "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step", "rkv_score_step"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER = 1, 2, 3
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
@@ -50,6 +50,8 @@ def _load() -> ctypes.CDLL:
     lib.rkv_workspace_bytes.argtypes = [cfgp]
     lib.rkv_workspace_bytes.restype = ctypes.c_size_t
     lib.rkv_full_step.argtypes = [vp, vp, cachep, vp, i32, vp, vp, vp, i64, vp, vp, i32, vp]
+    lib.rkv_score_step.argtypes = [vp, vp, cachep, vp, i32, vp, vp, i64, vp, vp, i32, vp]
+    lib.rkv_score_step.restype = i32
     lib.rkv_gather_small.argtypes = [vp, vp, vp, i32, cachep, cachep, vp, vp]
     lib.rkv_small_step.argtypes = [vp, vp, cachep, vp, vp, i32, vp]
     lib.rkv_append.argtypes = [vp, vp, vp, cachep, cachep, vp]
@@ -164,6 +166,13 @@ class Context:
         self._check(lib.rkv_full_step(self._h, _ptr(q), ctypes.byref(full), _ptr(k_small), k_max, _ptr(active),
                                       _ptr(out), _ptr(scores), stride, _ptr(topk_idx), _ptr(q_last_full),
                                       max_len_hint, _stream(stream)))
+
+    def score_step(self, q, full: RkvCache, k_small, k_max, topk_idx, active=None, scores=None, q_last_full=None,
+                   max_len_hint=0, stream=None):
+        stride = scores.shape[-1] if scores is not None else 0
+        self._check(lib.rkv_score_step(self._h, _ptr(q), ctypes.byref(full), _ptr(k_small), k_max, _ptr(active),
+                                       _ptr(scores), stride, _ptr(topk_idx), _ptr(q_last_full), max_len_hint,
+                                       _stream(stream)))
 
     def gather_small(self, topk_idx, k_small, k_max, full: RkvCache, small: RkvCache, active=None, stream=None):
         self._check(lib.rkv_gather_small(self._h, _ptr(topk_idx), _ptr(k_small), k_max, ctypes.byref(full),

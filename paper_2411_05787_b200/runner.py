@@ -44,6 +44,14 @@ class LayerState:
         self.ctx.gather_small(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c, active=active)
         return self.out
 
+    def refresh_scores_only(self, q, active=None, max_len_hint=0, small_hint=0):
+        """Score-only refresh: scores and top-K from K alone, rebuild of the small cache, attention over the new one."""
+        self.ctx.score_step(q, self.full_c, self.k_small, self.k_max, self.topk_idx, active=active, scores=self.scores,
+                            q_last_full=self.q_last_full, max_len_hint=max_len_hint)
+        self.ctx.gather_small(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c, active=active)
+        self.ctx.small_step(q, self.small_c, self.out, active=active, max_len_hint=small_hint)
+        return self.out
+
     def partial(self, q, active=None, max_len_hint=0):
         self.ctx.small_step(q, self.small_c, self.out, active=active, max_len_hint=max_len_hint)
         return self.out

@@ -406,3 +406,20 @@ def test_pins_catch_planted_mistakes():
     a, b = r.normal(size=(4, 8)), r.normal(size=(4, 8))
     per_head = np.mean([a[h] @ b[h] / np.linalg.norm(a[h]) / np.linalg.norm(b[h]) for h in range(4)])
     assert abs(per_head - O.cosine_similarity(a, b)) > 1e-3
+
+
+def test_score_only_step_pins():
+    """Sec. 4.2 "w/o full attention": same selection as the full step; output = attention over the selected rows.
+    With K = L it is the full step; with one dominant key the two outputs nearly coincide."""
+    q, k, v = _rand_case(31, n_q=4, n_kv=2, n=40, d=128)
+    full_out, score, idx, _ = O.full_step(q, k, v, 9)
+    out, score2, idx2 = O.score_only_step(q, k, v, 9)
+    assert all(np.array_equal(a, b) for a, b in zip(idx, idx2)) and np.array_equal(score, score2)
+    assert not np.allclose(out, full_out, atol=1e-6)          # 9 of 40 positions: a different softmax
+    out_all, _, _ = O.score_only_step(q, k, v, 40)
+    assert np.allclose(out_all, full_out, atol=1e-12)
+    # renormalised probabilities over the kept set: by hand for head 0
+    p = O.softmax_rows(O.attention_logits(q, k))[0][0]
+    keep = idx[0]
+    want = (p[keep] / p[keep].sum()) @ v[0, keep]
+    assert np.allclose(out[0], want, atol=1e-12)

@@ -246,6 +246,32 @@ def test_fused_append_small_step_equals_append_then_small_step(mods, n_small):
     assert fu_a.len.tolist() == [102, 43, 9] and sm_a.len.tolist() == [n_small + 3, n_small // 2 + 2, 8]
 
 
+@pytest.mark.parametrize("lens,k_small,n_q,n_kv", [([3000, 70], [300, 64], 32, 8), ([4096 + 37, 1], [512, 1], 28, 4)])
+def test_score_only_refresh_step(mods, lens, k_small, n_q, n_kv):
+    """rkv_score_step (K only) selects exactly what rkv_full_step selects; followed by the rebuild and a partial
+    step it gives the oracle's "w/o full attention" output."""
+    ctx, st, cache, q = make_layer(mods, lens, k_small, n_q, n_kv, seed=21, poison=True)
+    st.refresh(q)
+    idx_full, sc_full = st.topk_idx.clone(), st.scores.clone()
+    st.topk_idx.fill_(-9); st.scores.fill_(-1.0); st.out.fill_(5.0); st.q_last_full.fill_(0.0)
+    out = st.refresh_scores_only(q).clone()
+    assert ctx.device_status() == 0
+    assert torch.equal(st.topk_idx, idx_full) and torch.equal(st.q_last_full, q)
+    for b, n in enumerate(lens):
+        assert torch.equal(st.scores[b, :, :n], sc_full[b, :, :n])
+        k = O.bf16_bits_to_f64(host_heads(cache, b, n_kv, "k")[:, :n])
+        v = O.bf16_bits_to_f64(host_heads(cache, b, n_kv, "v")[:, :n])
+        # the oracle's output on the GPU's own (validated) selection, so that ties cannot differ
+        want_out, score, _ = O.score_only_step(O.bf16_bits_to_f64(bits(q[b])), k, v, k_small[b])
+        take = min(k_small[b], n)
+        sel = [st.topk_idx[b, g, :take].cpu().numpy().astype(np.int64) for g in range(n_kv)]
+        for g in range(n_kv):
+            assert O.check_topk_set(score[g], k_small[b], sel[g]) is None
+        ks = np.stack([k[g, sel[g]] for g in range(n_kv)]); vs = np.stack([v[g, sel[g]] for g in range(n_kv)])
+        want, _, _ = O.decode_attention(O.bf16_bits_to_f64(bits(q[b])), ks, vs)
+        check_out(out[b], want, f"score-only step seq {b}")
+
+
 def test_append_and_overflow_flag(mods):
     rkv, runner, synth = mods
     lens, k_small = [40, 9], [8, 4]
