@@ -188,6 +188,33 @@ rkv_status rkv_append_small_step(rkv_ctx* ctx, const void* q, const void* k_new,
                                  void* out, int32_t max_len_hint, void* stream);
 
 /*
+ * Fixed-size partial cache (Sec. 2.2 "Decoding with partial cache": to keep |C_p| = K while decoded tokens
+ * are stored, the entry with the lowest attention score of the last full step is removed for each new
+ * token).  Two calls replace rkv_gather_small / rkv_append_small_step:
+ *
+ * rkv_gather_small_evict  = rkv_gather_small, and additionally, from the scores of the rkv_full_step /
+ *   rkv_score_step issued just before on the same context and stream, the eviction order of the rebuilt
+ *   cache: evict_order[b][g][i] = row of the small cache (0 .. m-1) that the i-th new token will replace,
+ *   lowest score first, the later position first among equal scores; -1 beyond m.  evict_count[b] <- 0.
+ * rkv_append_small_step_evict = rkv_append_small_step, except that a sequence whose small cache has
+ *   reached k_small[b] rows does not grow: the new row overwrites row evict_order[b][g][evict_count[b]]
+ *   of every KV head and evict_count[b] += 1 (a shorter cache still grows).  After max_evict evictions
+ *   without a refresh the row is not stored in the small cache and RKV_DEV_APPEND_OVERFLOW is set.
+ *   evict_order  int32 [B][Hkv][max_evict];  evict_count  int32 [B];  max_evict  host value, 1..4096
+ *   k_max <= 4096.  Needs the clustered partial step (RKV_OPT_SMALL_CLUSTER on, length bound <= 8192).
+ */
+rkv_status rkv_gather_small_evict(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t* k_small, int32_t k_max,
+                                  const rkv_cache* full /*host struct*/, const rkv_cache* small_cache /*host struct*/,
+                                  const int32_t* active, int32_t* evict_order, int32_t* evict_count,
+                                  int32_t max_evict, void* stream);
+rkv_status rkv_append_small_step_evict(rkv_ctx* ctx, const void* q, const void* k_new, const void* v_new,
+                                       const rkv_cache* full /*host struct or NULL*/,
+                                       const rkv_cache* small_cache /*host struct*/, const int32_t* k_small,
+                                       const int32_t* active, void* out, const int32_t* evict_order,
+                                       int32_t* evict_count, int32_t max_evict, int32_t max_len_hint,
+                                       void* stream);
+
+/*
  * Refresh trigger (Sec. 2.2 "Deciding when to decode with full cache").
  *   qbar  = mean over the Hq heads of q_now[b];  qbar' likewise from q_last_full[b]
  *   sim   = <qbar, qbar'> / (|qbar| |qbar'|)          (fp32)

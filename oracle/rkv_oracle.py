@@ -237,8 +237,12 @@ class SequenceState:
 
     k_full, v_full: uint16 [Hkv, cap, d]; len_full positions valid.
     k_small, v_small: per KV head uint16 [cap_small, d]; len_small rows valid.
-    The small cache grows by one row per appended token until the next
-    refresh (reading taken here: no per-step eviction; see `evict` below).
+    By default the small cache grows by one row per appended token until the
+    next refresh.  With evict=True it keeps the paper's fixed size (Sec. 2.2
+    "Decoding with partial cache"): once it holds k_small_size rows, each new
+    token replaces the surviving entry that had the lowest attention score in
+    the last full step (among equal scores the later position goes first);
+    tokens appended since that step carry no score and are never the victim.
     """
     k_full: np.ndarray
     v_full: np.ndarray
@@ -246,6 +250,8 @@ class SequenceState:
     k_small_size: int
     agg: str = "max"
     pool: int = 1
+    evict: bool = False
+    evict_queue: list = field(default_factory=list)   # per KV head: small-cache rows in eviction order
     k_small: list = field(default_factory=list)
     v_small: list = field(default_factory=list)
     small_pos: list = field(default_factory=list)   # position in C_f of every small row
@@ -261,7 +267,13 @@ class SequenceState:
             raise IndexError("full cache capacity exceeded")
         self.k_full[:, self.len_full] = k_new
         self.v_full[:, self.len_full] = v_new
-        if to_small and self.k_small:
+        if to_small and self.k_small and self.evict and self.len_small >= self.k_small_size > 0:
+            for g in range(self.k_full.shape[0]):
+                slot = self.evict_queue[g].pop(0)          # lowest-scoring survivor of the last full step
+                self.k_small[g][slot] = k_new[g]
+                self.v_small[g][slot] = v_new[g]
+                self.small_pos[g][slot] = self.len_full
+        elif to_small and self.k_small:
             for g in range(self.k_full.shape[0]):
                 self.k_small[g] = np.concatenate([self.k_small[g], k_new[g][None]], axis=0)
                 self.v_small[g] = np.concatenate([self.v_small[g], v_new[g][None]], axis=0)
@@ -279,6 +291,8 @@ class SequenceState:
         self.v_small = gather_rows(self.v_full, idx)
         self.small_pos = [i.copy() for i in idx]
         self.len_small = len(idx[0])
+        # rows are in rank order (score descending, position ascending): the victims come from the back
+        self.evict_queue = [list(range(len(i) - 1, -1, -1)) for i in idx]
         self.q_last_full = q
         self.positions_touched += self.len_full
         self.n_full_steps += 1

@@ -38,7 +38,7 @@ int splits_for(const rkv_config* c) {
   return s < rkv::kMaxSplits ? (s < 1 ? 1 : s) : rkv::kMaxSplits;
 }
 
-struct WsLayout { size_t partials, tickets, len_tickets, logits, status, total; int64_t logit_stride; };
+struct WsLayout { size_t partials, tickets, len_tickets, win_keys, logits, status, total; int64_t logit_stride; };
 
 WsLayout ws_layout(const rkv_config* c) {
   WsLayout w;
@@ -50,6 +50,7 @@ WsLayout ws_layout(const rkv_config* c) {
   w.partials = off; off = up(off + bg * splits_for(c) * rkv::PartialLayout::kFloats * sizeof(float));
   w.tickets = off;  off = up(off + bg * sizeof(int32_t));
   w.len_tickets = off; off = up(off + (size_t)c->n_seq * sizeof(int32_t));
+  w.win_keys = off; off = up(off + bg * (size_t)c->max_small * sizeof(uint32_t));
   const int gp = group <= 4 ? 4 : 8;   // position-major logits, padded to a vector width
   w.logits = off;   off = up(off + bg * gp * (size_t)w.logit_stride * sizeof(float));
   w.status = off;   off = up(off + sizeof(int32_t));
@@ -147,7 +148,10 @@ int choose_chunk(const rkv_ctx* ctx, int n_max, bool full, int* grid_x) {
 // Longest small cache that the clustered partial step takes (8 CTAs x 1024 positions).
 constexpr int kClusterMaxLen = 8192;
 
-struct AppendArgs { const void* k_new; const void* v_new; const rkv_cache* full; };
+struct AppendArgs {
+  const void* k_new; const void* v_new; const rkv_cache* full;
+  const int32_t* evict_order; int32_t* evict_count; const int32_t* k_small; int max_evict;   // all null / 0: the cache grows
+};
 
 bool cluster_eligible(const rkv_ctx* ctx, int n_max) { return ctx->small_cluster != 0 && n_max <= kClusterMaxLen; }
 
@@ -199,6 +203,10 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
     p.small_len = cache->len;
     p.len_tickets = ctx->len_tickets;
     p.has_full = app->full != nullptr;
+    p.evict_order = app->evict_order;
+    p.evict_count = app->evict_count;
+    p.k_small = app->k_small;
+    p.max_evict = app->max_evict;
     if (app->full != nullptr) {
       p.full_k = app->full->k;
       p.full_v = app->full->v;
@@ -269,6 +277,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->partials = reinterpret_cast<float*>(ctx->workspace + w.partials);
   ctx->tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.tickets);
   ctx->len_tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.len_tickets);
+  ctx->win_keys = reinterpret_cast<uint32_t*>(ctx->workspace + w.win_keys);
   ctx->logits = reinterpret_cast<float*>(ctx->workspace + w.logits);
   ctx->status = reinterpret_cast<int32_t*>(ctx->workspace + w.status);
   ctx->logit_stride = w.logit_stride;
@@ -314,6 +323,8 @@ static rkv_status full_step_impl(rkv_ctx* ctx, const void* q, const rkv_cache* f
   sp.active = active;
   sp.scores = scores;
   sp.topk_idx = topk_idx;
+  sp.win_keys = ctx->win_keys;
+  sp.win_stride = ctx->cfg.max_small;
   sp.status = ctx->status;
   sp.logit_stride = ctx->logit_stride;
   sp.score_stride = score_stride;
@@ -387,12 +398,50 @@ rkv_status rkv_append_small_step(rkv_ctx* ctx, const void* q, const void* k_new,
   if (n_max < 1 || n_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cluster_eligible(ctx, n_max)) {   // one launch: the attention kernel appends
-    const AppendArgs app = {k_new, v_new, full};
+    const AppendArgs app = {k_new, v_new, full, nullptr, nullptr, nullptr, 0};
     return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, st, nullptr, nullptr, &app);
   }
   rkv_status s = rkv_append(ctx, k_new, v_new, full, small_cache, stream);
   if (s != RKV_OK) return s;
   return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, st, nullptr, nullptr);
+}
+
+// Largest small cache whose eviction order one block can sort in shared memory.
+constexpr int kEvictMaxK = 4096;
+
+rkv_status rkv_gather_small_evict(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t* k_small, int32_t k_max,
+                                  const rkv_cache* full, const rkv_cache* small_cache, const int32_t* active,
+                                  int32_t* evict_order, int32_t* evict_count, int32_t max_evict, void* stream) {
+  if (!evict_order || !evict_count || max_evict < 1 || max_evict > kEvictMaxK) return RKV_ERR_INVALID_ARG;
+  if (k_max > kEvictMaxK) return RKV_ERR_UNSUPPORTED;
+  rkv_status s = rkv_gather_small(ctx, topk_idx, k_small, k_max, full, small_cache, active, stream);
+  if (s != RKV_OK) return s;
+  cudaError_t e;
+  {
+    LaunchScope scope(ctx, static_cast<cudaStream_t>(stream), RKV_KERNEL_GATHER);
+    e = rkv::launch_evict_order(ctx->win_keys, ctx->cfg.max_small, k_small, k_max, full->len, active, evict_order,
+                                evict_count, max_evict, ctx->cfg.n_seq, ctx->cfg.n_kv_heads,
+                                static_cast<cudaStream_t>(stream));
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "eviction-order launch");
+  ctx->launches += 1;
+  return RKV_OK;
+}
+
+rkv_status rkv_append_small_step_evict(rkv_ctx* ctx, const void* q, const void* k_new, const void* v_new,
+                                       const rkv_cache* full, const rkv_cache* small_cache, const int32_t* k_small,
+                                       const int32_t* active, void* out, const int32_t* evict_order,
+                                       int32_t* evict_count, int32_t max_evict, int32_t max_len_hint, void* stream) {
+  if (!ctx || !q || !k_new || !v_new || !cache_ok(small_cache) || !out || !k_small || !evict_order || !evict_count)
+    return RKV_ERR_INVALID_ARG;
+  if (full != nullptr && !cache_ok(full)) return RKV_ERR_INVALID_ARG;
+  if (max_evict < 1 || max_evict > kEvictMaxK) return RKV_ERR_INVALID_ARG;
+  int n_max = max_len_hint == 0 ? ctx->cfg.max_small : max_len_hint;
+  if (n_max < 1 || n_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+  if (!cluster_eligible(ctx, n_max)) return RKV_ERR_UNSUPPORTED;   // the evicting append lives in the clustered kernel
+  const AppendArgs app = {k_new, v_new, full, evict_order, evict_count, k_small, max_evict};
+  return run_attention(ctx, q, small_cache, active, out, n_max, n_max, false, static_cast<cudaStream_t>(stream), nullptr,
+                       nullptr, &app);
 }
 
 rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const rkv_cache* full,

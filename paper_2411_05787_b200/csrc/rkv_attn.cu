@@ -192,6 +192,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   uint2 kn = make_uint2(0u, 0u), vn = make_uint2(0u, 0u);
   int pos_new = -1;            // where the new row lands in the attended cache (-1: no room, or no append)
   int new_len_s = -1, new_len_f = -1;
+  bool bump_evict = false;
   if (kAppend) {
     int len_f = 0, cap_f = 0;
     int64_t roff_f = 0;
@@ -205,11 +206,24 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       kn = __ldcg(static_cast<const uint2*>(p.k_new) + nrow + lane);
       vn = __ldcg(static_cast<const uint2*>(p.v_new) + nrow + lane);
     }
-    const bool ok_s = n >= 0 && n < cap;
+    // Where the new row goes in the attended cache: behind the last row (the cache grows), or - fixed-size small
+    // cache that has reached its size - into the slot of the lowest-scoring survivor of the last refresh.
+    int slot = n;
+    bool evicting = false, ok_s = n >= 0 && n < cap;
+    if (p.evict_order != nullptr) {
+      const int kk = __ldcg(p.k_small + b);
+      if (kk > 0 && n >= kk) {
+        evicting = true;
+        const int t = __ldcg(p.evict_count + b);
+        slot = (t >= 0 && t < p.max_evict)
+                   ? __ldcg(p.evict_order + ((int64_t)b * p.n_kv_heads + g) * p.max_evict + t) : -1;
+        ok_s = slot >= 0 && slot < n && slot < cap;     // out of eviction slots: flagged like a full cache
+      }
+    }
     const bool ok_f = p.has_full && len_f >= 0 && len_f < cap_f;
     if (split == 0 && warp == 0) {   // one warp per (sequence, KV head) writes the rows to global memory
       if (ok_s) {
-        const int64_t row = (roff + (int64_t)g * cap + n) * 32;
+        const int64_t row = (roff + (int64_t)g * cap + slot) * 32;
         static_cast<uint2*>(p.small_k)[row + lane] = kn;
         static_cast<uint2*>(p.small_v)[row + lane] = vn;
       }
@@ -220,11 +234,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       }
       if (lane == 0 && (!ok_s || (p.has_full && !ok_f))) atomicOr(p.status, RKV_DEV_APPEND_OVERFLOW);
     }
-    new_len_s = ok_s ? n + 1 : -1;
+    new_len_s = (ok_s && !evicting) ? n + 1 : -1;
     new_len_f = ok_f ? len_f + 1 : -1;
+    bump_evict = evicting && ok_s;
     if (ok_s) {
-      pos_new = n;
-      n = n + 1;
+      pos_new = slot;
+      if (!evicting) n = n + 1;
     }
   }
   // Fused append: the lengths are bumped by the last (sequence, KV head) cluster to get here.  Every cluster
@@ -235,6 +250,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       if (old == p.n_kv_heads - 1) {
         if (new_len_s >= 0) p.small_len[b] = new_len_s;
         if (new_len_f >= 0) p.full_len[b] = new_len_f;
+        if (bump_evict) p.evict_count[b] += 1;   // the same decision in every cluster of the sequence
         p.len_tickets[b] = 0;   // ready for the next call on this stream
       }
     }

@@ -56,6 +56,11 @@ struct AttnParams {
   const int64_t* full_row_offset; const int32_t* full_cap; int32_t* full_len;
   int32_t* len_tickets;       // [B] arrival counters of the (sequence, KV head) clusters
   int32_t has_full;
+  // fixed-size small cache: the new row replaces the lowest-scoring survivor of the last refresh
+  const int32_t* evict_order; // [B][Hkv][max_evict] slots in eviction order, or null (the cache grows)
+  int32_t* evict_count;       // [B] evictions since the refresh
+  const int32_t* k_small;     // [B] size of the small cache
+  int32_t max_evict;
 };
 
 struct SelectParams {
@@ -70,6 +75,8 @@ struct SelectParams {
   const int32_t* active;
   float* scores;              // [B][Hkv][score_stride] or null
   int32_t* topk_idx;          // [B][Hkv][k_max]
+  uint32_t* win_keys;         // [B*Hkv][win_stride]: key of every winner, in output order (for the eviction order)
+  int32_t win_stride;
   int32_t* status;
   int64_t logit_stride, score_stride;
   int32_t n_q_heads, n_kv_heads, group, agg;
@@ -95,6 +102,9 @@ cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k
                                     int n_seq, int grid_x, cudaStream_t st);
 cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                             int n_seq, int cluster, cudaStream_t st);
+cudaError_t launch_evict_order(const uint32_t* win_keys, int win_stride, const int32_t* k_small, int k_max,
+                               const int32_t* full_len, const int32_t* active, int32_t* evict_order,
+                               int32_t* evict_count, int max_evict, int n_seq, int n_kv_heads, cudaStream_t st);
 cudaError_t launch_select(const SelectParams& p, int n_seq, int sm_count, cudaStream_t st);
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
@@ -161,6 +171,7 @@ struct rkv_ctx {
   float* partials;
   int32_t* tickets;
   int32_t* len_tickets;
+  uint32_t* win_keys;
   float* logits;
   int32_t* status;
   int64_t launches;

@@ -156,7 +156,61 @@ __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __res
   }
 }
 
+// Eviction order of a freshly rebuilt small cache (Sec. 2.2 "Decoding with partial cache": to keep C_p at a fixed
+// size, the entry with the lowest attention score of the last full step is dropped for each new token).  One block
+// per (sequence, KV head): bitonic sort of (key, slot) pairs, largest key = lowest score first, the higher slot
+// (= later position) first among equal keys; the first max_evict slots are written out.
+constexpr int kEvictMaxK = 4096;
+__global__ void __launch_bounds__(1024) evict_order_kernel(const uint32_t* __restrict__ win_keys, int win_stride,
+                                                           const int32_t* __restrict__ k_small, int k_max,
+                                                           const int32_t* __restrict__ full_len,
+                                                           const int32_t* __restrict__ active, int32_t* evict_order,
+                                                           int32_t* evict_count, int max_evict, int n_kv_heads) {
+  __shared__ unsigned long long sk[kEvictMaxK];
+  const int b = blockIdx.y, g = blockIdx.x, tid = threadIdx.x;
+  pdl_launch();
+  pdl_wait();
+  if (active != nullptr && active[b] == 0) return;
+  int m = k_small[b];
+  const int n = full_len[b];
+  if (m > k_max) m = k_max;
+  if (m > n) m = n;
+  if (m < 0) m = 0;
+  int np2 = 1;
+  while (np2 < m) np2 <<= 1;
+  const uint32_t* wk = win_keys + (int64_t)(b * n_kv_heads + g) * win_stride;
+  for (int i = tid; i < np2; i += blockDim.x)
+    sk[i] = i < m ? (((unsigned long long)wk[i] << 32) | (unsigned)i) : 0ull;   // padding sorts last
+  __syncthreads();
+  for (int k2 = 2; k2 <= np2; k2 <<= 1) {
+    for (int j = k2 >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < np2; i += blockDim.x) {
+        const int ixj = i ^ j;
+        if (ixj > i) {
+          const unsigned long long a = sk[i], c = sk[ixj];
+          const bool desc = (i & k2) == 0;          // descending overall
+          if (desc ? (a < c) : (a > c)) {
+            sk[i] = c;
+            sk[ixj] = a;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  int32_t* eo = evict_order + (int64_t)(b * n_kv_heads + g) * max_evict;
+  for (int i = tid; i < max_evict; i += blockDim.x) eo[i] = i < m ? (int32_t)(sk[i] & 0xffffffffull) : -1;
+  if (g == 0 && tid == 0) evict_count[b] = 0;
+}
+
 }  // namespace
+
+cudaError_t launch_evict_order(const uint32_t* win_keys, int win_stride, const int32_t* k_small, int k_max,
+                               const int32_t* full_len, const int32_t* active, int32_t* evict_order,
+                               int32_t* evict_count, int max_evict, int n_seq, int n_kv_heads, cudaStream_t st) {
+  return launch_ex(evict_order_kernel, dim3(n_kv_heads, n_seq), dim3(1024), 0, st, 1, win_keys, win_stride, k_small,
+                   k_max, full_len, active, evict_order, evict_count, max_evict, n_kv_heads);
+}
 
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,

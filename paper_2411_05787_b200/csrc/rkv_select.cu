@@ -415,7 +415,10 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
     fold_slice();
     write_scores();
     if (all_selected)
-      for (int i = tid; i < cnt; i += NT) idx_out[lo + i] = lo + i;
+      for (int i = tid; i < cnt; i += NT) {
+        idx_out[lo + i] = lo + i;
+        if (p.win_keys != nullptr && need_keys) p.win_keys[(int64_t)bg * p.win_stride + lo + i] = keys[i];
+      }
     return;
   }
 
@@ -580,7 +583,10 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
         ++eq_seen;
       }
       if (win) {
-        if (offs < (uint32_t)kk) idx_out[offs] = lo + i_base + 4 * j + e;
+        if (offs < (uint32_t)kk) {
+          idx_out[offs] = lo + i_base + 4 * j + e;
+          if (p.win_keys != nullptr) p.win_keys[(int64_t)bg * p.win_stride + offs] = kv[e];
+        }
         ++offs;
       }
     }

@@ -21,7 +21,8 @@ DEV_APPEND_OVERFLOW, DEV_LEN_CLAMPED, DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT 
 EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", "rkv_gather_small",
            "rkv_small_step", "rkv_append", "rkv_should_refresh", "rkv_get_device_status",
            "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
-           "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step", "rkv_score_step"]
+           "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step", "rkv_score_step",
+           "rkv_gather_small_evict", "rkv_append_small_step_evict"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER = 1, 2, 3
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
@@ -50,6 +51,10 @@ def _load() -> ctypes.CDLL:
     lib.rkv_workspace_bytes.argtypes = [cfgp]
     lib.rkv_workspace_bytes.restype = ctypes.c_size_t
     lib.rkv_full_step.argtypes = [vp, vp, cachep, vp, i32, vp, vp, vp, i64, vp, vp, i32, vp]
+    lib.rkv_gather_small_evict.argtypes = [vp, vp, vp, i32, cachep, cachep, vp, vp, vp, i32, vp]
+    lib.rkv_gather_small_evict.restype = i32
+    lib.rkv_append_small_step_evict.argtypes = [vp, vp, vp, vp, cachep, cachep, vp, vp, vp, vp, vp, i32, i32, vp]
+    lib.rkv_append_small_step_evict.restype = i32
     lib.rkv_score_step.argtypes = [vp, vp, cachep, vp, i32, vp, vp, i64, vp, vp, i32, vp]
     lib.rkv_score_step.restype = i32
     lib.rkv_gather_small.argtypes = [vp, vp, vp, i32, cachep, cachep, vp, vp]
@@ -192,6 +197,20 @@ class Context:
         self._check(lib.rkv_append_small_step(self._h, _ptr(q), _ptr(k_new), _ptr(v_new),
                                               ctypes.byref(full) if full is not None else None, ctypes.byref(small),
                                               _ptr(active), _ptr(out), max_len_hint, _stream(stream)))
+
+    def gather_small_evict(self, topk_idx, k_small, k_max, full: RkvCache, small: RkvCache, evict_order, evict_count,
+                           active=None, stream=None):
+        self._check(lib.rkv_gather_small_evict(self._h, _ptr(topk_idx), _ptr(k_small), k_max, ctypes.byref(full),
+                                               ctypes.byref(small), _ptr(active), _ptr(evict_order), _ptr(evict_count),
+                                               evict_order.shape[-1], _stream(stream)))
+
+    def append_small_step_evict(self, q, k_new, v_new, full: RkvCache | None, small: RkvCache, k_small, out,
+                                evict_order, evict_count, active=None, max_len_hint=0, stream=None):
+        self._check(lib.rkv_append_small_step_evict(self._h, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                                    ctypes.byref(full) if full is not None else None,
+                                                    ctypes.byref(small), _ptr(k_small), _ptr(active), _ptr(out),
+                                                    _ptr(evict_order), _ptr(evict_count), evict_order.shape[-1],
+                                                    max_len_hint, _stream(stream)))
 
     def should_refresh(self, q_now, q_last_full, threshold, flag, sim=None, keep=None, stream=None):
         self._check(lib.rkv_should_refresh(self._h, _ptr(q_now), _ptr(q_last_full), float(threshold), _ptr(flag),

@@ -37,6 +37,25 @@ class LayerState:
             stride = int(full.cap.max().item())
             self.scores = torch.zeros((self.n_seq, n_kv_heads, stride), dtype=torch.float32, device=dev)
 
+    def enable_eviction(self, max_evict: int):
+        """Fixed-size small cache: allocate the eviction order and counter that the *_evict calls keep."""
+        dev = self.out.device
+        self.evict_order = torch.full((self.n_seq, self.n_kv, max_evict), -1, dtype=torch.int32, device=dev)
+        self.evict_count = torch.zeros((self.n_seq,), dtype=torch.int32, device=dev)
+
+    def refresh_evict(self, q, active=None, max_len_hint=0):
+        """Full step, rebuild of the small cache and its eviction order."""
+        self.ctx.full_step(q, self.full_c, self.k_small, self.k_max, self.out, self.topk_idx, active=active,
+                           scores=self.scores, q_last_full=self.q_last_full, max_len_hint=max_len_hint)
+        self.ctx.gather_small_evict(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c,
+                                    self.evict_order, self.evict_count, active=active)
+        return self.out
+
+    def append_partial_evict(self, q, k_new, v_new, active=None, max_len_hint=0):
+        self.ctx.append_small_step_evict(q, k_new, v_new, self.full_c, self.small_c, self.k_small, self.out,
+                                         self.evict_order, self.evict_count, active=active, max_len_hint=max_len_hint)
+        return self.out
+
     def refresh(self, q, active=None, max_len_hint=0):
         """Full step followed by the rebuild of the small cache."""
         self.ctx.full_step(q, self.full_c, self.k_small, self.k_max, self.out, self.topk_idx, active=active,

@@ -423,3 +423,47 @@ def test_score_only_step_pins():
     keep = idx[0]
     want = (p[keep] / p[keep].sum()) @ v[0, keep]
     assert np.allclose(out[0], want, atol=1e-12)
+
+
+def test_fixed_size_small_cache_evicts_the_lowest_score_first():
+    """Sec. 2.2 "Decoding with partial cache": |C_p| stays K; each new token replaces the entry with the lowest
+    score of the last full step.  Hand-checkable case: one head, keys aligned with the query by known amounts."""
+    d = 128
+    q = np.zeros((1, d)); q[0, 0] = math.sqrt(d)                 # logit of position j = k[j, 0]
+    levels = [0.0, 3.0, 1.0, 5.0, 2.0, 4.0]                      # scores order: pos 3 > 5 > 1 > 4 > 2 > 0
+    k = np.zeros((1, 8, d)); k[0, :6, 0] = levels
+    v = np.zeros((1, 8, d)); v[0, :6, 1] = np.arange(6)
+    st = O.SequenceState(O.f64_to_bf16_bits(k), O.f64_to_bf16_bits(v), 6, 3, evict=True)
+    st.full(O.f64_to_bf16_bits(q))
+    assert st.small_pos[0].tolist() == [3, 5, 1] and st.len_small == 3
+    new_k, new_v = O.f64_to_bf16_bits(np.ones((1, d))), O.f64_to_bf16_bits(np.full((1, d), 9.0))
+    st.append(new_k, new_v)                                       # victim: position 1 (lowest of the three)
+    assert st.len_small == 3 and sorted(st.small_pos[0].tolist()) == [3, 5, 6]
+    st.append(new_k, new_v)                                       # next victim: position 5, never the new token
+    assert st.len_small == 3 and sorted(st.small_pos[0].tolist()) == [3, 6, 7] and st.len_full == 8
+    assert np.array_equal(st.k_small[0][st.small_pos[0].tolist().index(6)], new_k[0])
+    # without eviction the same two appends grow the cache
+    st2 = O.SequenceState(O.f64_to_bf16_bits(k), O.f64_to_bf16_bits(v), 6, 3)
+    st2.full(O.f64_to_bf16_bits(q)); st2.append(new_k, new_v); st2.append(new_k, new_v)
+    assert st2.len_small == 5
+    # equal scores: the later position is dropped first
+    k3 = np.zeros((1, 6, d)); k3[0, :4, 0] = [2.0, 2.0, 2.0, 0.0]
+    st3 = O.SequenceState(O.f64_to_bf16_bits(k3), O.f64_to_bf16_bits(np.zeros((1, 6, d))), 4, 3, evict=True)
+    st3.full(O.f64_to_bf16_bits(q)); st3.append(new_k, new_v)
+    assert sorted(st3.small_pos[0].tolist()) == [0, 1, 4]
+
+
+def test_fixed_size_cache_matches_the_cost_model_exactly(golden_dir):
+    """With eviction a partial step touches exactly K positions: T steps at stride S cost
+    (T/S) full steps over the context plus K per partial step - the T*L/S + T*K form of App. A.2 without the
+    growth term of the growing cache."""
+    T, L, K, S = 12, 40, 6, 4
+    q, k, v = _rand_case(41, n_q=2, n_kv=1, n=L + T + 1, d=128)
+    kb, vb = O.f64_to_bf16_bits(k), O.f64_to_bf16_bits(v)
+    st = O.SequenceState(kb.copy(), vb.copy(), L, K, evict=True)
+    qs = [O.f64_to_bf16_bits(q + 0.01 * t) for t in range(T + 1)]
+    O.run_fixed_stride(st, qs, [kb[:, L + t] for t in range(T + 1)], [vb[:, L + t] for t in range(T + 1)], S)
+    n_full, n_small = T // S, T - T // S
+    assert st.n_full_steps == n_full + 1 and st.n_small_steps == n_small and st.len_small == K
+    full_part = L + sum(L + t for t in range(1, T + 1) if t % S == 0)
+    assert st.positions_touched == full_part + n_small * K

@@ -406,7 +406,7 @@ def test_host_side_argument_errors(mods):
 
 
 # ----------------------------------------------------------------------------- the five workload configs
-def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False):
+def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False, evict=0):
     """Run workload `w` for one layer on the GPU and step the oracle beside it on the same bytes."""
     rkv, runner, synth = mods
     dev = torch.device("cuda")
@@ -418,12 +418,17 @@ def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False):
     max_len = max(w.lens) + w.steps + 1
     ctx = rkv.Context(w.batch, w.n_q_heads, w.n_kv_heads, max_len, max(w.k_small) + w.steps + 1)
     st = runner.LayerState(ctx, cache, list(w.k_small), w.steps + 1, w.n_q_heads, w.n_kv_heads, want_scores=False)
+    if evict:       # fixed-size small cache: new tokens replace the lowest-scoring survivors
+        st.enable_eviction(evict)
+        st.refresh, st.append_partial = st.refresh_evict, st.append_partial_evict
+        fused = True
     seqs = list(range(w.batch)) if seqs is None else seqs
     # oracle state per checked sequence, on copies of the same bytes
     states = {}
     for b in seqs:
         states[b] = O.SequenceState(host_heads(cache, b, w.n_kv_heads, "k").copy(),
-                                    host_heads(cache, b, w.n_kv_heads, "v").copy(), w.lens[b], w.k_small[b])
+                                    host_heads(cache, b, w.n_kv_heads, "v").copy(), w.lens[b], w.k_small[b],
+                                    evict=bool(evict))
     st.refresh(qs[0])
     for b in seqs:
         o_out, o_score, o_idx = states[b].full(bits(qs[0, b]))
@@ -502,8 +507,23 @@ def follow_gpu_selection(st, state, b, o_score, w):
         sel.append(got.astype(np.int64))
     state.k_small = O.gather_rows(state.k_full, sel)
     state.v_small = O.gather_rows(state.v_full, sel)
-    state.small_pos = sel
+    state.small_pos = [x.copy() for x in sel]
     state.len_small = take
+    if state.evict:
+        # the eviction order the GPU derived: scores must not decrease along it (within the selection band), nothing
+        # left behind may score clearly lower than the last listed victim; the oracle then follows the same order
+        order = st.evict_order[b].cpu().numpy()
+        assert int(st.evict_count[b]) == 0
+        state.evict_queue = []
+        for g in range(w.n_kv_heads):
+            e = order[g][order[g] >= 0]
+            assert len(e) == min(order.shape[1], take) and len(set(e.tolist())) == len(e) and e.max() < take
+            sc = o_score[g][sel[g][e]]
+            assert (sc[:-1] <= sc[1:] * (1 + 1e-5)).all(), "victims must come lowest score first"
+            rest = np.ones(take, dtype=bool); rest[e] = False
+            if rest.any():
+                assert o_score[g][sel[g][rest]].min() >= sc[-1] * (1 - 1e-5)
+            state.evict_queue.append(e.tolist())
     # gathered rows on the GPU are bit-exact copies
     for which, small in (("k", state.k_small), ("v", state.v_small)):
         gpu_small = host_heads(st.small, b, w.n_kv_heads, which)
@@ -517,6 +537,53 @@ def test_config1_every_step_every_head(mods, fused):
     w = synth.config1()
     n_full = run_trajectory(mods, w, 0, fused=fused)
     assert n_full[0] == 4      # full steps at t = 4, 8, 12, 16
+
+
+def test_config1_fixed_size_small_cache_with_eviction(mods):
+    """Config 1 with the paper's fixed-size partial cache: every partial step attends over exactly K rows."""
+    rkv, runner, synth = mods
+    n_full = run_trajectory(mods, synth.config1(), 0, evict=8)
+    assert n_full[0] == 4
+
+
+def test_config3_shape_dynamic_with_eviction(mods):
+    rkv, runner, synth = mods
+    w = synth.scaled(synth.config3(n_layers=1, ctx=8192), steps=40)
+    n_full = run_trajectory(mods, w, 0, evict=64)
+    assert n_full[0] >= 1
+
+
+def test_eviction_runs_out_of_slots_and_short_caches_grow(mods):
+    rkv, runner, synth = mods
+    lens, k_small = [300, 20], [16, 32]            # sequence 1 is shorter than its K: its small cache grows instead
+    ctx, st, cache, q = make_layer(mods, lens, k_small, 8, 2, extra=8, seed=31)
+    st.enable_eviction(2)
+    st.refresh_evict(q)
+    assert st.small.len.tolist() == [16, 20] and st.evict_count.tolist() == [0, 0]
+    assert (st.evict_order[0] >= 0).all() and (st.evict_order[1] >= 0).all()
+    g = torch.Generator(device="cuda"); g.manual_seed(32)
+    for step in range(3):
+        kn = torch.randn((2, 2, 128), generator=g, device="cuda").to(torch.bfloat16)
+        vn = torch.randn((2, 2, 128), generator=g, device="cuda").to(torch.bfloat16)
+        before = st.small.k.clone()
+        victims = st.evict_order[0, :, min(step, 1)].tolist()
+        st.append_partial_evict(q, kn, vn)
+        bits_now = ctx.device_status()
+        assert st.small.len.tolist() == [16, 21 + step] and cache.len.tolist() == [301 + step, 21 + step]
+        sk = host_heads(st.small, 0, 2, "k")
+        if step < 2:
+            assert bits_now == 0 and st.evict_count.tolist()[0] == step + 1
+            for h in range(2):
+                assert np.array_equal(sk[h, victims[h]], bits(kn[0, h]))
+        else:                                      # third new token, two eviction slots: flagged, small cache of seq 0 untouched
+            assert bits_now & rkv.DEV_APPEND_OVERFLOW
+            cap0 = int(st.small.cap[0])
+            assert torch.equal(st.small.k[: 2 * cap0], before[: 2 * cap0]) and st.evict_count.tolist()[0] == 2
+        # attention of sequence 0 runs over exactly the 16 rows now in the cache
+        k = O.bf16_bits_to_f64(host_heads(st.small, 0, 2, "k")[:, :16])
+        v = O.bf16_bits_to_f64(host_heads(st.small, 0, 2, "v")[:, :16])
+        want, _, _ = O.decode_attention(O.bf16_bits_to_f64(bits(q[0])), k, v)
+        check_out(st.out[0], want, f"evicting step {step}")
 
 
 def test_config1_planted_positions_are_selected(mods):
