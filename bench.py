@@ -213,6 +213,22 @@ def workload_config(w):
 
 
 # ----------------------------------------------------------------------------------------------- our arm
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Replicas only: the job's time for a timed region is the slowest rank's (MAX all-reduce of the device time)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_us_per_token(ms: float, steps: int, world: int) -> float:
+    """N replicas decode N * steps tokens in the (max-over-ranks) time: whole-job microseconds per token."""
+    return ms * 1000.0 / (steps * world)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -360,12 +376,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            tt = torch.tensor([ms], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms = float(tt.item())
-        return ms, cnt
+        return max_over_ranks(e0.elapsed_time(e1), world, dev), cnt
 
     # ---- main measurement: inputs resident in HBM.  The token counter runs on through all phases, so a
     # refresh (or a check) comes every S tokens and the small caches never outgrow their capacity.
@@ -377,7 +388,7 @@ def run_ours(args):
     flag_total.zero_()
     ms, cnt = timed(args.steps)
     clocks = sampler.stop() if rank == 0 else {}
-    us_per_token = ms * 1000.0 / (args.steps * world)
+    us_per_token = whole_job_us_per_token(ms, args.steps, world)
     launches = sum(cnt[k] * launches_per[k] for k in kinds)
     refreshed = int(flag_total.sum().item()) if dynamic else cnt["full"] * NL * B
     checks = cnt.get("check", 0)
@@ -385,7 +396,7 @@ def run_ours(args):
     # ---- end to end: inputs from pinned host memory, outputs back to the host, every token
     run_tokens(min(args.warmup, 10), e2e=True)
     ms_e2e, _ = timed(args.steps, e2e=True)
-    e2e_us = ms_e2e * 1000.0 / (args.steps * world)
+    e2e_us = whole_job_us_per_token(ms_e2e, args.steps, world)
 
     # ---- always-full attention (the vanilla comparator) on the same caches, then partial steps only
     run_tokens(3, always_full=True)
