@@ -80,8 +80,9 @@ typedef struct {
   void* k;                   /* bf16 [n_rows][128]                                     */
   void* v;                   /* bf16 [n_rows][128]                                     */
   int64_t n_rows;            /* host value: rows in each buffer (< 2^31)               */
-  const int64_t* row_offset; /* [B] first row of sequence b                            */
-  const int32_t* cap;        /* [B] capacity of sequence b in positions                */
+  const int64_t* row_offset; /* [B] first row of sequence b      } constant while calls  */
+  const int32_t* cap;        /* [B] capacity of sequence b       } are in flight: kernels */
+                             /*     in positions                 } may read them early    */
   int32_t* len;              /* [B] current length; append / gather_small update it    */
 } rkv_cache;
 

@@ -9,8 +9,8 @@
 // the same pass that streams K, so the cache is read from HBM exactly once.
 //
 // Shape of the kernel: one CTA per (sequence, KV head, chunk of positions).
-// A copy warp streams 64-position tiles of K and V into a 3-stage shared-memory
-// ring with 2-D tensor-map TMA loads (128-byte swizzle, completion on
+// A copy warp streams 64-position tiles of K and V into a shared-memory ring (3 stages,
+// 6 in the clustered partial step) with 2-D tensor-map TMA loads (128-byte swizzle, completion on
 // mbarriers).  Four MMA warps each own 16 positions of a tile: S^T = K Q^T and
 // O^T += V^T P^T with m16n8k16 bf16 tensor-core MMAs (fp32 accumulate), where
 // the N=8 dimension holds all query heads of the group, so K/V are read once
@@ -115,7 +115,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+template <int kThreadsN>
+__device__ __forceinline__ void consumer_bar_n() {   // barrier among the MMA warps only (the copy warp is elsewhere)
+  asm volatile("bar.sync 1, %0;" ::"n"(kThreadsN) : "memory");
+}
 __device__ __forceinline__ uint32_t map_rank(uint32_t local_addr, int rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
@@ -132,14 +135,31 @@ __device__ __forceinline__ void cluster_sync_alive() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// Stage ring: the streaming modes run two CTAs per SM with three 32 KiB stages each; the clustered partial
+// step has few CTAs and short chunks, so it takes the whole SM and keeps six tiles in flight at once.
 template <int kMode>
-__global__ void __launch_bounds__(kAttnThreads, 2)
+struct Ring {
+  static constexpr bool kWide = (kMode == kModeCluster || kMode == kModeClusterAppend);
+  static constexpr int kStg = kWide ? 6 : kStages;
+  static constexpr int kMinBlocks = kWide ? 1 : 2;
+  // The clustered partial step is bound by the latency of one warp's MMA / softmax chain per tile, not by
+  // bandwidth: two groups of four MMA warps take alternate tiles.
+  static constexpr int kMmaWarps = kWide ? 8 : 4;
+  static constexpr int kThreads = 32 * (kMmaWarps + 1);
+};
+
+template <int kMode>
+__global__ void __launch_bounds__(Ring<kMode>::kThreads, Ring<kMode>::kMinBlocks)
 attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
             const AttnParams p) {
   constexpr bool kLogits = (kMode == kModeFull || kMode == kModeScore);
   constexpr bool kScoreOnly = (kMode == kModeScore);   // logits and softmax statistics only: V is never read
   constexpr bool kCluster = (kMode == kModeCluster || kMode == kModeClusterAppend);
   constexpr bool kAppend = (kMode == kModeClusterAppend);
+  constexpr int kStg = Ring<kMode>::kStg;
+  constexpr int kMW = Ring<kMode>::kMmaWarps;      // MMA warps; warp kMW is the copy warp
+  constexpr int kGroups = kMW / 4;                  // groups of four warps that take alternate tiles
+  auto consumer_bar = [] { consumer_bar_n<32 * kMW>(); };
   extern __shared__ uint8_t smem_raw[];
   __shared__ int s_last;
 
@@ -149,16 +169,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // shared memory: [stages][K lo | K hi | V lo | V hi], the barriers, then (cluster mode) the receive buffer
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_full = smem_base + kStages * kStageBytes;
-  const uint32_t bar_empty = bar_full + 8 * kStages;
+  const uint32_t bar_full = smem_base + kStg * kStageBytes;
+  const uint32_t bar_empty = bar_full + 8 * kStg;
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kStg; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 4);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (tid == kAttnThreads - 32) {
+  if (tid == 32 * kMW) {
     prefetch_tensormap(&tm_k);
     prefetch_tensormap(&tm_v);
   }
@@ -168,15 +188,40 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + head0;
   const int qd = lane >> 2;       // row inside an 8-row group
   const int qc = (lane & 3) * 2;  // first of the two columns this lane holds
-  pdl_wait();   // nothing above reads global memory
+  // The geometry of the cache (capacity, first row) is never written by any kernel, so it may be read while the
+  // stream predecessor is still running; everything else waits for the dependency.
+  const int cap = __ldg(p.cap + b);
+  const int64_t roff = __ldg(p.row_offset + b);
+  __syncthreads();   // barrier initialisation (above) is visible to every warp
+  pdl_wait();
+
+  // Clustered partial step without a mask: every sequence is attended, and the chunk of this CTA is known from the
+  // launch geometry alone, so its first tiles are requested before the length has even been read (tiles past the
+  // length are waited for and ignored).  Saves one memory round trip on a kernel that is a chain of latencies.
+  int n_spec = 0;
+  if (kCluster && p.active == nullptr) {
+    n_spec = p.chunk / kTile < kStg ? p.chunk / kTile : kStg;
+    if (tid == 32 * kMW) {
+      uint64_t policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      const int64_t row_s = roff + (int64_t)g * cap + (int64_t)split * p.chunk;
+      for (int t = 0; t < n_spec; ++t) {
+        const uint32_t dst = smem_base + t * kStageBytes, bar = bar_full + 8 * t;
+        const int y = (int)(row_s + (int64_t)t * kTile);
+        mbar_expect_tx(bar, kStageBytes);
+        tma_load_2d(dst, &tm_k, 0, y, bar, policy);
+        tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar, policy);
+        tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
+        tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
+      }
+    }
+  }
 
   // per-sequence sizes and (MMA warps) the query fragments: independent loads, one round trip
   const int act = (p.active != nullptr) ? __ldcg(p.active + b) : 1;
-  const int cap = __ldcg(p.cap + b);
   int n = __ldcg(p.len + b);
-  const int64_t roff = __ldcg(p.row_offset + b);
   uint32_t qb[8][2];              // B fragments of Q^T: [k = channel][n = head]
-  if (warp < 4) {
+  if (warp < kMW) {
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       if (qd < G) {
@@ -201,7 +246,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       cap_f = __ldcg(p.full_cap + b);
       roff_f = __ldcg(p.full_row_offset + b);
     }
-    if (warp < 4) {
+    if (warp < kMW) {
       const int64_t nrow = ((int64_t)b * p.n_kv_heads + g) * 32;   // uint2 units: 256 bytes per row
       kn = __ldcg(static_cast<const uint2*>(p.k_new) + nrow + lane);
       vn = __ldcg(static_cast<const uint2*>(p.v_new) + nrow + lane);
@@ -268,6 +313,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     if (n < 0) n = 0;
   }
   if (n == 0) {  // nothing cached: the output is defined as zero
+    if (n_spec > 0) {   // tiles requested ahead of the length must land before the CTA may go
+      if (tid == 0)
+        for (int t = 0; t < n_spec; ++t) mbar_wait(bar_full + 8 * t, 0);
+      __syncthreads();
+    }
     if (split == 0 && tid < kHeadDim)
       for (int h = 0; h < G; ++h) out[h * kHeadDim + tid] = __float2bfloat16(0.f);
     take_len_ticket();
@@ -280,15 +330,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   const int n_splits = (n + p.chunk - 1) / p.chunk;
   const int64_t row0 = roff + (int64_t)g * cap + start;
 
-  __syncthreads();   // barrier initialisation (above) is visible to every warp
-
-  if (warp == 4) {
+  if (warp == kMW) {
     // ------------------------------------------------------------ copy warp
     if (lane == 0) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-      for (int t = 0; t < n_tiles; ++t) {
-        const int s = t % kStages, use = t / kStages;
+      for (int t = n_spec; t < n_tiles; ++t) {
+        const int s = t % kStg, use = t / kStg;
         if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1)) {
           atomicOr(p.status, kDevTimeoutBit);
           break;
@@ -324,23 +372,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   if (kLogits) lg0 = p.logits + (int64_t)(b * p.n_kv_heads + g) * p.logit_stride * p.gp + qc;
   const bool lg_on = kLogits && qc < p.gp;
 
-  const int krow = 16 * warp + (lane & 15);
-  const int vrow = 16 * warp + ((lane >> 4) << 3) + (lane & 7);
+  const int w4 = warp & 3, grp = warp >> 2;   // 16-row band inside a tile; which tiles this warp takes
+  const int krow = 16 * w4 + (lane & 15);
+  const int vrow = 16 * w4 + ((lane >> 4) << 3) + (lane & 7);
   bool ok = true;
 
-  for (int t = 0; t < n_tiles; ++t) {
-    const int s = t % kStages;
-    if (!mbar_wait(bar_full + 8 * s, (t / kStages) & 1)) {
+  const int n_wait = n_tiles > n_spec ? n_tiles : n_spec;   // tiles requested ahead of the length are always consumed
+  for (int t = grp; t < n_wait; t += kGroups) {
+    const int s = t % kStg;
+    if (!mbar_wait(bar_full + 8 * s, (t / kStg) & 1)) {
       if (lane == 0) atomicOr(p.status, kDevTimeoutBit);
       ok = false;
       break;
     }
-    const int pos_base = start + t * kTile + 16 * warp;
+    const int pos_base = start + t * kTile + 16 * w4;
     if (kAppend) {
       // The tile came from global memory, where the new row may not have landed yet: the warp that owns the
       // row writes it into the tile itself (same 128-byte swizzle as the copy engine uses).
       const int rel = pos_new - (start + t * kTile);
-      if (rel >= 0 && rel < kTile && (rel >> 4) == warp) {
+      if (rel >= 0 && rel < kTile && (rel >> 4) == w4) {
         const uint32_t at = smem_base + s * kStageBytes + (lane >> 4) * kHalfBytes + rel * 128 +
                             ((((lane & 15) >> 1) ^ (rel & 7)) << 4) + (lane & 1) * 8;
         st_shared_v2(at, kn);
@@ -348,16 +398,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         __syncwarp();
       }
     }
-    if (pos_base < end) {
+    if (t < n_tiles && pos_base < end) {
       const uint32_t kbase = smem_base + s * kStageBytes;
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
+      float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};   // two chains: half the dependent MMA latency
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const int chunk = 2 * ks + (lane >> 4);
         uint32_t a[4];
         ldsm_x4(a, kbase + (chunk >> 3) * kHalfBytes + krow * 128 + (((chunk & 7) ^ (krow & 7)) << 4));
-        mma_bf16(c, a, qb[ks][0], qb[ks][1]);
+        if (ks & 1) mma_bf16(c2, a, qb[ks][0], qb[ks][1]);
+        else mma_bf16(c, a, qb[ks][0], qb[ks][1]);
       }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) c[i] += c2[i];
       const int r0 = pos_base + qd, r1 = r0 + 8;
       float s0 = c[0] * p.scale, s1 = c[1] * p.scale, s2 = c[2] * p.scale, s3 = c[3] * p.scale;
       if (kLogits) {
@@ -433,10 +486,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
   }
 
-  // ------------------------------------------------ merge the four warps (stage memory is free now)
+  // ------------------------------------------------ merge the MMA warps (stage memory is free now)
   consumer_bar();
-  float* sm_o = reinterpret_cast<float*>(smem_gen);   // [4][8][kOPad]
-  float* sm_ml = sm_o + 4 * 8 * kOPad;                // [4][8][2]
+  float* sm_o = reinterpret_cast<float*>(smem_gen);   // [kMW][8][kOPad]
+  float* sm_ml = sm_o + kMW * 8 * kOPad;              // [kMW][8][2]
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     const int d = 16 * mt + qd;
@@ -455,16 +508,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   }
   consumer_bar();
 
-  const int d = tid;  // 0..127: one output channel per thread
+  const int d = tid;  // 0..127: one output channel per thread (further MMA warps only keep the barriers company)
+  const bool chan = d < kHeadDim;
   float accO[kMaxGroup], accM[kMaxGroup], accL[kMaxGroup];
 #pragma unroll
   for (int h = 0; h < kMaxGroup; ++h) {
+    accO[h] = 0.f;
+    accM[h] = ninf;
+    accL[h] = 0.f;
+    if (!chan || h >= G) continue;
     float M = ninf;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) M = fmaxf(M, sm_ml[(w * 8 + h) * 2]);
+    for (int w = 0; w < kMW; ++w) M = fmaxf(M, sm_ml[(w * 8 + h) * 2]);
     float L = 0.f, O = 0.f;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
+    for (int w = 0; w < kMW; ++w) {
       const float mw = sm_ml[(w * 8 + h) * 2];
       const float e = (mw == ninf) ? 0.f : ex2((mw - M) * kLog2e);
       L += sm_ml[(w * 8 + h) * 2 + 1] * e;
@@ -481,10 +539,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     // ---------------------------------------------- merge the CTAs of the cluster through shared memory
     const int C = (int)gridDim.x;                       // cluster size = CTAs per (sequence, KV head)
     const int dchunk = kHeadDim / C;                    // channels of every head that one CTA finishes
-    float* recv = reinterpret_cast<float*>(smem_gen + kStages * kStageBytes + 16 * kStages + 16);
+    float* recv = reinterpret_cast<float*>(smem_gen + kStg * kStageBytes + 16 * kStg + 16);
     float* recv_ml = recv + kMaxGroup * kHeadDim;       // [source CTA][head][2]
     const uint32_t recv_u32 = smem_u32(recv), recv_ml_u32 = smem_u32(recv_ml);
-    {
+    if (chan) {
       const int owner = d / dchunk, dd = d - owner * dchunk;
 #pragma unroll
       for (int h = 0; h < kMaxGroup; ++h)
@@ -506,7 +564,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     cluster_sync_alive();
     take_len_ticket();
     if (!ok) return;
-    for (int item = d; item < G * dchunk; item += 128) {
+    for (int item = d; chan && item < G * dchunk; item += 128) {
       const int h = item / dchunk, dd = item - h * dchunk;
       float M = ninf;
       for (int r = 0; r < C; ++r) M = fmaxf(M, recv_ml[(r * kMaxGroup + h) * 2]);
@@ -556,7 +614,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     float* sm_red = reinterpret_cast<float*>(smem_gen);                 // [4][8][128]
     float* sm_w = sm_red + 4 * kMaxGroup * kHeadDim;                    // [n_splits][16]
     float* sm_ML = sm_w + kMaxSplits * 16;                              // [16]
-    auto bar = [] { consumer_bar(); };
+    auto bar = [] { consumer_bar_n<128>(); };
     fold_weights<128>(pbase, n_splits, tid, sm_w, sm_ML, bar);
     fold_out<128, kMaxGroup>(pbase, n_splits, 0, G, tid, sm_w, sm_red, bar);
 #pragma unroll
@@ -577,9 +635,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
 
 }  // namespace
 
-size_t attention_smem_bytes() {
-  return (size_t)kStages * kStageBytes + 16 * kStages + 16 + (size_t)kRecvFloats * sizeof(float) + 1024;
+static size_t ring_smem_bytes(int stages) {
+  return (size_t)stages * kStageBytes + 16 * stages + 16 + (size_t)kRecvFloats * sizeof(float) + 1024;
 }
+size_t attention_smem_bytes() { return ring_smem_bytes(kStages); }
+static size_t cluster_smem_bytes() { return ring_smem_bytes(Ring<kModeCluster>::kStg); }
 
 cudaError_t prepare_attention() {
   const int bytes = (int)attention_smem_bytes();
@@ -589,9 +649,11 @@ cudaError_t prepare_attention() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_kernel<kModeScore>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attn_kernel<kModeCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  e = cudaFuncSetAttribute(attn_kernel<kModeCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)cluster_smem_bytes());
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_kernel<kModeClusterAppend>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  return cudaFuncSetAttribute(attn_kernel<kModeClusterAppend>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)cluster_smem_bytes());
 }
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
@@ -611,14 +673,15 @@ cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k
 cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                      int n_seq, int cluster, cudaStream_t st) {
   dim3 grid(cluster, p.n_kv_heads, n_seq);
-  return launch_ex(attn_kernel<kModeCluster>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, cluster, tm_k, tm_v, p);
+  return launch_ex(attn_kernel<kModeCluster>, grid, dim3(Ring<kModeCluster>::kThreads), cluster_smem_bytes(), st, cluster,
+                   tm_k, tm_v, p);
 }
 
 cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                             int n_seq, int cluster, cudaStream_t st) {
   dim3 grid(cluster, p.n_kv_heads, n_seq);
-  return launch_ex(attn_kernel<kModeClusterAppend>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, cluster, tm_k,
-                   tm_v, p);
+  return launch_ex(attn_kernel<kModeClusterAppend>, grid, dim3(Ring<kModeClusterAppend>::kThreads), cluster_smem_bytes(), st,
+                   cluster, tm_k, tm_v, p);
 }
 
 }  // namespace rkv
