@@ -194,6 +194,8 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.max_splits = ctx->max_splits;
   p.max_len = limit;
   p.scale = ctx->cfg.softmax_scale;
+  // without a mask: a cluster per head always has work; a streaming grid has when it serves a single sequence
+  p.spec = (active == nullptr && (cluster || (logits && ctx->cfg.n_seq == 1))) ? 1 : 0;
   if (app != nullptr) {   // only the clustered partial step takes the append with it
     if (!cluster) return RKV_ERR_INVALID_ARG;
     p.k_new = app->k_new;

@@ -195,25 +195,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   __syncthreads();   // barrier initialisation (above) is visible to every warp
   pdl_wait();
 
-  // Clustered partial step without a mask: every sequence is attended, and the chunk of this CTA is known from the
-  // launch geometry alone, so its first tiles are requested before the length has even been read (tiles past the
-  // length are waited for and ignored).  Saves one memory round trip on a kernel that is a chain of latencies.
+  // One tile = K (and V) rows [y, y + 64) into stage t % kStg, completion on that stage's barrier.
+  auto issue_tile = [&](int t, int64_t row_first, uint64_t policy) {
+    const int s = t % kStg;
+    const uint32_t dst = smem_base + s * kStageBytes, bar = bar_full + 8 * s;
+    const int y = (int)(row_first + (int64_t)t * kTile);
+    mbar_expect_tx(bar, kScoreOnly ? 2 * kHalfBytes : kStageBytes);
+    tma_load_2d(dst, &tm_k, 0, y, bar, policy);
+    tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar, policy);
+    if (!kScoreOnly) {
+      tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
+      tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
+    }
+  };
+  // When the host knows that every CTA of the grid has work (no mask; one sequence, or a cluster per head), the
+  // chunk of this CTA follows from the launch geometry alone, so its first tiles are requested before the length
+  // has even been read (tiles past the length are waited for and ignored).  Saves one memory round trip.
   int n_spec = 0;
-  if (kCluster && p.active == nullptr) {
+  if (p.spec != 0) {
     n_spec = p.chunk / kTile < kStg ? p.chunk / kTile : kStg;
     if (tid == 32 * kMW) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
       const int64_t row_s = roff + (int64_t)g * cap + (int64_t)split * p.chunk;
-      for (int t = 0; t < n_spec; ++t) {
-        const uint32_t dst = smem_base + t * kStageBytes, bar = bar_full + 8 * t;
-        const int y = (int)(row_s + (int64_t)t * kTile);
-        mbar_expect_tx(bar, kStageBytes);
-        tma_load_2d(dst, &tm_k, 0, y, bar, policy);
-        tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar, policy);
-        tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
-        tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
-      }
+      for (int t = 0; t < n_spec; ++t) issue_tile(t, row_s, policy);
     }
   }
 
@@ -324,7 +329,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     return;
   }
   const int start = split * p.chunk;
-  if (!kCluster && start >= n) return;   // in a cluster an idle CTA still owns a slice of the output
+  if (!kCluster && start >= n) {   // in a cluster an idle CTA still owns a slice of the output
+    if (n_spec > 0) {
+      if (tid == 0)
+        for (int t = 0; t < n_spec; ++t) mbar_wait(bar_full + 8 * t, 0);
+      __syncthreads();
+    }
+    return;
+  }
   const int end = (start + p.chunk < n) ? start + p.chunk : n;
   const int n_tiles = (end > start) ? (end - start + kTile - 1) / kTile : 0;
   const int n_splits = (n + p.chunk - 1) / p.chunk;
@@ -341,16 +353,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
           atomicOr(p.status, kDevTimeoutBit);
           break;
         }
-        const uint32_t dst = smem_base + s * kStageBytes;
-        const uint32_t bar = bar_full + 8 * s;
-        const int y = (int)(row0 + (int64_t)t * kTile);
-        mbar_expect_tx(bar, kScoreOnly ? 2 * kHalfBytes : kStageBytes);
-        tma_load_2d(dst, &tm_k, 0, y, bar, policy);
-        tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar, policy);
-        if (!kScoreOnly) {
-          tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
-          tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
-        }
+        issue_tile(t, row0, policy);
       }
     }
     if (kCluster) {   // stay until the peers have pushed: every warp of the cluster meets at one barrier

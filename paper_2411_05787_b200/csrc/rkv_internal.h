@@ -46,6 +46,7 @@ struct AttnParams {
   int32_t chunk;              // positions per CTA
   int32_t max_splits;
   int32_t max_len;            // clamp for len[b]
+  int32_t spec;               // 1: every CTA has work by construction, first tiles may be requested before len is read
   float scale;
   // fused append (clustered partial step only): the new token's rows and where they go
   const void* k_new;          // bf16 [B][Hkv][128]
