@@ -220,10 +220,11 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   cudaError_t e;
   {
     LaunchScope scope(ctx, st, logits ? RKV_KERNEL_ATTN_FULL : RKV_KERNEL_ATTN_SMALL);
-    e = app != nullptr ? rkv::launch_attention_cluster_append(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
-        : score_only   ? rkv::launch_attention_scores(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
-        : cluster      ? rkv::launch_attention_cluster(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
-                       : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
+    // few clusters (half the SMs or fewer): the wide form of the clustered kernel, one CTA per SM
+    const bool wide = cluster && (int64_t)gx * ctx->cfg.n_kv_heads * ctx->cfg.n_seq * 2 <= ctx->sm_count;
+    e = cluster      ? rkv::launch_attention_cluster(p, tm_k, tm_v, ctx->cfg.n_seq, gx, app != nullptr, wide, st)
+        : score_only ? rkv::launch_attention_scores(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
+                     : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
   ctx->launches += 1;

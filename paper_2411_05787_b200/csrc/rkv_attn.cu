@@ -127,6 +127,11 @@ __device__ __forceinline__ uint32_t map_rank(uint32_t local_addr, int rank) {
 __device__ __forceinline__ void st_shared_v2(uint32_t addr, uint2 v) {
   asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(v.x), "r"(v.y) : "memory");
 }
+// Store that asks L2 to keep the line (the selection kernel reads the logits right after this kernel, while
+// 134 MB of K/V stream through the same cache with evict-first priority).
+__device__ __forceinline__ void st_keep_f2(float* addr, float a, float b, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(addr), "f"(a), "f"(b), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
@@ -135,11 +140,13 @@ __device__ __forceinline__ void cluster_sync_alive() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// Stage ring: the streaming modes run two CTAs per SM with three 32 KiB stages each; the clustered partial
-// step has few CTAs and short chunks, so it takes the whole SM and keeps six tiles in flight at once.
-template <int kMode>
+// Stage ring: normally two CTAs per SM with three 32 KiB stages each.  The clustered partial step with few
+// clusters (batch 1) is a pure latency chain on half-empty SMs: its "wide" form takes the whole SM, keeps six
+// tiles in flight and splits the tiles over two groups of MMA warps.  With many clusters the narrow form wins
+// (two CTAs per SM place clusters more freely and overlap each other's latencies).
+template <int kMode, bool kWideT>
 struct Ring {
-  static constexpr bool kWide = (kMode == kModeCluster || kMode == kModeClusterAppend);
+  static constexpr bool kWide = kWideT && (kMode == kModeCluster || kMode == kModeClusterAppend);
   static constexpr int kStg = kWide ? 6 : kStages;
   static constexpr int kMinBlocks = kWide ? 1 : 2;
   // The clustered partial step is bound by the latency of one warp's MMA / softmax chain per tile, not by
@@ -148,16 +155,16 @@ struct Ring {
   static constexpr int kThreads = 32 * (kMmaWarps + 1);
 };
 
-template <int kMode>
-__global__ void __launch_bounds__(Ring<kMode>::kThreads, Ring<kMode>::kMinBlocks)
+template <int kMode, bool kWideT = false>
+__global__ void __launch_bounds__(Ring<kMode, kWideT>::kThreads, Ring<kMode, kWideT>::kMinBlocks)
 attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
             const AttnParams p) {
   constexpr bool kLogits = (kMode == kModeFull || kMode == kModeScore);
   constexpr bool kScoreOnly = (kMode == kModeScore);   // logits and softmax statistics only: V is never read
   constexpr bool kCluster = (kMode == kModeCluster || kMode == kModeClusterAppend);
   constexpr bool kAppend = (kMode == kModeClusterAppend);
-  constexpr int kStg = Ring<kMode>::kStg;
-  constexpr int kMW = Ring<kMode>::kMmaWarps;      // MMA warps; warp kMW is the copy warp
+  constexpr int kStg = Ring<kMode, kWideT>::kStg;
+  constexpr int kMW = Ring<kMode, kWideT>::kMmaWarps;      // MMA warps; warp kMW is the copy warp
   constexpr int kGroups = kMW / 4;                  // groups of four warps that take alternate tiles
   auto consumer_bar = [] { consumer_bar_n<32 * kMW>(); };
   extern __shared__ uint8_t smem_raw[];
@@ -374,6 +381,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   float* lg0 = nullptr;
   if (kLogits) lg0 = p.logits + (int64_t)(b * p.n_kv_heads + g) * p.logit_stride * p.gp + qc;
   const bool lg_on = kLogits && qc < p.gp;
+  uint64_t keep_policy = 0;
+  if (kLogits) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep_policy));
 
   const int w4 = warp & 3, grp = warp >> 2;   // 16-row band inside a tile; which tiles this warp takes
   const int krow = 16 * w4 + (lane & 15);
@@ -418,8 +427,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       float s0 = c[0] * p.scale, s1 = c[1] * p.scale, s2 = c[2] * p.scale, s3 = c[3] * p.scale;
       if (kLogits) {
         if (lg_on) {
-          if (r0 < end) *reinterpret_cast<float2*>(lg0 + (int64_t)r0 * p.gp) = make_float2(s0, s1);
-          if (r1 < end) *reinterpret_cast<float2*>(lg0 + (int64_t)r1 * p.gp) = make_float2(s2, s3);
+          if (r0 < end) st_keep_f2(lg0 + (int64_t)r0 * p.gp, s0, s1, keep_policy);
+          if (r1 < end) st_keep_f2(lg0 + (int64_t)r1 * p.gp, s2, s3, keep_policy);
         }
       }
       if (r0 >= end) s0 = s1 = ninf;
@@ -642,7 +651,7 @@ static size_t ring_smem_bytes(int stages) {
   return (size_t)stages * kStageBytes + 16 * stages + 16 + (size_t)kRecvFloats * sizeof(float) + 1024;
 }
 size_t attention_smem_bytes() { return ring_smem_bytes(kStages); }
-static size_t cluster_smem_bytes() { return ring_smem_bytes(Ring<kModeCluster>::kStg); }
+static size_t cluster_smem_bytes(bool wide) { return ring_smem_bytes(wide ? Ring<kModeCluster, true>::kStg : kStages); }
 
 cudaError_t prepare_attention() {
   const int bytes = (int)attention_smem_bytes();
@@ -652,11 +661,16 @@ cudaError_t prepare_attention() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_kernel<kModeScore>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attn_kernel<kModeCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)cluster_smem_bytes());
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_kernel<kModeClusterAppend>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)cluster_smem_bytes());
+  e = cudaFuncSetAttribute(attn_kernel<kModeCluster, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(attn_kernel<kModeClusterAppend, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(attn_kernel<kModeCluster, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)cluster_smem_bytes(true));
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(attn_kernel<kModeClusterAppend, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)cluster_smem_bytes(true));
+  return e;
 }
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
@@ -674,17 +688,17 @@ cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k
 }
 
 cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                     int n_seq, int cluster, cudaStream_t st) {
+                                     int n_seq, int cluster, bool append, bool wide, cudaStream_t st) {
   dim3 grid(cluster, p.n_kv_heads, n_seq);
-  return launch_ex(attn_kernel<kModeCluster>, grid, dim3(Ring<kModeCluster>::kThreads), cluster_smem_bytes(), st, cluster,
-                   tm_k, tm_v, p);
-}
-
-cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                            int n_seq, int cluster, cudaStream_t st) {
-  dim3 grid(cluster, p.n_kv_heads, n_seq);
-  return launch_ex(attn_kernel<kModeClusterAppend>, grid, dim3(Ring<kModeClusterAppend>::kThreads), cluster_smem_bytes(), st,
-                   cluster, tm_k, tm_v, p);
+  const size_t smem = cluster_smem_bytes(wide);
+  if (wide) {
+    const dim3 block(Ring<kModeCluster, true>::kThreads);
+    if (append) return launch_ex(attn_kernel<kModeClusterAppend, true>, grid, block, smem, st, cluster, tm_k, tm_v, p);
+    return launch_ex(attn_kernel<kModeCluster, true>, grid, block, smem, st, cluster, tm_k, tm_v, p);
+  }
+  const dim3 block(kAttnThreads);
+  if (append) return launch_ex(attn_kernel<kModeClusterAppend, false>, grid, block, smem, st, cluster, tm_k, tm_v, p);
+  return launch_ex(attn_kernel<kModeCluster, false>, grid, block, smem, st, cluster, tm_k, tm_v, p);
 }
 
 }  // namespace rkv

@@ -98,11 +98,9 @@ struct CacheDev {
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                              int n_seq, int grid_x, bool write_logits, cudaStream_t st);
 cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                     int n_seq, int cluster, cudaStream_t st);
+                                     int n_seq, int cluster, bool append, bool wide, cudaStream_t st);
 cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                     int n_seq, int grid_x, cudaStream_t st);
-cudaError_t launch_attention_cluster_append(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                            int n_seq, int cluster, cudaStream_t st);
 cudaError_t launch_evict_order(const uint32_t* win_keys, int win_stride, const int32_t* k_small, int k_max,
                                const int32_t* full_len, const int32_t* active, int32_t* evict_order,
                                int32_t* evict_count, int max_evict, int n_seq, int n_kv_heads, cudaStream_t st);
