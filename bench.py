@@ -596,7 +596,7 @@ def run_cfg5(args):
                    "layer_refreshes_in_timed_region": refreshed, "check_tokens": cnt["check"],
                    "of_possible": cnt["check"] * shape.n_layers, "device_status": status,
                    "library_launches_per_token": {k: v for k, v in launches_per.items() if "_" not in k},
-                   "harness_launches_per_token": 7 * shape.n_layers + 4,
+                   "harness_launches_per_token": 5 * shape.n_layers + 3,
                    "first_tokens": history[3: 19].tolist()},
     }
     result["roofline"]["frac"] = result["roofline"]["achieved"] / peak

@@ -23,15 +23,17 @@ extern "C" {
 /* y[i] = x[i] / sqrt(mean(x^2) + eps) * w[i];  n <= 16384, n % 4 == 0.  x, y fp32 [n]; w bf16 [n]. */
 int llh_rmsnorm(const float* x, const void* w, float eps, float* y, int32_t n, void* stream);
 
-/* y[o] = sum_i W[o][i] * x[i] (+ residual[o]).  W bf16 [n_out][n_in], n_in % 256 == 0, n_in <= 16384.
- * x is fp32 [n_in] (x_is_bf16 == 0) or bf16 [n_in] (x_is_bf16 != 0); y, residual fp32 [n_out];
- * residual may be NULL and may alias y. */
-int llh_gemv(const void* w, const void* x, int32_t x_is_bf16, const float* residual, float* y,
-             int32_t n_out, int32_t n_in, void* stream);
+/* y[o] = sum_i W[o][i] * x'[i] (+ residual[o]).  W bf16 [n_out][n_in], n_in % 256 == 0, n_in <= 16384.
+ * x is fp32 [n_in] (x_is_bf16 == 0) or bf16 [n_in] (x_is_bf16 != 0).  With norm_w != NULL (bf16 [n_in]) the input
+ * is RMS-normalised on the way in: x'[i] = x[i] / sqrt(mean(x^2) + eps) * norm_w[i]; otherwise x' = x.
+ * y, residual fp32 [n_out]; residual may be NULL and may alias y (but not x). */
+int llh_gemv(const void* w, const void* x, int32_t x_is_bf16, const void* norm_w, float eps, const float* residual,
+             float* y, int32_t n_out, int32_t n_in, void* stream);
 
-/* SwiGLU feed-forward input half: y[f] = silu(<Wg[f], x>) * <Wu[f], x>, with W = [Wg ; Wu] stacked as
- * bf16 [2 * n_ff][n_in]; silu(t) = t / (1 + exp(-t)).  x fp32 [n_in], y fp32 [n_ff]. */
-int llh_gemv_swiglu(const void* w_gate_up, const float* x, float* y, int32_t n_ff, int32_t n_in, void* stream);
+/* SwiGLU feed-forward input half: y[f] = silu(<Wg[f], x'>) * <Wu[f], x'>, with W = [Wg ; Wu] stacked as
+ * bf16 [2 * n_ff][n_in]; silu(t) = t / (1 + exp(-t)); x' as in llh_gemv.  x fp32 [n_in], y fp32 [n_ff]. */
+int llh_gemv_swiglu(const void* w_gate_up, const float* x, const void* norm_w, float eps, float* y, int32_t n_ff,
+                    int32_t n_in, void* stream);
 
 /* Rotary embedding (rotate-half pairing: channel c with c + 64, angle pos * theta^(-c/64), c < 64) of the
  * query and key heads of one token, and the split of the fused projection into bf16 tensors:

@@ -2,7 +2,9 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
+#include <utility>
 
 #include "rkv_internal.h"
 
@@ -17,7 +19,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn g_encode = nullptr;
-bool g_prepared = false;
+// kernel attributes (dynamic shared-memory sizes) are set per device, once
+constexpr int kMaxDevices = 64;
+bool g_prepared[kMaxDevices] = {};
+std::mutex g_prepare_mu;
 
 bool config_ok(const rkv_config* c, rkv_status* why) {
   if (c == nullptr) { *why = RKV_ERR_INVALID_ARG; return false; }
@@ -92,7 +97,7 @@ CacheDev dev_of(const rkv_cache* c) { return CacheDev{c->k, c->v, c->row_offset,
 
 // 2-D view [n_rows][128] bf16, box = 64 rows x 64 channels (128 bytes), 128-byte swizzle
 rkv_status tensor_map(rkv_ctx* ctx, void* base, int64_t n_rows, CUtensorMap* out) {
-  const uint64_t key = reinterpret_cast<uint64_t>(base) ^ ((uint64_t)n_rows * 0x9E3779B97F4A7C15ull);
+  const std::pair<uint64_t, int64_t> key(reinterpret_cast<uint64_t>(base), n_rows);   // the map depends on nothing else
   auto it = ctx->tmaps.find(key);
   if (it != ctx->tmaps.end()) { *out = it->second; return RKV_OK; }
   if (g_encode == nullptr) {
@@ -265,11 +270,15 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
   if (e != cudaSuccess) { delete ctx; return RKV_ERR_CUDA; }
-  if (!g_prepared) {
-    e = rkv::prepare_attention();
-    if (e == cudaSuccess) e = rkv::prepare_select();
-    if (e != cudaSuccess) { delete ctx; return RKV_ERR_CUDA; }
-    g_prepared = true;
+  if (ctx->device < 0 || ctx->device >= kMaxDevices) { delete ctx; return RKV_ERR_UNSUPPORTED; }
+  {
+    std::lock_guard<std::mutex> lock(g_prepare_mu);
+    if (!g_prepared[ctx->device]) {
+      e = rkv::prepare_attention();
+      if (e == cudaSuccess) e = rkv::prepare_select();
+      if (e != cudaSuccess) { delete ctx; return RKV_ERR_CUDA; }
+      g_prepared[ctx->device] = true;
+    }
   }
   const WsLayout w = ws_layout(cfg);
   e = cudaMalloc(reinterpret_cast<void**>(&ctx->workspace), w.total);

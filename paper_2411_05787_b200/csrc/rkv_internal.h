@@ -5,7 +5,8 @@
 #include <stdint.h>
 
 #include <string>
-#include <unordered_map>
+#include <map>
+#include <utility>
 #include <vector>
 
 #include "rkv.h"
@@ -180,7 +181,7 @@ struct rkv_ctx {
   int small_cluster;   // 1: the partial step merges its splits inside a thread-block cluster when the length allows
   int gp;              // floats per position in the logit scratch
   std::string last_error;
-  std::unordered_map<uint64_t, CUtensorMap> tmaps;
+  std::map<std::pair<uint64_t, int64_t>, CUtensorMap> tmaps;   // (base address, rows) -> tensor map
   // optional per-kernel timing (rkv_set_profiling): event pairs recorded around every launch
   bool profiling;
   struct Timed { int kind; cudaEvent_t start, stop; };

@@ -9,7 +9,7 @@
 
 namespace {
 
-constexpr int kGemvThreads = 256;
+constexpr int kGemvThreads = 512;
 constexpr int kMaxIn = 16384;
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -26,18 +26,20 @@ __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
     f[2 * i + 1] = t.y;
   }
 }
-// <row, x> for one weight row: lane l takes 16-byte chunks l, l+32, ...; x sits in shared memory as fp32
+// <row, x> for one weight row: lane l takes 16-byte chunks l, l+32, ...; x sits in shared memory as fp32.
+// Eight chunks (128 bytes) per lane are in flight at once, so a 4096-wide row costs two memory round trips.
 __device__ __forceinline__ float row_dot(const uint4* __restrict__ row, const float* xs, int n_chunks, int lane) {
+  constexpr int kFly = 8;
   float acc = 0.f;
-  for (int c0 = lane; c0 < n_chunks; c0 += 128) {   // four chunks (64 bytes) per lane in flight
-    uint4 u[4];
+  for (int c0 = lane; c0 < n_chunks; c0 += 32 * kFly) {
+    uint4 u[kFly];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < kFly; ++k) {
       const int c = c0 + 32 * k;
       u[k] = (c < n_chunks) ? __ldcs(row + c) : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < kFly; ++k) {
       const int c = c0 + 32 * k;
       if (c < n_chunks) {
         float f[8];
@@ -51,21 +53,44 @@ __device__ __forceinline__ float row_dot(const uint4* __restrict__ row, const fl
   }
   return warp_sum(acc);
 }
-__device__ __forceinline__ void stage_x(const void* x, int x_is_bf16, float* xs, int n_in) {
+// Bring x into shared memory as fp32; with a norm weight, apply RMSNorm on the way (every block recomputes the
+// mean square of the few thousand inputs, which is cheaper than a separate launch).
+__device__ __forceinline__ void stage_x(const void* x, int x_is_bf16, const __nv_bfloat16* norm_w, float eps, float* xs,
+                                        int n_in) {
+  __shared__ float red[32];
+  float ss = 0.f;
   if (x_is_bf16) {
     const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
-    for (int i = threadIdx.x; i < n_in; i += blockDim.x) xs[i] = __bfloat162float(xb[i]);
+    for (int i = threadIdx.x; i < n_in; i += blockDim.x) {
+      const float v = __bfloat162float(xb[i]);
+      xs[i] = v;
+      ss = fmaf(v, v, ss);
+    }
   } else {
     const float* xf = static_cast<const float*>(x);
-    for (int i = threadIdx.x; i < n_in; i += blockDim.x) xs[i] = xf[i];
+    for (int i = threadIdx.x; i < n_in; i += blockDim.x) {
+      const float v = xf[i];
+      xs[i] = v;
+      ss = fmaf(v, v, ss);
+    }
+  }
+  if (norm_w != nullptr) {
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) tot += red[i];
+    const float r = rsqrtf(tot / (float)n_in + eps);
+    for (int i = threadIdx.x; i < n_in; i += blockDim.x) xs[i] = xs[i] * r * __bfloat162float(norm_w[i]);
   }
   __syncthreads();
 }
 
 __global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const uint4* __restrict__ w, const void* x, int x_is_bf16,
-                                                            const float* residual, float* y, int n_out, int n_in) {
+                                                            const __nv_bfloat16* norm_w, float eps, const float* residual,
+                                                            float* y, int n_out, int n_in) {
   extern __shared__ float xs[];
-  stage_x(x, x_is_bf16, xs, n_in);
+  stage_x(x, x_is_bf16, norm_w, eps, xs, n_in);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = kGemvThreads / 32;
   const int n_chunks = n_in / 8;
   for (int o = blockIdx.x * wpb + warp; o < n_out; o += gridDim.x * wpb) {
@@ -74,10 +99,11 @@ __global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const uint4* __restr
   }
 }
 
-__global__ void __launch_bounds__(kGemvThreads) gemv_swiglu_kernel(const uint4* __restrict__ w, const float* x, float* y,
+__global__ void __launch_bounds__(kGemvThreads) gemv_swiglu_kernel(const uint4* __restrict__ w, const float* x,
+                                                                   const __nv_bfloat16* norm_w, float eps, float* y,
                                                                    int n_ff, int n_in) {
   extern __shared__ float xs[];
-  stage_x(x, 0, xs, n_in);
+  stage_x(x, 0, norm_w, eps, xs, n_in);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = kGemvThreads / 32;
   const int n_chunks = n_in / 8;
   for (int f = blockIdx.x * wpb + warp; f < n_ff; f += gridDim.x * wpb) {
@@ -166,29 +192,37 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float* logits, int n
   }
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
+// per-device state: SM count and whether the kernels' shared-memory attribute has been set there
+constexpr int kMaxDevices = 64;
+int g_sm_count[kMaxDevices] = {};
+bool g_attr_set[kMaxDevices] = {};
+int current_device() {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  return (dev >= 0 && dev < kMaxDevices) ? dev : 0;
 }
-bool g_attr_set = false;
+int sm_count() {
+  const int dev = current_device();
+  if (g_sm_count[dev] == 0) {
+    int n = 0;
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    g_sm_count[dev] = n > 0 ? n : 148;
+  }
+  return g_sm_count[dev];
+}
 int ensure_attrs() {
-  if (g_attr_set) return 0;
+  const int dev = current_device();
+  if (g_attr_set[dev]) return 0;
   cudaError_t e = cudaFuncSetAttribute(gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_swiglu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
   if (e != cudaSuccess) return (int)e;
-  g_attr_set = true;
+  g_attr_set[dev] = true;
   return 0;
 }
 int gemv_grid(int n_rows) {
   const int per_block = kGemvThreads / 32;
   int blocks = (n_rows + per_block - 1) / per_block;
-  const int cap = sm_count() * 8;
+  const int cap = sm_count() * 2;   // two blocks of 16 warps per SM: few copies of x, many rows in flight
   return blocks < cap ? (blocks < 1 ? 1 : blocks) : cap;
 }
 
@@ -202,20 +236,21 @@ int llh_rmsnorm(const float* x, const void* w, float eps, float* y, int32_t n, v
   return (int)cudaGetLastError();
 }
 
-int llh_gemv(const void* w, const void* x, int32_t x_is_bf16, const float* residual, float* y, int32_t n_out,
-             int32_t n_in, void* stream) {
+int llh_gemv(const void* w, const void* x, int32_t x_is_bf16, const void* norm_w, float eps, const float* residual,
+             float* y, int32_t n_out, int32_t n_in, void* stream) {
   if (!w || !x || !y || n_out < 1 || n_in < 256 || n_in > kMaxIn || n_in % 256) return -1;
   if (int e = ensure_attrs()) return e;
   gemv_kernel<<<gemv_grid(n_out), kGemvThreads, (size_t)n_in * 4, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const uint4*>(w), x, x_is_bf16, residual, y, n_out, n_in);
+      static_cast<const uint4*>(w), x, x_is_bf16, static_cast<const __nv_bfloat16*>(norm_w), eps, residual, y, n_out, n_in);
   return (int)cudaGetLastError();
 }
 
-int llh_gemv_swiglu(const void* w_gate_up, const float* x, float* y, int32_t n_ff, int32_t n_in, void* stream) {
+int llh_gemv_swiglu(const void* w_gate_up, const float* x, const void* norm_w, float eps, float* y, int32_t n_ff,
+                    int32_t n_in, void* stream) {
   if (!w_gate_up || !x || !y || n_ff < 1 || n_in < 256 || n_in > kMaxIn || n_in % 256) return -1;
   if (int e = ensure_attrs()) return e;
   gemv_swiglu_kernel<<<gemv_grid(n_ff), kGemvThreads, (size_t)n_in * 4, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const uint4*>(w_gate_up), x, y, n_ff, n_in);
+      static_cast<const uint4*>(w_gate_up), x, static_cast<const __nv_bfloat16*>(norm_w), eps, y, n_ff, n_in);
   return (int)cudaGetLastError();
 }
 

@@ -32,8 +32,8 @@ def _load() -> ctypes.CDLL:
     lib = ctypes.CDLL(_LIB_PATH)
     vp, i32, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float
     lib.llh_rmsnorm.argtypes = [vp, vp, f32, vp, i32, vp]
-    lib.llh_gemv.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp]
-    lib.llh_gemv_swiglu.argtypes = [vp, vp, vp, i32, i32, vp]
+    lib.llh_gemv.argtypes = [vp, vp, i32, vp, f32, vp, vp, i32, i32, vp]
+    lib.llh_gemv_swiglu.argtypes = [vp, vp, vp, f32, vp, i32, i32, vp]
     lib.llh_rope_split.argtypes = [vp, vp, f32, vp, vp, vp, i32, i32, vp]
     lib.llh_embed.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.llh_argmax.argtypes = [vp, i32, vp, vp]
@@ -62,15 +62,16 @@ def rmsnorm(x, w, eps, y):
     _ck(lib.llh_rmsnorm(_p(x), _p(w), eps, _p(y), x.numel(), _st()), "llh_rmsnorm")
 
 
-def gemv(w, x, y, residual=None):
+def gemv(w, x, y, residual=None, norm_w=None, eps=1e-5):
+    """y = W x' (+ residual); with norm_w the input is RMS-normalised inside the kernel."""
     n_out, n_in = w.shape
-    _ck(lib.llh_gemv(_p(w), _p(x), 1 if x.dtype == torch.bfloat16 else 0, _p(residual), _p(y), n_out, n_in, _st()),
-        "llh_gemv")
+    _ck(lib.llh_gemv(_p(w), _p(x), 1 if x.dtype == torch.bfloat16 else 0, _p(norm_w), eps, _p(residual), _p(y), n_out,
+                     n_in, _st()), "llh_gemv")
 
 
-def gemv_swiglu(w_gate_up, x, y):
-    _ck(lib.llh_gemv_swiglu(_p(w_gate_up), _p(x), _p(y), w_gate_up.shape[0] // 2, w_gate_up.shape[1], _st()),
-        "llh_gemv_swiglu")
+def gemv_swiglu(w_gate_up, x, y, norm_w=None, eps=1e-5):
+    _ck(lib.llh_gemv_swiglu(_p(w_gate_up), _p(x), _p(norm_w), eps, _p(y), w_gate_up.shape[0] // 2, w_gate_up.shape[1],
+                            _st()), "llh_gemv_swiglu")
 
 
 def rope_split(qkv, pos, theta, q, k, v, n_q, n_kv):
@@ -222,18 +223,15 @@ class LlamaDecoder:
             embed(self.embed_w, self.token, self.x)
         for l, wl in enumerate(self.layers_w):
             if with_harness:
-                rmsnorm(self.x, wl["norm1"], s.eps, self.h)
-                gemv(wl["wqkv"], self.h, self.qkv)
+                gemv(wl["wqkv"], self.x, self.qkv, norm_w=wl["norm1"], eps=s.eps)        # RMSNorm fused into the read of x
                 rope_split(self.qkv, self.states[l].full.len, s.theta, self.q[l], self.k[l], self.v[l], s.n_q, s.n_kv)
             out = self.attention(l, kind) if with_attention else self.states[l].out
             if with_harness:
                 gemv(wl["wo"], out.view(-1), self.x, residual=self.x)
-                rmsnorm(self.x, wl["norm2"], s.eps, self.h)
-                gemv_swiglu(wl["wgu"], self.h, self.act)
+                gemv_swiglu(wl["wgu"], self.x, self.act, norm_w=wl["norm2"], eps=s.eps)
                 gemv(wl["wd"], self.act, self.x, residual=self.x)
         if with_harness:
-            rmsnorm(self.x, self.final_norm, s.eps, self.h)
-            gemv(self.lm_head, self.h, self.logits)
+            gemv(self.lm_head, self.x, self.logits, norm_w=self.final_norm, eps=s.eps)
             argmax(self.logits, self.token)
 
     def kind_of(self, t: int) -> str:

@@ -67,5 +67,5 @@ def test_harness_library_exports_every_declared_symbol():
     assert len(names) == 6 and sorted(harness.EXPORTS) == names
     for n in names:
         assert hasattr(harness.lib, n), n
-    assert harness.lib.llh_gemv(None, None, 0, None, None, 8, 256, None) == -1      # null pointers: rejected on the host
+    assert harness.lib.llh_gemv(None, None, 0, None, 1e-5, None, None, 8, 256, None) == -1      # null pointers: rejected on the host
     assert harness.lib.llh_rmsnorm(None, None, 1e-5, None, 4096, None) == -1

@@ -48,6 +48,9 @@ def test_rmsnorm_gemv_swiglu(H):
         assert (np.abs(f64(out) - want) <= 1e-5 * scale + 1e-6).all()
         H.gemv(w, x, out, residual=res)
         assert (np.abs(f64(out) - (want + f64(res))) <= 1e-5 * scale + 1e-5).all()
+        H.gemv(w, x, out, norm_w=wn, eps=1e-5)              # RMSNorm fused into the read of x
+        xn = LO.rmsnorm(f64(x), f64(wn), 1e-5)
+        assert (np.abs(f64(out) - LO.gemv(f64(w), xn)) <= 2e-5 * (np.abs(f64(w)) @ np.abs(xn)) + 1e-6).all()
         xb = x.to(torch.bfloat16)                           # bf16 input vector (the attention output)
         H.gemv(w, xb, out)
         assert (np.abs(f64(out) - LO.gemv(f64(w), f64(xb))) <= 1e-5 * scale + 1e-6).all()
@@ -59,6 +62,9 @@ def test_rmsnorm_gemv_swiglu(H):
     act = torch.empty(777, device="cuda")
     H.gemv_swiglu(wgu, x, act)
     assert np.allclose(f64(act), LO.swiglu_in(f64(wgu), f64(x)), rtol=1e-4, atol=1e-5)
+    wn = (1.0 + 0.1 * torch.randn(1024, generator=g, device="cuda")).to(torch.bfloat16)
+    H.gemv_swiglu(wgu, x, act, norm_w=wn, eps=1e-5)
+    assert np.allclose(f64(act), LO.swiglu_in(f64(wgu), LO.rmsnorm(f64(x), f64(wn), 1e-5)), rtol=2e-4, atol=2e-5)
 
 
 @pytest.mark.parametrize("pos", [0, 1, 777, 33791])
