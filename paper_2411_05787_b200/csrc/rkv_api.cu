@@ -43,7 +43,7 @@ int splits_for(const rkv_config* c) {
   return s < rkv::kMaxSplits ? (s < 1 ? 1 : s) : rkv::kMaxSplits;
 }
 
-struct WsLayout { size_t partials, tickets, len_tickets, win_keys, logits, status, total; int64_t logit_stride; };
+struct WsLayout { size_t partials, ml_t, tickets, len_tickets, win_keys, logits, status, total; int64_t logit_stride; };
 
 WsLayout ws_layout(const rkv_config* c) {
   WsLayout w;
@@ -53,6 +53,7 @@ WsLayout ws_layout(const rkv_config* c) {
   w.logit_stride = ((int64_t)c->max_len + 63) & ~int64_t(63);
   size_t off = 0;
   w.partials = off; off = up(off + bg * splits_for(c) * rkv::PartialLayout::kFloats * sizeof(float));
+  w.ml_t = off;     off = up(off + bg * 16 * (size_t)splits_for(c) * sizeof(float));
   w.tickets = off;  off = up(off + bg * sizeof(int32_t));
   w.len_tickets = off; off = up(off + (size_t)c->n_seq * sizeof(int32_t));
   w.win_keys = off; off = up(off + bg * (size_t)c->max_small * sizeof(uint32_t));
@@ -189,6 +190,7 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.out = out;
   p.partials = ctx->partials;
   p.tickets = ctx->tickets;
+  p.ml_t = ctx->ml_t;
   p.logits = logits ? ctx->logits : nullptr;
   p.status = ctx->status;
   p.logit_stride = ctx->logit_stride;
@@ -287,6 +289,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   if (e != cudaSuccess) { cudaFree(ctx->workspace); delete ctx; return RKV_ERR_CUDA; }
   ctx->workspace_bytes = w.total;
   ctx->partials = reinterpret_cast<float*>(ctx->workspace + w.partials);
+  ctx->ml_t = reinterpret_cast<float*>(ctx->workspace + w.ml_t);
   ctx->tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.tickets);
   ctx->len_tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.len_tickets);
   ctx->win_keys = reinterpret_cast<uint32_t*>(ctx->workspace + w.win_keys);
@@ -324,6 +327,7 @@ static rkv_status full_step_impl(rkv_ctx* ctx, const void* q, const rkv_cache* f
   memset(&sp, 0, sizeof(sp));
   sp.logits = ctx->logits;
   sp.partials = ctx->partials;
+  sp.ml_t = ctx->ml_t;
   sp.q = q;
   sp.out = out;
   sp.q_last_full = q_last_full;

@@ -610,6 +610,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         }
       part[kMaxGroup * kHeadDim + d] = Md;
       part[kMaxGroup * kHeadDim + kMaxGroup + d] = Ld;
+      if (kLogits && p.ml_t != nullptr) {   // the selection kernel reads these across the splits: keep a contiguous copy
+        float* t = p.ml_t + (int64_t)bg * 16 * p.max_splits + split;
+        t[(int64_t)d * p.max_splits] = Md;
+        t[(int64_t)(kMaxGroup + d) * p.max_splits] = Ld;
+      }
     }
     if (kLogits) return;   // full step: the selection kernel folds the partials
     __threadfence();

@@ -38,6 +38,7 @@ struct AttnParams {
   const int32_t* active;      // [B] or null
   void* out;                  // bf16 [B][Hq][128]
   float* partials;            // [B*Hkv][max_splits][PartialLayout::kFloats]
+  float* ml_t;                // [B*Hkv][16][max_splits]: the (m, l) of the partials again, split-contiguous, or null
   int32_t* tickets;           // [B*Hkv]
   float* logits;              // [B*Hkv][logit_stride][gp] (position-major) or null
   int32_t* status;
@@ -68,6 +69,7 @@ struct AttnParams {
 struct SelectParams {
   const float* logits;        // [B*Hkv][logit_stride][gp]
   const float* partials;      // split partials written by the attention kernel
+  const float* ml_t;          // [B*Hkv][16][max_splits]: m of head j (j < 8) / l of head j - 8, contiguous over the splits
   const void* q;              // bf16 [B][Hq][128]
   void* out;                  // bf16 [B][Hq][128]
   void* q_last_full;          // bf16 [B][Hq][128] or null
@@ -169,6 +171,7 @@ struct rkv_ctx {
   char* workspace;
   size_t workspace_bytes;
   float* partials;
+  float* ml_t;
   int32_t* tickets;
   int32_t* len_tickets;
   uint32_t* win_keys;

@@ -231,9 +231,9 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
   for (int k = 0; k < 4; ++k) {
     const int s = lane + 32 * k;
     const bool on = warp < kMaxGroup && s < gx;
-    const float* ps = pbase + (int64_t)s * PartialLayout::kFloats + kMaxGroup * kHeadDim;
-    wm[k] = on ? __ldcg(ps + warp) : -INFINITY;
-    wl[k] = on ? __ldcg(ps + kMaxGroup + warp) : 0.f;
+    const float* pt = p.ml_t + ((int64_t)bg * 16 + warp) * p.max_splits + s;   // contiguous over the splits
+    wm[k] = on ? __ldcg(pt) : -INFINITY;
+    wl[k] = on ? __ldcg(pt + (int64_t)kMaxGroup * p.max_splits) : 0.f;
   }
   float opre[kOPre];
 #pragma unroll
@@ -462,6 +462,7 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
   const bool ident = count > (uint32_t)kCandMax;
 
   // ---------------------------------------------------------------- 4: exchange the final bin
+  if (tid < kCandMax && tid >= (int)count) sh->flat[tid] = kPadKey;   // nobody pushes there: lets the search read vectors
   uint32_t flat_base = 0;   // where this CTA's keys start in the flat array (CTA order)
 #pragma unroll
   for (int r = 0; r < kSelectCluster; ++r)
@@ -509,18 +510,21 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
     while (lp < 5 && ((int)count << (lp + 1)) <= NT) ++lp;
     const int ci = tid >> lp, part = tid & ((1 << lp) - 1);
     if (ci < (int)count) {                        // whole groups of P lanes take this branch together
-      const int len = ((int)count + (1 << lp) - 1) >> lp;
-      const int j0 = part * len, j1 = (j0 + len < (int)count) ? j0 + len : (int)count;
+      const int len = ((((int)count + (1 << lp) - 1) >> lp) + 3) & ~3;   // a multiple of four: 16-byte reads
+      const int j0 = part * len;
       const uint32_t c = sh->flat[ci];
       uint32_t less = 0, eq = 0, less_p = 0, eq_p = 0;
-#pragma unroll 4
-      for (int j = j0; j < j1; ++j) {
-        const uint32_t x = sh->flat[j];
-        const bool pre = j < (int)flat_base;
-        less += (x < c);
-        eq += (x == c);
-        less_p += (pre && x < c);
-        eq_p += (pre && x == c);
+      for (int j = j0; j < j0 + len && j < kCandMax; j += 4) {
+        const uint4 x4 = *reinterpret_cast<const uint4*>(&sh->flat[j]);
+        const uint32_t xs[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool pre = j + e < (int)flat_base;
+          less += (xs[e] < c);
+          eq += (xs[e] == c);
+          less_p += (pre && xs[e] < c);
+          eq_p += (pre && xs[e] == c);
+        }
       }
       const uint32_t gmask = __activemask();
       for (int o = 1; o < (1 << lp); o <<= 1) {
