@@ -30,9 +30,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 # DRAM traffic of one full-step attention launch per algorithmic K/V byte, from the ncu capture of the cfg-2
-# launch summarised in profiles/attn_kernel_full_step_cfg2_L32768.md (134.26 MB read + 4.88 MB written for
+# launch summarised in profiles/attn_kernel_full_step_cfg2_L32768.md (134.27 MB read + 3.54 MB written for
 # 134.22 MB of K/V); traffic grows with the positions streamed.  Set to None when the kernel changes.
-ATTN_FULL_TRAFFIC_PER_KV_BYTE = 139.14 / 134.22
+ATTN_FULL_TRAFFIC_PER_KV_BYTE = 137.81 / 134.22
 
 METRIC = "decode attention us/token (all layers, refresh schedule of the workload; full step and small step also reported)"
 UNIT = "us/token"
