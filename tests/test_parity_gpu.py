@@ -637,3 +637,93 @@ def test_config4_ragged_sampled_sequences(mods):
     seqs = [int(order[0]), int(order[len(order) // 2]), int(order[-1])]
     n_full = run_trajectory(mods, w, 0, seqs=seqs)
     assert all(v == 1 for v in n_full.values())
+
+
+def test_largest_supported_length(mods):
+    """One sequence close to the selection kernel's limit (8 CTAs x 40960 keys): 300000 positions, top-4096."""
+    lens, k_small = [300000], [4096]
+    ctx, st, cache, q = make_layer(mods, lens, k_small, 2, 1, seed=41, want_scores=True)
+    st.refresh(q)
+    assert ctx.device_status() == 0
+    check_full_against_oracle(st, cache, q, lens, k_small, 1)
+    out = st.partial(q).clone()
+    n = 300000
+    kf, vf = host_heads(cache, 0, 1, "k"), host_heads(cache, 0, 1, "v")
+    sel = [st.topk_idx[0, 0, :4096].cpu().numpy().astype(np.int64)]
+    want, _, _ = O.decode_attention(O.bf16_bits_to_f64(bits(q[0])), O.bf16_bits_to_f64(np.stack(O.gather_rows(kf, sel))),
+                                    O.bf16_bits_to_f64(np.stack(O.gather_rows(vf, sel))))
+    check_out(out[0], want, "partial step on 4096 of 300000")
+    rkv = mods[0]
+    with pytest.raises(rkv.RkvError):
+        rkv.Context(1, 2, 1, 8 * 40960 + 1, 64)            # beyond the limit: refused at creation
+
+
+def test_bench_configuration_graph_replay_shared_context(mods):
+    """The launch configuration bench.py times, at config 2's full size: several layers share one context, a token's
+    calls (rkv_append_small_step, or rkv_append + rkv_full_step + rkv_gather_small) are replayed from CUDA graphs
+    with the inputs staged in a device buffer.  Every layer's output of every token is compared with the oracle."""
+    rkv, runner, synth = mods
+    dev = torch.device("cuda")
+    NL, S, T = 2, 10, 11
+    w = synth.scaled(synth.config2(n_layers=NL), steps=T)
+    L, K, Hq, Hkv = w.lens[0], w.k_small[0], w.n_q_heads, w.n_kv_heads
+    full_hint, small_hint = L + T + 1, K + S + 2
+    ctx = rkv.Context(1, Hq, Hkv, full_hint, small_hint)
+    q_stage = torch.zeros((NL, 1, Hq, 128), dtype=torch.bfloat16, device=dev)
+    k_stage = torch.zeros((NL, 1, Hkv, 128), dtype=torch.bfloat16, device=dev)
+    v_stage = torch.zeros((NL, 1, Hkv, 128), dtype=torch.bfloat16, device=dev)
+    layers, states, inputs = [], [], []
+    for l in range(NL):
+        cache = synth.fill_layer(w, l, dev)
+        qs = synth.query_trajectory(w, l).to(dev)
+        kn, vn = synth.new_token_kv(w, l)
+        synth.plant_heavy(w, cache, l, qs[0])
+        st = runner.LayerState(ctx, cache, [K], S + 2, Hq, Hkv)
+        layers.append(st)
+        inputs.append((qs, kn.to(dev), vn.to(dev)))
+        states.append(O.SequenceState(host_heads(cache, 0, Hkv, "k").copy(), host_heads(cache, 0, Hkv, "v").copy(), L, K))
+
+    def stage(t):
+        for l in range(NL):
+            q_stage[l].copy_(inputs[l][0][t]); k_stage[l].copy_(inputs[l][1][t]); v_stage[l].copy_(inputs[l][2][t])
+
+    def token(kind):
+        for l, st in enumerate(layers):
+            if kind == "full":
+                st.append(k_stage[l], v_stage[l])
+                st.refresh(q_stage[l], max_len_hint=full_hint)
+            else:
+                st.append_partial(q_stage[l], k_stage[l], v_stage[l], max_len_hint=small_hint)
+
+    class W1:      # what follow_gpu_selection needs to know about the workload
+        n_kv_heads, k_small = Hkv, [K]
+    stage(0)
+    for l, st in enumerate(layers):          # initial small caches (eager; also builds the tensor maps)
+        st.refresh(q_stage[l], max_len_hint=full_hint)
+        o_out, o_score, _ = states[l].full(bits(inputs[l][0][0, 0]))
+        check_out(st.out[0], o_out, f"init layer {l}")
+        follow_gpu_selection(st, states[l], 0, o_score, W1)
+    # warm both kinds eagerly on throw-away copies?  No: capture directly; capture does not execute
+    torch.cuda.synchronize()
+    graphs, side = {}, torch.cuda.Stream()
+    for kind in ("small", "full"):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(gr, stream=side):
+                token(kind)
+        graphs[kind] = gr
+    for t in range(1, T + 1):
+        stage(t)
+        kind = "full" if t % S == 0 else "small"
+        graphs[kind].replay()
+        torch.cuda.synchronize()
+        for l, st in enumerate(layers):
+            states[l].append(bits(inputs[l][1][t, 0]), bits(inputs[l][2][t, 0]))
+            if kind == "full":
+                o_out, o_score, _ = states[l].full(bits(inputs[l][0][t, 0]))
+                check_out(st.out[0], o_out, f"full token {t} layer {l}")
+                follow_gpu_selection(st, states[l], 0, o_score, W1)
+            else:
+                check_out(st.out[0], states[l].small(bits(inputs[l][0][t, 0])), f"partial token {t} layer {l}")
+    assert ctx.device_status() == 0
+    assert all(int(st.full.len[0]) == L + T and int(st.small.len[0]) == K + 1 for st in layers)
