@@ -380,10 +380,11 @@ def run_ours(args):
 
     # ---- main measurement: inputs resident in HBM.  The token counter runs on through all phases, so a
     # refresh (or a check) comes every S tokens and the small caches never outgrow their capacity.
-    run_tokens(args.warmup)
+    # clocks are sampled from the warm-up on (same load as the timed region, which may be shorter than one sample period)
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else 0)
     if rank == 0:
         sampler.start()
+    run_tokens(args.warmup)
     torch.cuda.synchronize()
     flag_total.zero_()
     ms, cnt = timed(args.steps)
