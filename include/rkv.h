@@ -18,6 +18,8 @@
  *    word), sized once in rkv_create.  Calls on one context must not overlap
  *    on the GPU (they share that workspace): issue them on one stream.
  *  - bf16 tensors are plain arrays of 16-bit brain floats.  head_dim is 128.
+ *    Every bf16 tensor (q, out, k_new, v_new, cache buffers) starts on a
+ *    16-byte boundary; a misaligned base is RKV_ERR_INVALID_ARG.
  *  - Query head h reads KV head h / G, G = n_q_heads / n_kv_heads (1..8).
  *  - Errors: every call returns an rkv_status.  Bad arguments are detected on
  *    the host before anything is launched.  Conditions only the device can

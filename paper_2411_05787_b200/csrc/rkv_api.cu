@@ -14,11 +14,7 @@ using rkv::AttnParams;
 using rkv::CacheDev;
 using rkv::SelectParams;
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn g_encode = nullptr;
+rkv::EncodeTiledFn g_encode = nullptr;
 // kernel attributes (dynamic shared-memory sizes) are set per device, once
 constexpr int kMaxDevices = 64;
 bool g_prepared[kMaxDevices] = {};
@@ -69,6 +65,7 @@ rkv_status cuda_fail(rkv_ctx* ctx, cudaError_t e, const char* where) {
   return RKV_ERR_CUDA;
 }
 
+bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }   // NULL counts as aligned
 bool cache_ok(const rkv_cache* c) {
   return c && c->k && c->v && c->row_offset && c->cap && c->len && c->n_rows > 0 && c->n_rows < (int64_t(1) << 31) &&
          (reinterpret_cast<uintptr_t>(c->k) & 15) == 0 && (reinterpret_cast<uintptr_t>(c->v) & 15) == 0;
@@ -96,7 +93,7 @@ struct LaunchScope {
 
 CacheDev dev_of(const rkv_cache* c) { return CacheDev{c->k, c->v, c->row_offset, c->cap, c->len}; }
 
-// 2-D view [n_rows][128] bf16, box = 64 rows x 64 channels (128 bytes), 128-byte swizzle
+// [n_rows][128] bf16 as {64 channels, row, half}: one box = 64 rows x both halves, 128-byte swizzle
 rkv_status tensor_map(rkv_ctx* ctx, void* base, int64_t n_rows, CUtensorMap* out) {
   const std::pair<uint64_t, int64_t> key(reinterpret_cast<uint64_t>(base), n_rows);   // the map depends on nothing else
   auto it = ctx->tmaps.find(key);
@@ -107,16 +104,10 @@ rkv_status tensor_map(rkv_ctx* ctx, void* base, int64_t n_rows, CUtensorMap* out
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
     if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess)
       return cuda_fail(ctx, e == cudaSuccess ? cudaErrorUnknown : e, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)");
-    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    g_encode = reinterpret_cast<rkv::EncodeTiledFn>(fn);
   }
-  cuuint64_t dims[2] = {(cuuint64_t)rkv::kHeadDim, (cuuint64_t)n_rows};
-  cuuint64_t strides[1] = {(cuuint64_t)rkv::kHeadDim * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)rkv::kTile};
-  cuuint32_t estr[2] = {1, 1};
   CUtensorMap tm;
-  CUresult r = g_encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = rkv::encode_cache_map(g_encode, base, n_rows, &tm);
   if (r != CUDA_SUCCESS) {
     ctx->last_error = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string((int)r);
     return RKV_ERR_CUDA;
@@ -164,6 +155,8 @@ bool cluster_eligible(const rkv_ctx* ctx, int n_max) { return ctx->small_cluster
 rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
                          int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out, int* gx_out,
                          const AppendArgs* app = nullptr, bool score_only = false) {
+  if (!aligned16(q) || !aligned16(out) || (app != nullptr && (!aligned16(app->k_new) || !aligned16(app->v_new))))
+    return RKV_ERR_INVALID_ARG;   // the kernels read and write these 16 bytes at a time
   CUtensorMap tm_k, tm_v;
   rkv_status s = tensor_map(ctx, cache->k, cache->n_rows, &tm_k);
   if (s != RKV_OK) return s;

@@ -10,7 +10,7 @@
 //
 // Shape of the kernel: one CTA per (sequence, KV head, chunk of positions).
 // A copy warp streams 64-position tiles of K and V into a shared-memory ring (3 stages,
-// 6 in the clustered partial step) with 2-D tensor-map TMA loads (128-byte swizzle, completion on
+// 6 in the clustered partial step) with tensor-map TMA loads, one per K or V tile (128-byte swizzle, completion on
 // mbarriers).  Four MMA warps each own 16 positions of a tile: S^T = K Q^T and
 // O^T += V^T P^T with m16n8k16 bf16 tensor-core MMAs (fp32 accumulate), where
 // the N=8 dimension holds all query heads of the group, so K/V are read once
@@ -40,6 +40,7 @@ constexpr int kHalfBytes = kTile * 128;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kOPad = 132;  // floats per head row in the merge buffer (bank spread)
+constexpr int kQPad = 68;   // 32-bit words per query row in shared memory (64 + 4: the fragment reads spread over all banks)
 constexpr int kRecvFloats = kMaxGroup * kHeadDim + kAttnCluster * kMaxGroup * 2;   // pushed slices + (m, l) pairs
 
 enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2, kModeClusterAppend = 3, kModeScore = 4 };
@@ -73,13 +74,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
-                                            uint32_t bar, uint64_t policy) {
+// One K (or V) tile: the box {64 channels, 64 rows, 2 halves} at row y.
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* tm, int y, uint32_t bar,
+                                              uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-      " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
-      "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
+      "l"(tm), "r"(0), "r"(y), "r"(0), "r"(bar), "l"(policy)
       : "memory");
+}
+// Pulls one tile into L2 only.  L2 is the point of coherence, so this is safe while another kernel still writes
+// the rows: a later load sees whatever has been written by then.
+__device__ __forceinline__ void tma_prefetch_tile_l2(const CUtensorMap* tm, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tm), "r"(0), "r"(y),
+               "r"(0)
+               : "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void* ptr) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr) : "memory");
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
@@ -149,9 +161,10 @@ struct Ring {
   static constexpr bool kWide = kWideT && (kMode == kModeCluster || kMode == kModeClusterAppend);
   static constexpr int kStg = kWide ? 6 : kStages;
   static constexpr int kMinBlocks = kWide ? 1 : 2;
-  // The clustered partial step is bound by the latency of one warp's MMA / softmax chain per tile, not by
-  // bandwidth: two groups of four MMA warps take alternate tiles.
-  static constexpr int kMmaWarps = kWide ? 8 : 4;
+  // The clustered partial step is bound by the length of one warp's MMA / softmax instruction chain, not by
+  // bandwidth: five pairs of MMA warps take alternate tiles, so that a chunk of up to five tiles (a small
+  // cache of 2048 rows plus the rows appended since, over eight CTAs) is one pass for every warp.
+  static constexpr int kMmaWarps = kWide ? 10 : 4;
   static constexpr int kThreads = 32 * (kMmaWarps + 1);
 };
 
@@ -165,7 +178,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   constexpr bool kAppend = (kMode == kModeClusterAppend);
   constexpr int kStg = Ring<kMode, kWideT>::kStg;
   constexpr int kMW = Ring<kMode, kWideT>::kMmaWarps;      // MMA warps; warp kMW is the copy warp
-  constexpr int kGroups = kMW / 4;                  // groups of four warps that take alternate tiles
+  // Rows of a tile per MMA warp.  The bandwidth-bound forms use 16 (four warps per tile).  The clustered
+  // partial step is bound by the length of one warp's instruction chain: there a warp takes 32 rows, two
+  // independent 16-row blocks that share one softmax update, and two warps cover a tile.
+  constexpr int kNB = kWideT ? 2 : 1;               // 16-row blocks per warp
+  constexpr int kBand = 16 * kNB;
+  constexpr int kWT = kTile / kBand;                // warps per tile
+  constexpr int kGroups = kMW / kWT;                // groups of warps that take alternate tiles
   auto consumer_bar = [] { consumer_bar_n<32 * kMW>(); };
   extern __shared__ uint8_t smem_raw[];
   __shared__ int s_last;
@@ -181,7 +200,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   if (tid == 0) {
     for (int s = 0; s < kStg; ++s) {
       mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, 4);
+      mbar_init(bar_empty + 8 * s, kWT);   // one arrival per MMA warp that reads the tile
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -199,6 +218,37 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // stream predecessor is still running; everything else waits for the dependency.
   const int cap = __ldg(p.cap + b);
   const int64_t roff = __ldg(p.row_offset + b);
+  // A clustered step is short and usually sits at the dependency wait while its stream predecessor runs: use
+  // that time to bring this CTA's rows from DRAM into L2, so that the copies after the wait are L2 hits.
+  // The same goes for the few lines the step reads first (sizes, query, new rows): with many layers' caches
+  // streaming through L2 between two calls on one layer they have usually been evicted.
+  if (kCluster && warp == kMW) {
+    if (p.spec != 0 && lane == 0) {
+      const int n_pre = (p.chunk + kTile - 1) / kTile < kStg ? (p.chunk + kTile - 1) / kTile : kStg;   // = n_spec below
+      const int y0 = (int)(roff + (int64_t)g * cap + (int64_t)split * p.chunk);
+      for (int t = 0; t < n_pre; ++t) {
+        tma_prefetch_tile_l2(&tm_k, y0 + t * kTile);
+        tma_prefetch_tile_l2(&tm_v, y0 + t * kTile);
+      }
+    }
+    const int64_t nrow_b = ((int64_t)b * p.n_kv_heads + g) * kHeadDim * 2;   // byte offset of this head's new row
+    if (lane == 1) prefetch_l2(p.len + b);
+    if (lane == 2 && p.active != nullptr) prefetch_l2(p.active + b);
+    if (lane >= 3 && lane < 3 + 2 * G) prefetch_l2(qg + (lane - 3) * 64);   // 128-byte lines of the G query rows
+    if (kAppend) {
+      if (lane == 19 || lane == 20) prefetch_l2(static_cast<const uint8_t*>(p.k_new) + nrow_b + (lane - 19) * 128);
+      if (lane == 21 || lane == 22) prefetch_l2(static_cast<const uint8_t*>(p.v_new) + nrow_b + (lane - 21) * 128);
+      if (p.has_full) {
+        if (lane == 23) prefetch_l2(p.full_len + b);
+        if (lane == 24) prefetch_l2(p.full_cap + b);
+        if (lane == 25) prefetch_l2(p.full_row_offset + b);
+      }
+      if (p.evict_order != nullptr) {
+        if (lane == 26) prefetch_l2(p.k_small + b);
+        if (lane == 27) prefetch_l2(p.evict_count + b);
+      }
+    }
+  }
   __syncthreads();   // barrier initialisation (above) is visible to every warp
   pdl_wait();
 
@@ -208,19 +258,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     const uint32_t dst = smem_base + s * kStageBytes, bar = bar_full + 8 * s;
     const int y = (int)(row_first + (int64_t)t * kTile);
     mbar_expect_tx(bar, kScoreOnly ? 2 * kHalfBytes : kStageBytes);
-    tma_load_2d(dst, &tm_k, 0, y, bar, policy);
-    tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar, policy);
-    if (!kScoreOnly) {
-      tma_load_2d(dst + 2 * kHalfBytes, &tm_v, 0, y, bar, policy);
-      tma_load_2d(dst + 3 * kHalfBytes, &tm_v, 64, y, bar, policy);
-    }
+    tma_load_tile(dst, &tm_k, y, bar, policy);
+    if (!kScoreOnly) tma_load_tile(dst + 2 * kHalfBytes, &tm_v, y, bar, policy);
   };
   // When the host knows that every CTA of the grid has work (no mask; one sequence, or a cluster per head), the
   // chunk of this CTA follows from the launch geometry alone, so its first tiles are requested before the length
   // has even been read (tiles past the length are waited for and ignored).  Saves one memory round trip.
   int n_spec = 0;
   if (p.spec != 0) {
-    n_spec = p.chunk / kTile < kStg ? p.chunk / kTile : kStg;
+    n_spec = (p.chunk + kTile - 1) / kTile < kStg ? (p.chunk + kTile - 1) / kTile : kStg;
     if (tid == 32 * kMW) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
@@ -232,19 +278,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // per-sequence sizes and (MMA warps) the query fragments: independent loads, one round trip
   const int act = (p.active != nullptr) ? __ldcg(p.active + b) : 1;
   int n = __ldcg(p.len + b);
-  uint32_t qb[8][2];              // B fragments of Q^T: [k = channel][n = head]
-  if (warp < kMW) {
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      if (qd < G) {
-        qb[ks][0] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc);
-        qb[ks][1] = *reinterpret_cast<const uint32_t*>(qg + qd * kHeadDim + 16 * ks + qc + 8);
-      } else {
-        qb[ks][0] = 0u;
-        qb[ks][1] = 0u;
-      }
-    }
-  }
+  // The G query rows go through shared memory: G * 16 coalesced 16-byte loads for the whole CTA instead of
+  // sixteen 4-byte loads per lane (the memory pipe's request rate, not its latency, is what those cost).
+  uint32_t* sm_q = reinterpret_cast<uint32_t*>(smem_gen + kStg * kStageBytes + 16 * kStg + 16 + kRecvFloats * 4);
+  const bool q_lane = warp < kMW && tid < G * 16;
+  uint4 qv = make_uint4(0u, 0u, 0u, 0u);
+  if (q_lane) qv = __ldcg(reinterpret_cast<const uint4*>(qg) + tid);
   // fused append: this lane's 8 bytes of the new K and V rows, and the second cache's sizes
   uint2 kn = make_uint2(0u, 0u), vn = make_uint2(0u, 0u);
   int pos_new = -1;            // where the new row lands in the attended cache (-1: no room, or no append)
@@ -263,6 +302,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       kn = __ldcg(static_cast<const uint2*>(p.k_new) + nrow + lane);
       vn = __ldcg(static_cast<const uint2*>(p.v_new) + nrow + lane);
     }
+    // (the query's store to shared memory waits for its load; it comes after every other load has been issued)
+    if (q_lane) *reinterpret_cast<uint4*>(sm_q + (tid >> 4) * kQPad + (tid & 15) * 4) = qv;
     // Where the new row goes in the attended cache: behind the last row (the cache grows), or - fixed-size small
     // cache that has reached its size - into the slot of the lowest-scoring survivor of the last refresh.
     int slot = n;
@@ -297,6 +338,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     if (ok_s) {
       pos_new = slot;
       if (!evicting) n = n + 1;
+    }
+  }
+  if (!kAppend && q_lane) *reinterpret_cast<uint4*>(sm_q + (tid >> 4) * kQPad + (tid & 15) * 4) = qv;
+  uint32_t qb[8][2];              // B fragments of Q^T: [k = channel][n = head]
+  if (warp < kMW) {
+    consumer_bar();               // the query rows are in shared memory
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qb[ks][0] = qd < G ? sm_q[qd * kQPad + 8 * ks + (lane & 3)] : 0u;
+      qb[ks][1] = qd < G ? sm_q[qd * kQPad + 8 * ks + 4 + (lane & 3)] : 0u;
     }
   }
   // Fused append: the lengths are bumped by the last (sequence, KV head) cluster to get here.  Every cluster
@@ -384,9 +435,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   uint64_t keep_policy = 0;
   if (kLogits) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep_policy));
 
-  const int w4 = warp & 3, grp = warp >> 2;   // 16-row band inside a tile; which tiles this warp takes
-  const int krow = 16 * w4 + (lane & 15);
-  const int vrow = 16 * w4 + ((lane >> 4) << 3) + (lane & 7);
+  // A warp owns a band of kNB 16-row blocks of every tile its group takes (kWT warps per tile).
+  const int wb = warp % kWT, grp = warp / kWT;
+  const int band0 = kBand * wb;               // first row of the band inside a tile
   bool ok = true;
 
   const int n_wait = n_tiles > n_spec ? n_tiles : n_spec;   // tiles requested ahead of the length are always consumed
@@ -397,12 +448,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       ok = false;
       break;
     }
-    const int pos_base = start + t * kTile + 16 * w4;
+    const int pos_base = start + t * kTile + band0;
     if (kAppend) {
       // The tile came from global memory, where the new row may not have landed yet: the warp that owns the
       // row writes it into the tile itself (same 128-byte swizzle as the copy engine uses).
       const int rel = pos_new - (start + t * kTile);
-      if (rel >= 0 && rel < kTile && (rel >> 4) == w4) {
+      if (rel >= 0 && rel < kTile && rel / kBand == wb) {
         const uint32_t at = smem_base + s * kStageBytes + (lane >> 4) * kHalfBytes + rel * 128 +
                             ((((lane & 15) >> 1) ^ (rel & 7)) << 4) + (lane & 1) * 8;
         st_shared_v2(at, kn);
@@ -412,28 +463,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     }
     if (t < n_tiles && pos_base < end) {
       const uint32_t kbase = smem_base + s * kStageBytes;
-      float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};   // two chains: half the dependent MMA latency
+      // S^T = K Q^T for the band: two accumulator chains per block (half the dependent MMA latency)
+      float c[kNB][4], c2[kNB][4];
+#pragma unroll
+      for (int i = 0; i < kNB; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c[i][j] = c2[i][j] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const int chunk = 2 * ks + (lane >> 4);
-        uint32_t a[4];
-        ldsm_x4(a, kbase + (chunk >> 3) * kHalfBytes + krow * 128 + (((chunk & 7) ^ (krow & 7)) << 4));
-        if (ks & 1) mma_bf16(c2, a, qb[ks][0], qb[ks][1]);
-        else mma_bf16(c, a, qb[ks][0], qb[ks][1]);
-      }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) c[i] += c2[i];
-      const int r0 = pos_base + qd, r1 = r0 + 8;
-      float s0 = c[0] * p.scale, s1 = c[1] * p.scale, s2 = c[2] * p.scale, s3 = c[3] * p.scale;
-      if (kLogits) {
-        if (lg_on) {
-          if (r0 < end) st_keep_f2(lg0 + (int64_t)r0 * p.gp, s0, s1, keep_policy);
-          if (r1 < end) st_keep_f2(lg0 + (int64_t)r1 * p.gp, s2, s3, keep_policy);
+        for (int i = 0; i < kNB; ++i) {
+          const int krow = band0 + 16 * i + (lane & 15);
+          uint32_t a[4];
+          ldsm_x4(a, kbase + (chunk >> 3) * kHalfBytes + krow * 128 + (((chunk & 7) ^ (krow & 7)) << 4));
+          if (ks & 1) mma_bf16(c2[i], a, qb[ks][0], qb[ks][1]);
+          else mma_bf16(c[i], a, qb[ks][0], qb[ks][1]);
         }
       }
-      if (r0 >= end) s0 = s1 = ninf;
-      if (r1 >= end) s2 = s3 = ninf;
-      float t0 = fmaxf(s0, s2), t1 = fmaxf(s1, s3);
+      float sc[kNB][4];
+      float t0 = ninf, t1 = ninf;
+#pragma unroll
+      for (int i = 0; i < kNB; ++i) {
+        const int r0 = pos_base + 16 * i + qd, r1 = r0 + 8;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sc[i][j] = (c[i][j] + c2[i][j]) * p.scale;
+        if (kLogits) {
+          if (lg_on) {
+            if (r0 < end) st_keep_f2(lg0 + (int64_t)r0 * p.gp, sc[i][0], sc[i][1], keep_policy);
+            if (r1 < end) st_keep_f2(lg0 + (int64_t)r1 * p.gp, sc[i][2], sc[i][3], keep_policy);
+          }
+        }
+        if (r0 >= end) sc[i][0] = sc[i][1] = ninf;
+        if (r1 >= end) sc[i][2] = sc[i][3] = ninf;
+        t0 = fmaxf(t0, fmaxf(sc[i][0], sc[i][2]));
+        t1 = fmaxf(t1, fmaxf(sc[i][1], sc[i][3]));
+      }
 #pragma unroll
       for (int sh = 4; sh <= 16; sh <<= 1) {
         t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, sh));
@@ -457,35 +522,46 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       }
       const float nm0 = (m0 == ninf) ? 0.f : -m0 * kLog2e;
       const float nm1 = (m1 == ninf) ? 0.f : -m1 * kLog2e;
-      const float p0 = ex2(fmaf(s0, kLog2e, nm0)), p1 = ex2(fmaf(s1, kLog2e, nm1));
-      const float p2 = ex2(fmaf(s2, kLog2e, nm0)), p3 = ex2(fmaf(s3, kLog2e, nm1));
-      l0 += p0 + p2;
-      l1 += p1 + p3;
-      if (!kScoreOnly) {
-      // P^T as the B operand: transpose the two 8x8 [position][head] blocks inside the warp
-      const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1));
-      const uint32_t pb1 = movmatrix_t(pack_bf16(p2, p3));
-      const uint32_t vbase = kbase + 2 * kHalfBytes;
-      const bool tail = pos_base + 16 > end;
-      uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
-      if (tail) {  // rows past the end may hold anything (even NaN): zero them so that 0 * x stays 0
-        const int pa = pos_base + qc;
-        mk0 = (pa < end ? 0x0000ffffu : 0u) | (pa + 1 < end ? 0xffff0000u : 0u);
-        mk1 = (pa + 8 < end ? 0x0000ffffu : 0u) | (pa + 9 < end ? 0xffff0000u : 0u);
-      }
+      uint32_t pb[kNB][2];   // P^T as the B operand: the two 8x8 [position][head] blocks transposed inside the warp
 #pragma unroll
-      for (int mt = 0; mt < 8; ++mt) {
-        const int chunk = 2 * mt + ((lane >> 3) & 1);
-        uint32_t a[4];
-        ldsm_x4_t(a, vbase + (chunk >> 3) * kHalfBytes + vrow * 128 + (((chunk & 7) ^ (vrow & 7)) << 4));
-        if (tail) {
-          a[0] &= mk0;
-          a[1] &= mk0;
-          a[2] &= mk1;
-          a[3] &= mk1;
+      for (int i = 0; i < kNB; ++i) {
+        const float p0 = ex2(fmaf(sc[i][0], kLog2e, nm0)), p1 = ex2(fmaf(sc[i][1], kLog2e, nm1));
+        const float p2 = ex2(fmaf(sc[i][2], kLog2e, nm0)), p3 = ex2(fmaf(sc[i][3], kLog2e, nm1));
+        l0 += p0 + p2;
+        l1 += p1 + p3;
+        if (!kScoreOnly) {
+          pb[i][0] = movmatrix_t(pack_bf16(p0, p1));
+          pb[i][1] = movmatrix_t(pack_bf16(p2, p3));
         }
-        mma_bf16(o[mt], a, pb0, pb1);
       }
+      if (!kScoreOnly) {
+        const uint32_t vbase = kbase + 2 * kHalfBytes;
+#pragma unroll
+        for (int i = 0; i < kNB; ++i) {
+          const int pos_i = pos_base + 16 * i;
+          if (pos_i >= end) continue;   // the whole block lies past the end: its probabilities are zero
+          const int vrow = band0 + 16 * i + ((lane >> 4) << 3) + (lane & 7);
+          const bool tail = pos_i + 16 > end;
+          uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
+          if (tail) {  // rows past the end may hold anything (even NaN): zero them so that 0 * x stays 0
+            const int pa = pos_i + qc;
+            mk0 = (pa < end ? 0x0000ffffu : 0u) | (pa + 1 < end ? 0xffff0000u : 0u);
+            mk1 = (pa + 8 < end ? 0x0000ffffu : 0u) | (pa + 9 < end ? 0xffff0000u : 0u);
+          }
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt) {
+            const int chunk = 2 * mt + ((lane >> 3) & 1);
+            uint32_t a[4];
+            ldsm_x4_t(a, vbase + (chunk >> 3) * kHalfBytes + vrow * 128 + (((chunk & 7) ^ (vrow & 7)) << 4));
+            if (tail) {
+              a[0] &= mk0;
+              a[1] &= mk0;
+              a[2] &= mk1;
+              a[3] &= mk1;
+            }
+            mma_bf16(o[mt], a, pb[i][0], pb[i][1]);
+          }
+        }
       }
     }
     __syncwarp();
@@ -498,52 +574,69 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
   }
 
-  // ------------------------------------------------ merge the MMA warps (stage memory is free now)
-  consumer_bar();
-  float* sm_o = reinterpret_cast<float*>(smem_gen);   // [kMW][8][kOPad]
-  float* sm_ml = sm_o + kMW * 8 * kOPad;              // [kMW][8][2]
-#pragma unroll
-  for (int mt = 0; mt < 8; ++mt) {
-    const int d = 16 * mt + qd;
-    float* base = sm_o + (warp * 8 + qc) * kOPad;
-    base[d] = o[mt][0];
-    base[kOPad + d] = o[mt][1];
-    base[d + 8] = o[mt][2];
-    base[kOPad + d + 8] = o[mt][3];
-  }
+  // ------------------------------------------------ merge the MMA warps
+  // Every warp publishes its (m, l); after one barrier each warp knows the CTA-wide maximum of its two heads
+  // and writes its accumulators already scaled to it, so that the merge itself is a plain sum (few
+  // instructions per thread: this phase is bound by instruction issue, not by memory).
+  float* sm_wm = reinterpret_cast<float*>(sm_q + kMaxGroup * kQPad);   // [kMW][8]: per-warp maximum (own memory)
   if (lane < 4) {
-    float* ml = sm_ml + (warp * 8 + qc) * 2;
-    ml[0] = m0;
-    ml[1] = l0;
-    ml[2] = m1;
-    ml[3] = l1;
+    sm_wm[warp * 8 + qc] = m0;
+    sm_wm[warp * 8 + qc + 1] = m1;
+  }
+  consumer_bar();   // (m) of every warp is visible, and the stage memory is free
+  float* sm_o = reinterpret_cast<float*>(smem_gen);   // [kMW][8][kOPad] scaled accumulators
+  float* sm_l = sm_o + kMW * 8 * kOPad;               // [kMW][8] scaled denominators
+  float* sm_M = sm_l + kMW * 8;                       // [8] CTA-wide maximum per head
+  {
+    float M0 = ninf, M1 = ninf;
+#pragma unroll
+    for (int w = 0; w < kMW; ++w) {
+      M0 = fmaxf(M0, sm_wm[w * 8 + qc]);
+      M1 = fmaxf(M1, sm_wm[w * 8 + qc + 1]);
+    }
+    const float e0 = (m0 == ninf) ? 0.f : ex2((m0 - M0) * kLog2e);
+    const float e1 = (m1 == ninf) ? 0.f : ex2((m1 - M1) * kLog2e);
+    float* base = sm_o + (warp * 8 + qc) * kOPad + qd;
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      base[16 * mt] = o[mt][0] * e0;
+      base[kOPad + 16 * mt] = o[mt][1] * e1;
+      base[16 * mt + 8] = o[mt][2] * e0;
+      base[kOPad + 16 * mt + 8] = o[mt][3] * e1;
+    }
+    if (lane < 4) {
+      sm_l[warp * 8 + qc] = l0 * e0;
+      sm_l[warp * 8 + qc + 1] = l1 * e1;
+      if (warp == 0) {
+        sm_M[qc] = M0;
+        sm_M[qc + 1] = M1;
+      }
+    }
   }
   consumer_bar();
 
   const int d = tid;  // 0..127: one output channel per thread (further MMA warps only keep the barriers company)
   const bool chan = d < kHeadDim;
-  float accO[kMaxGroup], accM[kMaxGroup], accL[kMaxGroup];
+  float accO[kMaxGroup];
 #pragma unroll
   for (int h = 0; h < kMaxGroup; ++h) {
     accO[h] = 0.f;
-    accM[h] = ninf;
-    accL[h] = 0.f;
     if (!chan || h >= G) continue;
-    float M = ninf;
+    float O = 0.f;
 #pragma unroll
-    for (int w = 0; w < kMW; ++w) M = fmaxf(M, sm_ml[(w * 8 + h) * 2]);
-    float L = 0.f, O = 0.f;
-#pragma unroll
-    for (int w = 0; w < kMW; ++w) {
-      const float mw = sm_ml[(w * 8 + h) * 2];
-      const float e = (mw == ninf) ? 0.f : ex2((mw - M) * kLog2e);
-      L += sm_ml[(w * 8 + h) * 2 + 1] * e;
-      O += sm_o[(w * 8 + h) * kOPad + d] * e;
-    }
+    for (int w = 0; w < kMW; ++w) O += sm_o[(w * 8 + h) * kOPad + d];
     accO[h] = O;
-    accM[h] = M;
-    accL[h] = L;
   }
+  // (m, l) of one head for the whole CTA; heads beyond the group read as (-inf, 0)
+  auto head_ml = [&](int h, float& M, float& L) {
+    M = ninf;
+    L = 0.f;
+    if (h < G) {
+      M = sm_M[h];
+#pragma unroll
+      for (int w = 0; w < kMW; ++w) L += sm_l[w * 8 + h];
+    }
+  };
 
   const int bg = b * p.n_kv_heads + g;
 
@@ -561,13 +654,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         if (h < G) st_cluster_f32(map_rank(recv_u32 + 4u * ((split * kMaxGroup + h) * dchunk + dd), owner), accO[h]);
       if (d < kMaxGroup * C) {   // (m, l) of head d % 8 to peer d / 8
         const int h = d & 7, peer = d >> 3;
-        float Md = ninf, Ld = 0.f;
-#pragma unroll
-        for (int hh = 0; hh < kMaxGroup; ++hh)
-          if (hh == h) {
-            Md = accM[hh];
-            Ld = accL[hh];
-          }
+        float Md, Ld;
+        head_ml(h, Md, Ld);
         const uint32_t dst = map_rank(recv_ml_u32 + 4u * ((split * kMaxGroup + h) * 2), peer);
         st_cluster_f32(dst, Md);
         st_cluster_f32(dst + 4u, Ld);
@@ -593,6 +681,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   }
 
   const bool single = (kMode == kModeTicket) && n_splits == 1;   // the full step always leaves its partials to the selector
+  float accL[kMaxGroup];
+#pragma unroll
+  for (int h = 0; h < kMaxGroup; ++h) {
+    accL[h] = 1.f;
+    float Mh;
+    if (single) head_ml(h, Mh, accL[h]);
+  }
   if (!single) {
     float* part = p.partials + ((int64_t)bg * p.max_splits + split) * PartialLayout::kFloats;
     if (!kScoreOnly) {
@@ -601,13 +696,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         if (h < G) part[h * kHeadDim + d] = accO[h];
     }
     if (d < kMaxGroup) {
-      float Md = ninf, Ld = 0.f;
-#pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h)
-        if (h == d) {
-          Md = accM[h];
-          Ld = accL[h];
-        }
+      float Md, Ld;
+      head_ml(d, Md, Ld);
       part[kMaxGroup * kHeadDim + d] = Md;
       part[kMaxGroup * kHeadDim + kMaxGroup + d] = Ld;
       if (kLogits && p.ml_t != nullptr) {   // the selection kernel reads these across the splits: keep a contiguous copy
@@ -653,7 +743,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
 }  // namespace
 
 static size_t ring_smem_bytes(int stages) {
-  return (size_t)stages * kStageBytes + 16 * stages + 16 + (size_t)kRecvFloats * sizeof(float) + 1024;
+  return (size_t)stages * kStageBytes + 16 * stages + 16 + (size_t)kRecvFloats * sizeof(float) +
+         (size_t)kMaxGroup * kQPad * 4 + 16 * 8 * sizeof(float) + 1024;   // ring, barriers, receive buffer, query, warp maxima
 }
 size_t attention_smem_bytes() { return ring_smem_bytes(kStages); }
 static size_t cluster_smem_bytes(bool wide) { return ring_smem_bytes(wide ? Ring<kModeCluster, true>::kStg : kStages); }

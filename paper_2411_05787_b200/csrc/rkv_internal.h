@@ -161,6 +161,24 @@ size_t select_smem_bytes(int keys_per_cta, int pool_half);
 int select_keys_cap(int keys_per_cta);
 constexpr int kSelectMaxKeysPerCtaPooled = 20480;   // with pooling a CTA keeps two key arrays
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map of one cache buffer ([n_rows][128] bf16) as the attention kernel reads it: a box is 64 rows of both
+// 64-channel halves, {channel 0..63, row, half}, so that ONE copy instruction lands a whole K (or V) tile in
+// shared memory as [half][row][64 channels] with the 128-byte swizzle - the layout the ldmatrix addressing
+// expects.  (The copy engine's cost per instruction is what makes one large box better than two small ones.)
+inline CUresult encode_cache_map(EncodeTiledFn encode, void* base, int64_t n_rows, CUtensorMap* out) {
+  const cuuint64_t dims[3] = {64, (cuuint64_t)n_rows, 2};
+  const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, 128};   // bytes: next row, next half
+  const cuuint32_t box[3] = {64, (cuuint32_t)kTile, 2};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 }  // namespace rkv
 
 struct rkv_ctx {

@@ -37,10 +37,7 @@ std::mutex g_mu;
 unsigned char* g_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
 bool g_device_ready[kMaxDevices] = {};
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode_na = nullptr;
+rkv::EncodeTiledFn g_encode_na = nullptr;
 
 rkv_status fail(char* err, size_t cap, rkv_status code, const char* fmt, const char* detail = "") {
   if (err != nullptr && cap > 0) snprintf(err, cap, fmt, detail);
@@ -66,22 +63,15 @@ rkv_status setup_device(int dev, char* err, size_t cap) {
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
     if (e != cudaSuccess || fn == nullptr || q != cudaDriverEntryPointSuccess)
       return fail(err, cap, RKV_ERR_CUDA, "cuTensorMapEncodeTiled is not available: %s", cudaGetErrorString(e));
-    g_encode_na = reinterpret_cast<EncodeTiledFn>(fn);
+    g_encode_na = reinterpret_cast<rkv::EncodeTiledFn>(fn);
   }
   g_scratch_addr[dev] = static_cast<unsigned char*>(addr);
   g_device_ready[dev] = true;
   return RKV_OK;
 }
 
-// [n_rows][128] bf16 viewed as 64-row x 64-channel boxes with the 128-byte swizzle (what the kernel expects)
 bool encode_map(void* base, int64_t n_rows, CUtensorMap* out) {
-  cuuint64_t dims[2] = {(cuuint64_t)rkv::kHeadDim, (cuuint64_t)n_rows};
-  cuuint64_t strides[1] = {(cuuint64_t)rkv::kHeadDim * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)rkv::kTile};
-  cuuint32_t estr[2] = {1, 1};
-  return g_encode_na(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return rkv::encode_cache_map(g_encode_na, base, n_rows, out) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -114,6 +104,8 @@ extern "C" rkv_status rkv_small_step_noalloc(const rkv_config* cfg, const void* 
       snprintf(err_msg, err_cap, "small-cache length bound %d exceeds RKV_NOALLOC_MAX_LEN = %d", n_max, kMaxLenNA);
     return RKV_ERR_UNSUPPORTED;
   }
+  if ((reinterpret_cast<uintptr_t>(q) & 15) != 0 || (reinterpret_cast<uintptr_t>(out) & 15) != 0)
+    return fail(err_msg, err_cap, RKV_ERR_INVALID_ARG, "q and out must start on a 16-byte boundary");
   const rkv_cache* c = small_cache;
   if (!c->k || !c->v || !c->row_offset || !c->cap || !c->len || c->n_rows <= 0 || c->n_rows >= (int64_t(1) << 31) ||
       (reinterpret_cast<uintptr_t>(c->k) & 15) != 0 || (reinterpret_cast<uintptr_t>(c->v) & 15) != 0)
