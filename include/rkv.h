@@ -291,10 +291,18 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
  *   RKV_OPT_DEPENDENT_LAUNCH  1 (default): kernels are launched with programmatic stream
  *                             serialisation so that a kernel's launch overlaps the tail of its
  *                             predecessor; 0: plain stream order.  Process-wide.
+ *   RKV_OPT_EARLY_CACHE_READ  1 (default): the clustered partial step may request its share of the
+ *                             attended cache before its stream dependency has resolved, when the
+ *                             library's previous launch on the same stream wrote no row of that
+ *                             cache (the library keeps a host-side record per stream; kernels of
+ *                             other origin complete before a kernel of this library starts, unless
+ *                             they themselves release their dependents early while still writing
+ *                             the cache - turn the option off in that case); 0: never.
  */
 #define RKV_OPT_SMALL_MIN_CHUNK 1
 #define RKV_OPT_DEPENDENT_LAUNCH 2
 #define RKV_OPT_SMALL_CLUSTER 3
+#define RKV_OPT_EARLY_CACHE_READ 4
 rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
 
 /*

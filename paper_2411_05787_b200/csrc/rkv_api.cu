@@ -196,6 +196,9 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.scale = ctx->cfg.softmax_scale;
   // without a mask: a cluster per head always has work; a streaming grid has when it serves a single sequence
   p.spec = (active == nullptr && (cluster || (logits && ctx->cfg.n_seq == 1))) ? 1 : 0;
+  // Early cache read: only when the call before this one on the stream leaves the attended cache alone (a
+  // gather or an append into it forbids it; so does an unknown history).
+  p.early = (cluster && p.spec != 0 && ctx->early_read && !rkv::last_call_wrote(st, cache)) ? 1 : 0;
   if (app != nullptr) {   // only the clustered partial step takes the append with it
     if (!cluster) return RKV_ERR_INVALID_ARG;
     p.k_new = app->k_new;
@@ -228,6 +231,7 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
   ctx->launches += 1;
+  rkv::note_call_writes(st, app != nullptr ? cache : nullptr, app != nullptr ? app->full : nullptr);
   return RKV_OK;
 }
 
@@ -235,7 +239,46 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
 
 namespace rkv {
 bool g_use_pdl = true;
+
+namespace {
+struct ByteRange { uintptr_t lo, hi; };
+std::mutex g_writes_mu;
+std::map<cudaStream_t, std::vector<ByteRange>> g_writes;   // per stream: what the last call wrote
+bool g_writes_lost = false;   // the record was dropped once: a stream without an entry is then unknown, not clean
+constexpr size_t kMaxTrackedStreams = 1024;
+void add_ranges(std::vector<ByteRange>* v, const rkv_cache* c) {
+  if (c == nullptr || c->k == nullptr || c->v == nullptr) return;
+  const uintptr_t bytes = (uintptr_t)c->n_rows * kHeadDim * 2;
+  v->push_back({reinterpret_cast<uintptr_t>(c->k), reinterpret_cast<uintptr_t>(c->k) + bytes});
+  v->push_back({reinterpret_cast<uintptr_t>(c->v), reinterpret_cast<uintptr_t>(c->v) + bytes});
 }
+}  // namespace
+
+void note_call_writes(cudaStream_t st, const rkv_cache* a, const rkv_cache* b) {
+  std::lock_guard<std::mutex> lock(g_writes_mu);
+  if (g_writes.size() >= kMaxTrackedStreams && g_writes.find(st) == g_writes.end()) {
+    g_writes.clear();
+    g_writes_lost = true;
+  }
+  std::vector<ByteRange>& v = g_writes[st];
+  v.clear();
+  add_ranges(&v, a);
+  add_ranges(&v, b);
+}
+
+bool last_call_wrote(cudaStream_t st, const rkv_cache* c) {
+  std::lock_guard<std::mutex> lock(g_writes_mu);
+  auto it = g_writes.find(st);
+  if (it == g_writes.end()) return g_writes_lost;   // never launched here: whatever runs before is not ours and
+                                                    // therefore complete before a kernel of ours starts
+  std::vector<ByteRange> mine;
+  add_ranges(&mine, c);
+  for (const ByteRange& w : it->second)
+    for (const ByteRange& r : mine)
+      if (w.lo < r.hi && r.lo < w.hi) return true;
+  return false;
+}
+}  // namespace rkv
 
 extern "C" {
 
@@ -260,6 +303,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->profiling = false;
   ctx->small_min_chunk = 256;
   ctx->small_cluster = 1;
+  ctx->early_read = 1;
   ctx->gp = ctx->group <= 4 ? 4 : 8;
   ctx->workspace = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
@@ -356,6 +400,7 @@ static rkv_status full_step_impl(rkv_ctx* ctx, const void* q, const rkv_cache* f
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
   ctx->launches += 1;
+  rkv::note_call_writes(st, nullptr, nullptr);
   return RKV_OK;
 }
 
@@ -386,6 +431,7 @@ rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "gather launch");
   ctx->launches += 1;
+  rkv::note_call_writes(static_cast<cudaStream_t>(stream), small_cache, nullptr);
   return RKV_OK;
 }
 
@@ -434,6 +480,7 @@ rkv_status rkv_gather_small_evict(rkv_ctx* ctx, const int32_t* topk_idx, const i
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "eviction-order launch");
   ctx->launches += 1;
+  rkv::note_call_writes(static_cast<cudaStream_t>(stream), nullptr, nullptr);
   return RKV_OK;
 }
 
@@ -467,6 +514,7 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const 
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "append launch");
   ctx->launches += 1;
+  rkv::note_call_writes(static_cast<cudaStream_t>(stream), full, small_cache);
   return RKV_OK;
 }
 
@@ -481,6 +529,7 @@ rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_las
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "trigger launch");
   ctx->launches += 1;
+  rkv::note_call_writes(static_cast<cudaStream_t>(stream), nullptr, nullptr);
   return RKV_OK;
 }
 
@@ -524,6 +573,9 @@ rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value) {
       return RKV_OK;
     case RKV_OPT_DEPENDENT_LAUNCH:
       rkv::g_use_pdl = value != 0;
+      return RKV_OK;
+    case RKV_OPT_EARLY_CACHE_READ:
+      ctx->early_read = value != 0;
       return RKV_OK;
     default:
       return RKV_ERR_INVALID_ARG;

@@ -83,16 +83,6 @@ __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* t
       "l"(tm), "r"(0), "r"(y), "r"(0), "r"(bar), "l"(policy)
       : "memory");
 }
-// Pulls one tile into L2 only.  L2 is the point of coherence, so this is safe while another kernel still writes
-// the rows: a later load sees whatever has been written by then.
-__device__ __forceinline__ void tma_prefetch_tile_l2(const CUtensorMap* tm, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tm), "r"(0), "r"(y),
-               "r"(0)
-               : "memory");
-}
-__device__ __forceinline__ void prefetch_l2(const void* ptr) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr) : "memory");
-}
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -144,8 +134,12 @@ __device__ __forceinline__ void st_shared_v2(uint32_t addr, uint2 v) {
 __device__ __forceinline__ void st_keep_f2(float* addr, float a, float b, uint64_t policy) {
   asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(addr), "f"(a), "f"(b), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+__device__ __forceinline__ void st_cluster_f32x4(uint32_t addr, float4 v) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+               : "memory");
+}
+__device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
 // Cluster barrier (all five warps of every CTA of the cluster arrive).
 __device__ __forceinline__ void cluster_sync_alive() {
@@ -191,7 +185,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
 
   const int b = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  pdl_launch();
   // shared memory: [stages][K lo | K hi | V lo | V hi], the barriers, then (cluster mode) the receive buffer
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -218,39 +211,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // stream predecessor is still running; everything else waits for the dependency.
   const int cap = __ldg(p.cap + b);
   const int64_t roff = __ldg(p.row_offset + b);
-  // A clustered step is short and usually sits at the dependency wait while its stream predecessor runs: use
-  // that time to bring this CTA's rows from DRAM into L2, so that the copies after the wait are L2 hits.
-  // The same goes for the few lines the step reads first (sizes, query, new rows): with many layers' caches
-  // streaming through L2 between two calls on one layer they have usually been evicted.
-  if (kCluster && warp == kMW) {
-    if (p.spec != 0 && lane == 0) {
-      const int n_pre = (p.chunk + kTile - 1) / kTile < kStg ? (p.chunk + kTile - 1) / kTile : kStg;   // = n_spec below
-      const int y0 = (int)(roff + (int64_t)g * cap + (int64_t)split * p.chunk);
-      for (int t = 0; t < n_pre; ++t) {
-        tma_prefetch_tile_l2(&tm_k, y0 + t * kTile);
-        tma_prefetch_tile_l2(&tm_v, y0 + t * kTile);
-      }
-    }
-    const int64_t nrow_b = ((int64_t)b * p.n_kv_heads + g) * kHeadDim * 2;   // byte offset of this head's new row
-    if (lane == 1) prefetch_l2(p.len + b);
-    if (lane == 2 && p.active != nullptr) prefetch_l2(p.active + b);
-    if (lane >= 3 && lane < 3 + 2 * G) prefetch_l2(qg + (lane - 3) * 64);   // 128-byte lines of the G query rows
-    if (kAppend) {
-      if (lane == 19 || lane == 20) prefetch_l2(static_cast<const uint8_t*>(p.k_new) + nrow_b + (lane - 19) * 128);
-      if (lane == 21 || lane == 22) prefetch_l2(static_cast<const uint8_t*>(p.v_new) + nrow_b + (lane - 21) * 128);
-      if (p.has_full) {
-        if (lane == 23) prefetch_l2(p.full_len + b);
-        if (lane == 24) prefetch_l2(p.full_cap + b);
-        if (lane == 25) prefetch_l2(p.full_row_offset + b);
-      }
-      if (p.evict_order != nullptr) {
-        if (lane == 26) prefetch_l2(p.k_small + b);
-        if (lane == 27) prefetch_l2(p.evict_count + b);
-      }
-    }
-  }
   __syncthreads();   // barrier initialisation (above) is visible to every warp
-  pdl_wait();
 
   // One tile = K (and V) rows [y, y + 64) into stage t % kStg, completion on that stage's barrier.
   auto issue_tile = [&](int t, int64_t row_first, uint64_t policy) {
@@ -261,19 +222,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     tma_load_tile(dst, &tm_k, y, bar, policy);
     if (!kScoreOnly) tma_load_tile(dst + 2 * kHalfBytes, &tm_v, y, bar, policy);
   };
-  // When the host knows that every CTA of the grid has work (no mask; one sequence, or a cluster per head), the
-  // chunk of this CTA follows from the launch geometry alone, so its first tiles are requested before the length
-  // has even been read (tiles past the length are waited for and ignored).  Saves one memory round trip.
-  int n_spec = 0;
-  if (p.spec != 0) {
-    n_spec = (p.chunk + kTile - 1) / kTile < kStg ? (p.chunk + kTile - 1) / kTile : kStg;
+  // Tiles requested ahead of the length (see below).  When the host has established that the launch before
+  // this one on the stream does not write this cache (p.early), they are requested even before the
+  // dependency wait: a clustered step usually sits at that wait while its predecessor runs, and a CTA's
+  // share of the cache takes longer to arrive (about 64 bytes per cycle per SM) than the rest of the step
+  // takes to get ready.  Every kernel of this library releases its dependents only after its own wait, so the
+  // predecessor is the only kernel that can still be running at that point.
+  auto issue_spec = [&](int n_tiles_spec) {
     if (tid == 32 * kMW) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
       const int64_t row_s = roff + (int64_t)g * cap + (int64_t)split * p.chunk;
-      for (int t = 0; t < n_spec; ++t) issue_tile(t, row_s, policy);
+      for (int t = 0; t < n_tiles_spec; ++t) issue_tile(t, row_s, policy);
     }
-  }
+  };
+  int n_spec = 0;
+  if (p.spec != 0) n_spec = (p.chunk + kTile - 1) / kTile < kStg ? (p.chunk + kTile - 1) / kTile : kStg;
+  if (kCluster && p.early != 0) issue_spec(n_spec);
+  pdl_wait();
+  pdl_launch();   // after the wait: at most one predecessor is ever in flight behind a kernel of this library
+  if (!(kCluster && p.early != 0)) issue_spec(n_spec);
+
+  // (When the host knows that every CTA of the grid has work - no mask; one sequence, or a cluster per head - the
+  // chunk of this CTA follows from the launch geometry alone, so its first tiles have been requested above, before
+  // the length has even been read; tiles past the length are waited for and ignored.)
 
   // per-sequence sizes and (MMA warps) the query fragments: independent loads, one round trip
   const int act = (p.active != nullptr) ? __ldcg(p.active + b) : 1;
@@ -615,17 +587,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   }
   consumer_bar();
 
-  const int d = tid;  // 0..127: one output channel per thread (further MMA warps only keep the barriers company)
-  const bool chan = d < kHeadDim;
-  float accO[kMaxGroup];
+  // The merged accumulators as items of (head, four channels): G * 32 items over the MMA threads.
+  constexpr int kNT = 32 * kMW;
+  constexpr int kIt = (kMaxGroup * 32 + kNT - 1) / kNT;
+  const int n_items = G * 32;
+  float4 acc4[kIt];
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) {
-    accO[h] = 0.f;
-    if (!chan || h >= G) continue;
-    float O = 0.f;
+  for (int it = 0; it < kIt; ++it) {
+    acc4[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int item = tid + it * kNT;
+    if (item < n_items) {
+      const float* src = sm_o + (item >> 5) * kOPad + (item & 31) * 4;
 #pragma unroll
-    for (int w = 0; w < kMW; ++w) O += sm_o[(w * 8 + h) * kOPad + d];
-    accO[h] = O;
+      for (int w = 0; w < kMW; ++w) {
+        const float4 v = *reinterpret_cast<const float4*>(src + w * 8 * kOPad);
+        acc4[it].x += v.x;
+        acc4[it].y += v.y;
+        acc4[it].z += v.z;
+        acc4[it].w += v.w;
+      }
+    }
   }
   // (m, l) of one head for the whole CTA; heads beyond the group read as (-inf, 0)
   auto head_ml = [&](int h, float& M, float& L) {
@@ -642,58 +623,95 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
 
   if (kCluster) {
     // ---------------------------------------------- merge the CTAs of the cluster through shared memory
-    const int C = (int)gridDim.x;                       // cluster size = CTAs per (sequence, KV head)
-    const int dchunk = kHeadDim / C;                    // channels of every head that one CTA finishes
+    const int C = (int)gridDim.x;                       // cluster size = CTAs per (sequence, KV head): 1, 2, 4 or 8
+    const int c_sh = __ffs(C) - 1;                      // C is a power of two: shifts instead of divisions below
+    const int dchunk = kHeadDim >> c_sh;                // channels of every head that one CTA finishes
     float* recv = reinterpret_cast<float*>(smem_gen + kStg * kStageBytes + 16 * kStg + 16);
     float* recv_ml = recv + kMaxGroup * kHeadDim;       // [source CTA][head][2]
     const uint32_t recv_u32 = smem_u32(recv), recv_ml_u32 = smem_u32(recv_ml);
-    if (chan) {
-      const int owner = d / dchunk, dd = d - owner * dchunk;
 #pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h)
-        if (h < G) st_cluster_f32(map_rank(recv_u32 + 4u * ((split * kMaxGroup + h) * dchunk + dd), owner), accO[h]);
-      if (d < kMaxGroup * C) {   // (m, l) of head d % 8 to peer d / 8
-        const int h = d & 7, peer = d >> 3;
-        float Md, Ld;
-        head_ml(h, Md, Ld);
-        const uint32_t dst = map_rank(recv_ml_u32 + 4u * ((split * kMaxGroup + h) * 2), peer);
-        st_cluster_f32(dst, Md);
-        st_cluster_f32(dst + 4u, Ld);
+    for (int it = 0; it < kIt; ++it) {
+      const int item = tid + it * kNT;
+      if (item < n_items) {   // four channels never straddle two owners: dchunk is a multiple of 16
+        const int h = item >> 5, d4 = (item & 31) * 4;
+        const int owner = d4 >> (7 - c_sh), dd = d4 & (dchunk - 1);
+        st_cluster_f32x4(map_rank(recv_u32 + 4u * ((split * kMaxGroup + h) * dchunk + dd), owner), acc4[it]);
       }
+    }
+    if (tid < kMaxGroup * C) {   // (m, l) of head tid % 8 to peer tid / 8
+      const int h = tid & 7, peer = tid >> 3;
+      float Md, Ld;
+      head_ml(h, Md, Ld);
+      st_cluster_f32x2(map_rank(recv_ml_u32 + 4u * ((split * kMaxGroup + h) * 2), peer), Md, Ld);
     }
     cluster_sync_alive();
     take_len_ticket();
     if (!ok) return;
-    for (int item = d; chan && item < G * dchunk; item += 128) {
-      const int h = item / dchunk, dd = item - h * dchunk;
-      float M = ninf;
-      for (int r = 0; r < C; ++r) M = fmaxf(M, recv_ml[(r * kMaxGroup + h) * 2]);
-      float L = 0.f, O = 0.f;
-      for (int r = 0; r < C; ++r) {
-        const float mr = recv_ml[(r * kMaxGroup + h) * 2];
-        const float e = (mr == ninf) ? 0.f : ex2((mr - M) * kLog2e);
-        L = fmaf(recv_ml[(r * kMaxGroup + h) * 2 + 1], e, L);
-        O = fmaf(recv[(r * kMaxGroup + h) * dchunk + dd], e, O);
+    // This CTA finishes dchunk channels of every head: G * dchunk / 4 items of four channels, and C adjacent
+    // lanes per item, one per source CTA, that combine through shuffles (G * 32 lanes in all, as above).
+    const int ph_sh = 5 - c_sh;             // log2 of the items per head, dchunk / 4
+#pragma unroll
+    for (int it = 0; it < kIt; ++it) {
+      const int j = tid + it * kNT;
+      if (j >= n_items) continue;          // whole warps: n_items is a multiple of 32
+      const int item = j >> c_sh, r = j & (C - 1);
+      const int h = item >> ph_sh, dd = (item & ((1 << ph_sh) - 1)) * 4;
+      const float2 ml = *reinterpret_cast<const float2*>(recv_ml + (r * kMaxGroup + h) * 2);
+      float4 v = *reinterpret_cast<const float4*>(recv + (r * kMaxGroup + h) * dchunk + dd);
+      float M = ml.x;
+      for (int sh = 1; sh < C; sh <<= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+      const float e = (ml.x == ninf) ? 0.f : ex2((ml.x - M) * kLog2e);
+      float L = ml.y * e;
+      v.x *= e;
+      v.y *= e;
+      v.z *= e;
+      v.w *= e;
+      for (int sh = 1; sh < C; sh <<= 1) {
+        L += __shfl_xor_sync(0xffffffffu, L, sh);
+        v.x += __shfl_xor_sync(0xffffffffu, v.x, sh);
+        v.y += __shfl_xor_sync(0xffffffffu, v.y, sh);
+        v.z += __shfl_xor_sync(0xffffffffu, v.z, sh);
+        v.w += __shfl_xor_sync(0xffffffffu, v.w, sh);
       }
-      out[h * kHeadDim + split * dchunk + dd] = __float2bfloat16(O / L);
+      if (r == 0) {
+        const float inv = __fdividef(1.f, L);
+        uint2 o2;
+        o2.x = pack_bf16(v.x * inv, v.y * inv);
+        o2.y = pack_bf16(v.z * inv, v.w * inv);
+        *reinterpret_cast<uint2*>(out + h * kHeadDim + split * dchunk + dd) = o2;
+      }
     }
     return;
   }
 
+  const int d = tid;   // the other forms run with four MMA warps: one thread per channel below
   const bool single = (kMode == kModeTicket) && n_splits == 1;   // the full step always leaves its partials to the selector
-  float accL[kMaxGroup];
+  if (single) {
+    if (!ok) return;
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) {
-    accL[h] = 1.f;
-    float Mh;
-    if (single) head_ml(h, Mh, accL[h]);
+    for (int it = 0; it < kIt; ++it) {
+      const int item = tid + it * kNT;
+      if (item < n_items) {
+        const int h = item >> 5, d4 = (item & 31) * 4;
+        float Mh, Lh;
+        head_ml(h, Mh, Lh);
+        const float inv = 1.f / Lh;
+        uint2 o2;
+        o2.x = pack_bf16(acc4[it].x * inv, acc4[it].y * inv);
+        o2.y = pack_bf16(acc4[it].z * inv, acc4[it].w * inv);
+        *reinterpret_cast<uint2*>(out + h * kHeadDim + d4) = o2;
+      }
+    }
+    return;
   }
-  if (!single) {
+  {
     float* part = p.partials + ((int64_t)bg * p.max_splits + split) * PartialLayout::kFloats;
     if (!kScoreOnly) {
 #pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h)
-        if (h < G) part[h * kHeadDim + d] = accO[h];
+      for (int it = 0; it < kIt; ++it) {
+        const int item = tid + it * kNT;
+        if (item < n_items) *reinterpret_cast<float4*>(part + (item >> 5) * kHeadDim + (item & 31) * 4) = acc4[it];
+      }
     }
     if (d < kMaxGroup) {
       float Md, Ld;
@@ -724,20 +742,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     auto bar = [] { consumer_bar_n<128>(); };
     fold_weights<128>(pbase, n_splits, tid, sm_w, sm_ML, bar);
     fold_out<128, kMaxGroup>(pbase, n_splits, 0, G, tid, sm_w, sm_red, bar);
-#pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h) {
-      if (h < G) {
-        accO[h] = sm_red[h * kHeadDim + d];
-        accL[h] = sm_ML[8 + h];
-      }
-    }
     if (tid == 0) p.tickets[bg] = 0;  // ready for the next call on this stream
-  }
-
-  if (!ok) return;
+    if (!ok) return;
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h)
-    if (h < G) out[h * kHeadDim + d] = __float2bfloat16(accO[h] / accL[h]);
+    for (int h = 0; h < kMaxGroup; ++h)
+      if (h < G) out[h * kHeadDim + d] = __float2bfloat16(sm_red[h * kHeadDim + d] / sm_ML[8 + h]);
+  }
 }
 
 }  // namespace

@@ -49,6 +49,7 @@ struct AttnParams {
   int32_t max_splits;
   int32_t max_len;            // clamp for len[b]
   int32_t spec;               // 1: every CTA has work by construction, first tiles may be requested before len is read
+  int32_t early;              // 1 (clustered step with spec): request them before the dependency wait as well
   float scale;
   // fused append (clustered partial step only): the new token's rows and where they go
   const void* k_new;          // bf16 [B][Hkv][128]
@@ -118,7 +119,10 @@ cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshol
                            float* sim, int n_seq, int n_q_heads, cudaStream_t st);
 // Launch with optional programmatic dependent launch (the kernel may start while its predecessor on
 // the stream drains; every kernel waits with pdl_wait() before touching global memory) and an
-// optional thread-block cluster along x.
+// optional thread-block cluster along x.  Every kernel calls pdl_launch() only AFTER its own pdl_wait():
+// a kernel can then begin no earlier than the moment its predecessor's own dependency has resolved, so at
+// most one earlier launch of this library is still running while a kernel executes the part above its wait.
+// The partial step's early cache read (AttnParams::early, last_call_wrote below) relies on exactly that.
 extern bool g_use_pdl;
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
@@ -153,6 +157,11 @@ inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
+
+// K/V buffers written by the library's most recent call on each stream (host-side record).  A call notes what
+// it writes; the partial step asks whether its stream predecessor wrote the cache it is about to read.
+void note_call_writes(cudaStream_t st, const rkv_cache* a, const rkv_cache* b);   // either may be NULL
+bool last_call_wrote(cudaStream_t st, const rkv_cache* c);
 
 cudaError_t prepare_attention();  // one-time function attributes (dynamic shared memory sizes)
 cudaError_t prepare_select();
@@ -200,6 +209,7 @@ struct rkv_ctx {
   int sm_count;
   int small_min_chunk;
   int small_cluster;   // 1: the partial step merges its splits inside a thread-block cluster when the length allows
+  int early_read;      // 1: the clustered partial step may request its cache rows before its dependency wait
   int gp;              // floats per position in the logit scratch
   std::string last_error;
   std::map<std::pair<uint64_t, int64_t>, CUtensorMap> tmaps;   // (base address, rows) -> tensor map

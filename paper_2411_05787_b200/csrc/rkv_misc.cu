@@ -14,8 +14,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const int32_t* __restrict__
                                                      const int32_t* __restrict__ active, int n_kv_heads,
                                                      int32_t* status) {
   const int b = blockIdx.z, g = blockIdx.y;
-  pdl_launch();
   pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
   if (active != nullptr && active[b] == 0) return;
   const int n = full.len[b];
   int m = k_small[b];
@@ -76,8 +76,8 @@ __global__ void __launch_bounds__(128) append_kernel(const uint4* __restrict__ k
                                                      CacheDev full, CacheDev small_cache, int has_full,
                                                      int has_small, int n_kv_heads, int32_t* status) {
   const int b = blockIdx.x, tid = threadIdx.x;
-  pdl_launch();
   pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
   int pos_f = -1, cap_f = 0, pos_s = -1, cap_s = 0;
   int64_t off_f = 0, off_s = 0;
   if (has_full) {
@@ -120,8 +120,8 @@ __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __res
                                                       const __nv_bfloat16* __restrict__ q_last, float threshold,
                                                       int32_t* flag, int32_t* keep, float* sim, int n_q_heads) {
   const int b = blockIdx.x, d = threadIdx.x;
-  pdl_launch();
   pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
   float a = 0.f, c = 0.f;
   for (int h = 0; h < n_q_heads; ++h) {
     a += __bfloat162float(q_now[((int64_t)b * n_q_heads + h) * kHeadDim + d]);
@@ -168,8 +168,8 @@ __global__ void __launch_bounds__(1024) evict_order_kernel(const uint32_t* __res
                                                            int32_t* evict_count, int max_evict, int n_kv_heads) {
   __shared__ unsigned long long sk[kEvictMaxK];
   const int b = blockIdx.y, g = blockIdx.x, tid = threadIdx.x;
-  pdl_launch();
   pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
   if (active != nullptr && active[b] == 0) return;
   int m = k_small[b];
   const int n = full_len[b];

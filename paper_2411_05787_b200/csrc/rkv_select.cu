@@ -190,7 +190,6 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
   const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   SelectShared* sh = reinterpret_cast<SelectShared*>(smem_raw);
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + ((sizeof(SelectShared) + 15) & ~size_t(15)));
-  pdl_launch();
   for (int i = tid; i < 2 * kHistWords; i += NT) (&sh->hist[0][0])[i] = 0u;
   if (tid == 0) {
     sh->cand_fill = 0u;
@@ -220,6 +219,7 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
   const int o_flat = rank * 16 * G + o_local;
   const int64_t hrow0 = ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
   pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
 
   // ---------------------------------------------------------------- 1: everything the kernel reads, in one round trip
   const int act = (p.active != nullptr) ? __ldcg(p.active + b) : 1;

@@ -246,6 +246,70 @@ def test_fused_append_small_step_equals_append_then_small_step(mods, n_small):
     assert fu_a.len.tolist() == [102, 43, 9] and sm_a.len.tolist() == [n_small + 3, n_small // 2 + 2, 8]
 
 
+def test_early_cache_read_changes_nothing(mods):
+    """The clustered partial step may request its cache rows before its stream dependency has resolved when the
+    launch before it wrote none of them.  A mix of calls where that is allowed (another cache's step before it)
+    and where it is not (the same cache's step, an append, a gather directly before it) must give the same bits as
+    the same calls with the option off, and match the oracle."""
+    rkv, runner, synth = mods
+    dev = torch.device("cuda")
+    n_q, n_kv, B, n0 = 32, 8, 1, 700
+    g = torch.Generator(device=dev); g.manual_seed(77)
+
+    def make(n_caches):
+        out = []
+        for _ in range(n_caches):
+            c = synth.alloc_cache([n0 + 40], [n0], n_kv, dev)
+            out.append(c)
+        return out
+    on, off = make(3), make(3)
+    for x, y in zip(on, off):
+        x.k.copy_(torch.randn(x.k.shape, generator=g, device=dev).to(torch.bfloat16))
+        x.v.copy_(torch.randn(x.v.shape, generator=g, device=dev).to(torch.bfloat16))
+        y.k.copy_(x.k); y.v.copy_(x.v)
+    ctx_on = rkv.Context(B, n_q, n_kv, n0 + 40, n0 + 40)
+    ctx_off = rkv.Context(B, n_q, n_kv, n0 + 40, n0 + 40)
+    ctx_off.set_option(rkv.OPT_EARLY_CACHE_READ, 0)
+    cs = lambda c: rkv.cache_struct(c.k, c.v, c.row_offset, c.cap, c.len)
+    order = [0, 1, 2, 0, 0, 1, 1, 2, 0, 2, 2, 1]          # neighbours equal: the predecessor wrote the same cache
+    outs = {}
+    for name, ctx, caches in (("on", ctx_on, on), ("off", ctx_off, off)):
+        gg = torch.Generator(device=dev); gg.manual_seed(78)
+        structs = [cs(c) for c in caches]
+        res = []
+        ins = [(torch.randn((B, n_q, 128), generator=gg, device=dev).to(torch.bfloat16),
+                torch.randn((B, n_kv, 128), generator=gg, device=dev).to(torch.bfloat16),
+                torch.randn((B, n_kv, 128), generator=gg, device=dev).to(torch.bfloat16),
+                torch.zeros((B, n_q, 128), dtype=torch.bfloat16, device=dev)) for _ in order]
+        torch.cuda.synchronize()
+        for step, i in enumerate(order):                   # nothing but the library's launches in the stream
+            q, kn, vn, o = ins[step]
+            if step % 5 == 4:                              # a plain append, then the step on the cache just written
+                ctx.append(kn, vn, None, structs[i])
+                ctx.small_step(q, structs[i], o)
+            else:
+                ctx.append_small_step(q, kn, vn, None, structs[i], o)
+            res.append((i, q, o))
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        outs[name] = res
+    for (i, q, a), (_, _, b) in zip(outs["on"], outs["off"]):
+        assert torch.equal(a, b)
+    for x, y in zip(on, off):
+        assert torch.equal(x.k, y.k) and torch.equal(x.v, y.v) and x.len.tolist() == y.len.tolist()
+    # the last step on every cache against the oracle, on the bytes now in the cache
+    seen = set()
+    for i, q, o in reversed(outs["on"]):
+        if i in seen:
+            continue
+        seen.add(i)
+        n = int(on[i].len[0])
+        k = O.bf16_bits_to_f64(host_heads(on[i], 0, n_kv, "k")[:, :n])
+        v = O.bf16_bits_to_f64(host_heads(on[i], 0, n_kv, "v")[:, :n])
+        want, _, _ = O.decode_attention(O.bf16_bits_to_f64(bits(q[0])), k, v)
+        check_out(o[0], want, f"cache {i}")
+
+
 @pytest.mark.parametrize("lens,k_small,n_q,n_kv", [([3000, 70], [300, 64], 32, 8), ([4096 + 37, 1], [512, 1], 28, 4)])
 def test_score_only_refresh_step(mods, lens, k_small, n_q, n_kv):
     """rkv_score_step (K only) selects exactly what rkv_full_step selects; followed by the rebuild and a partial
