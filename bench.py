@@ -51,6 +51,9 @@ def parse_args():
     ap.add_argument("--small-min-chunk", type=int, default=0, help="override rkv_small_step chunking (0: library default)")
     ap.add_argument("--no-dependent-launch", action="store_true", help="plain stream order between kernels")
     ap.add_argument("--no-small-cluster", action="store_true", help="merge partial-step splits through the workspace")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="full-step tokens run every layer's attention, selection and rebuild in one stream order "
+                         "(default: a layer's selection and rebuild overlap the next layer's attention)")
     return ap.parse_args()
 
 
@@ -260,13 +263,18 @@ def run_ours(args):
     # a sequence that never refreshes keeps growing its small cache (dynamic schedule); fixed: at most S - 1 rows
     small_extra = (total_tokens + 2) if dynamic else (S + 2)
     small_hint = k_max + small_extra
-    ctx = rkv.Context(B, Hq, Hkv, full_hint, small_hint)
-    if args.small_min_chunk:
-        ctx.set_option(rkv.OPT_SMALL_MIN_CHUNK, args.small_min_chunk)
-    if args.no_dependent_launch:
-        ctx.set_option(rkv.OPT_DEPENDENT_LAUNCH, 0)
-    if args.no_small_cluster:
-        ctx.set_option(rkv.OPT_SMALL_CLUSTER, 0)
+    # Two contexts, alternate layers: a context's workspace holds one full step's logits, and a layer's selection
+    # may still be reading them while the next layer's attention runs (see token("full") below).
+    ctxs = [rkv.Context(B, Hq, Hkv, full_hint, small_hint) for _ in range(2)]
+    ctx = ctxs[0]
+    for c in ctxs:
+        if args.small_min_chunk:
+            c.set_option(rkv.OPT_SMALL_MIN_CHUNK, args.small_min_chunk)
+        if args.no_dependent_launch:
+            c.set_option(rkv.OPT_DEPENDENT_LAUNCH, 0)
+        if args.no_small_cluster:
+            c.set_option(rkv.OPT_SMALL_CLUSTER, 0)
+    launch_total = lambda: sum(c.launch_count for c in ctxs)
 
     # per-token inputs: one contiguous block per token = all layers' q, then all k_new, then all v_new, so that
     # one copy stages a token and the calls get contiguous views.  Queries follow the workload's AR(1) process
@@ -296,14 +304,42 @@ def run_ours(args):
     for l in range(NL):
         cache = synth.fill_layer(wl, l, dev)
         synth.plant_heavy(w, cache, l, q_stage[l])
-        st = runner.LayerState(ctx, cache, list(w.k_small), small_extra, Hq, Hkv)
+        st = runner.LayerState(ctxs[l % 2], cache, list(w.k_small), small_extra, Hq, Hkv)
         st.out = outs[l].view(B, Hq, 128)
         layers.append(st)
 
+    overlap = not args.no_overlap
+    stream2 = torch.cuda.Stream(priority=-1)
+    ev_attn = [torch.cuda.Event() for _ in range(NL)]
+    ev_sel = [torch.cuda.Event() for _ in range(NL)]
+
+    def full_token_overlapped():
+        """Full-step token, layers in order.  What the next layer needs from a layer is its attention output, which
+        is final when rkv_full_attention's kernel ends; the layer's selection and the rebuild of its small cache
+        (first read by the NEXT token) are off that path.  The attention passes of all layers follow each other
+        in the main stream; each layer's selection and rebuild run in a second stream behind its attention and
+        overlap the next layers' attention (the contexts alternate, so a workspace is reused only after the
+        selection that reads it has ended)."""
+        main = torch.cuda.current_stream()
+        for l, st in enumerate(layers):
+            if l >= 2:
+                main.wait_event(ev_sel[l - 2])
+            st.append(k_stage[l], v_stage[l])
+            st.refresh_attention(q_stage[l], max_len_hint=full_hint)
+            ev_attn[l].record(main)
+            stream2.wait_event(ev_attn[l])
+            with torch.cuda.stream(stream2):
+                st.refresh_select(q_stage[l])
+                ev_sel[l].record(stream2)
+        for l in range(max(NL - 2, 0), NL):
+            main.wait_event(ev_sel[l])
+
     def token(kind: str):
+        if kind == "full" and overlap:
+            return full_token_overlapped()
         for l, st in enumerate(layers):
             q, kn, vn = q_stage[l], k_stage[l], v_stage[l]
-            if kind == "full":
+            if kind in ("full", "full_seq"):
                 st.append(kn, vn)
                 st.refresh(q, max_len_hint=full_hint)
             elif kind == "score":      # score-only refresh: K-only pass + top-K, rebuild, attention over the new small cache
@@ -320,7 +356,7 @@ def run_ours(args):
     # initial small caches + eager warm-up of every kernel (also creates the tensor maps)
     for l, st in enumerate(layers):
         st.refresh(q_stage[l], max_len_hint=full_hint)
-    kinds = ["small", "full", "score"] + (["check"] if dynamic else [])
+    kinds = ["small", "full", "score"] + (["full_seq"] if overlap else []) + (["check"] if dynamic else [])
     for kind in kinds:
         token(kind)
     torch.cuda.synchronize()
@@ -330,11 +366,11 @@ def run_ours(args):
     graphs, launches_per = {}, {}
     for kind in kinds:
         gr = torch.cuda.CUDAGraph()
-        before = ctx.launch_count
+        before = launch_total()
         with torch.cuda.stream(side):
             with torch.cuda.graph(gr, stream=side):
                 token(kind)
-        launches_per[kind] = ctx.launch_count - before
+        launches_per[kind] = launch_total() - before
         graphs[kind] = gr
     torch.cuda.synchronize()
 
@@ -404,6 +440,7 @@ def run_ours(args):
     ms_full, _ = timed(20, always_full=True)
     full_token_us = ms_full * 1000.0 / (20 * world)
     ms_score, _ = timed(20, force_kind="score")    # every token refreshes from scores alone (K half of the cache)
+    ms_full_seq = timed(20, force_kind="full_seq")[0] if overlap else ms_full   # the same work in one stream order
     run_tokens(1, always_full=True)
     ms_small, _ = timed(S - 1, force_small=True)   # right after a full token: K .. K+S-2 rows
     run_tokens(1, always_full=True)
@@ -411,17 +448,24 @@ def run_ours(args):
     # two periods, every sequence active).  A spin kernel first keeps the GPU busy while the host enqueues, so
     # that the launches sit back to back in the queue and an event pair measures the kernel, not the host.
     torch.cuda.synchronize()
-    ctx.set_profiling(True)
-    ctx.get_profile()
+    for c in ctxs:
+        c.set_profiling(True)
+        c.get_profile()
     torch.cuda._sleep(int(8e7))
     for i in range(n_prof):
         t = tok_counter[0]; tok_counter[0] += 1
         stage.copy_(inputs_dev[t % n_in])
-        token("full" if i % S == 0 else "small")
+        token("full_seq" if i % S == 0 else "small")
     torch.cuda.synchronize()
-    prof = ctx.get_profile()
-    ctx.set_profiling(False)
-    status = ctx.device_status()
+    prof = {}
+    for c in ctxs:
+        for name, (us, n) in c.get_profile().items():
+            us0, n0 = prof.get(name, (0.0, 0))
+            prof[name] = (us0 + us, n0 + n)
+        c.set_profiling(False)
+    status = 0
+    for c in ctxs:
+        status |= c.device_status()
 
     if rank != 0:
         if world > 1:
@@ -472,8 +516,12 @@ def run_ours(args):
             "small_step_frac_of_8TBs": kv_bytes_small / (small_us * 1e-6) / 8e12,
             "attn_full_frac_of_8TBs": achieved / 8000.0,
             "in_graph_us_per_layer": {"full_token": full_token_us / NL,
+                                      "full_token_one_stream": ms_full_seq * 1000.0 / (20 * world) / NL,
                                       "score_only_refresh_token": ms_score * 1000.0 / (20 * world) / NL,
                                       "small_token": ms_small * 1000.0 / ((S - 1) * world) / NL},
+            "full_token_schedule": ("two streams: the layers' attention passes follow each other; a layer's selection "
+                                    "and small-cache rebuild run behind its attention in a second stream" if overlap
+                                    else "one stream"),
             "device_status": status,
             "graph_launches": launches_per,
         },

@@ -129,6 +129,28 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*ho
                          void* q_last_full, int32_t max_len_hint, void* stream);
 
 /*
+ * The two halves of rkv_full_step as calls of their own (Sec. 2.1: the full step's attention output is
+ * what the decoder needs next; the refreshed partial cache is first read by the NEXT token's partial
+ * step).  A caller that wants the attention output early - and the selection and the rebuild of C_p
+ * off the layer's critical path, e.g. on a second stream under the next layer's work - calls
+ *   rkv_full_attention   attention over C_f: out is complete when this call's one kernel ends; the
+ *                        logits and softmax statistics stay in the context's workspace;
+ *   rkv_select_topk      scores, topk_idx, q_last_full from that workspace (same values as
+ *                        rkv_full_step; out differs from rkv_full_step's by summation order only).
+ * rkv_select_topk completes the LAST rkv_full_attention of the same context and must be given the same
+ * cache and mask (otherwise RKV_ERR_INVALID_ARG; also when there is no attention pass to complete).  The
+ * workspace holds one pass: no other rkv_full_step / rkv_score_step / rkv_full_attention on this
+ * context may run between the two (stream order, or an event, must put them after rkv_select_topk);
+ * callers that overlap the halves of consecutive layers use one context per layer in flight.
+ * Arguments as in rkv_full_step; q may be NULL in rkv_select_topk when q_last_full is.
+ */
+rkv_status rkv_full_attention(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
+                              const int32_t* active, void* out, int32_t max_len_hint, void* stream);
+rkv_status rkv_select_topk(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
+                           const int32_t* k_small, int32_t k_max, const int32_t* active, float* scores,
+                           int64_t score_stride, int32_t* topk_idx, void* q_last_full, void* stream);
+
+/*
  * Score-only refresh step (Sec. 4.2 "Impact of full attention steps", the "w/o full attention" setting:
  * at the stride the attention scores over the entire cache update the partial cache, and the step then
  * attends to the UPDATED partial cache instead of the full one; the paper reports the same quality as

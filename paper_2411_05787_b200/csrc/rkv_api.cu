@@ -154,7 +154,7 @@ bool cluster_eligible(const rkv_ctx* ctx, int n_max) { return ctx->small_cluster
 
 rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
                          int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out, int* gx_out,
-                         const AppendArgs* app = nullptr, bool score_only = false) {
+                         const AppendArgs* app = nullptr, bool score_only = false, bool fold_out = false) {
   if (!aligned16(q) || !aligned16(out) || (app != nullptr && (!aligned16(app->k_new) || !aligned16(app->v_new))))
     return RKV_ERR_INVALID_ARG;   // the kernels read and write these 16 bytes at a time
   CUtensorMap tm_k, tm_v;
@@ -196,9 +196,10 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.scale = ctx->cfg.softmax_scale;
   // without a mask: a cluster per head always has work; a streaming grid has when it serves a single sequence
   p.spec = (active == nullptr && (cluster || (logits && ctx->cfg.n_seq == 1))) ? 1 : 0;
-  // Early cache read: only when the call before this one on the stream leaves the attended cache alone (a
+  p.fold_out = (logits && !score_only && fold_out) ? 1 : 0;
+  // Early cache read: only when the launch before this one on the stream leaves the attended cache alone (a
   // gather or an append into it forbids it; so does an unknown history).
-  p.early = (cluster && p.spec != 0 && ctx->early_read && !rkv::last_call_wrote(st, cache)) ? 1 : 0;
+  p.early = (cluster && p.spec != 0 && ctx->early_read && rkv::early_read_safe(st, cache)) ? 1 : 0;
   if (app != nullptr) {   // only the clustered partial step takes the append with it
     if (!cluster) return RKV_ERR_INVALID_ARG;
     p.k_new = app->k_new;
@@ -231,7 +232,7 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
   ctx->launches += 1;
-  rkv::note_call_writes(st, app != nullptr ? cache : nullptr, app != nullptr ? app->full : nullptr);
+  rkv::note_launch(st, app != nullptr ? cache : nullptr, app != nullptr ? app->full : nullptr);
   return RKV_OK;
 }
 
@@ -243,7 +244,8 @@ bool g_use_pdl = true;
 namespace {
 struct ByteRange { uintptr_t lo, hi; };
 std::mutex g_writes_mu;
-std::map<cudaStream_t, std::vector<ByteRange>> g_writes;   // per stream: what the last call wrote
+struct LastLaunch { std::vector<ByteRange> writes; };
+std::map<cudaStream_t, LastLaunch> g_writes;   // per stream: the library's last launch
 bool g_writes_lost = false;   // the record was dropped once: a stream without an entry is then unknown, not clean
 constexpr size_t kMaxTrackedStreams = 1024;
 void add_ranges(std::vector<ByteRange>* v, const rkv_cache* c) {
@@ -254,29 +256,29 @@ void add_ranges(std::vector<ByteRange>* v, const rkv_cache* c) {
 }
 }  // namespace
 
-void note_call_writes(cudaStream_t st, const rkv_cache* a, const rkv_cache* b) {
+void note_launch(cudaStream_t st, const rkv_cache* a, const rkv_cache* b) {
   std::lock_guard<std::mutex> lock(g_writes_mu);
   if (g_writes.size() >= kMaxTrackedStreams && g_writes.find(st) == g_writes.end()) {
     g_writes.clear();
     g_writes_lost = true;
   }
-  std::vector<ByteRange>& v = g_writes[st];
-  v.clear();
-  add_ranges(&v, a);
-  add_ranges(&v, b);
+  LastLaunch& v = g_writes[st];
+  v.writes.clear();
+  add_ranges(&v.writes, a);
+  add_ranges(&v.writes, b);
 }
 
-bool last_call_wrote(cudaStream_t st, const rkv_cache* c) {
+bool early_read_safe(cudaStream_t st, const rkv_cache* c) {
   std::lock_guard<std::mutex> lock(g_writes_mu);
   auto it = g_writes.find(st);
-  if (it == g_writes.end()) return g_writes_lost;   // never launched here: whatever runs before is not ours and
-                                                    // therefore complete before a kernel of ours starts
+  if (it == g_writes.end()) return !g_writes_lost;   // never launched here: whatever runs before is not ours and
+                                                     // therefore complete before a kernel of ours starts
   std::vector<ByteRange> mine;
   add_ranges(&mine, c);
-  for (const ByteRange& w : it->second)
+  for (const ByteRange& w : it->second.writes)
     for (const ByteRange& r : mine)
-      if (w.lo < r.hi && r.lo < w.hi) return true;
-  return false;
+      if (w.lo < r.hi && r.lo < w.hi) return false;
+  return true;
 }
 }  // namespace rkv
 
@@ -347,19 +349,34 @@ rkv_status rkv_destroy(rkv_ctx* ctx) {
   return e == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 
-static rkv_status full_step_impl(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small,
-                                 int32_t k_max, const int32_t* active, void* out, float* scores, int64_t score_stride,
-                                 int32_t* topk_idx, void* q_last_full, int32_t max_len_hint, void* stream,
-                                 bool score_only) {
-  if (!ctx || !q || !cache_ok(full) || !k_small || (!out && !score_only) || !topk_idx) return RKV_ERR_INVALID_ARG;
-  if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+// First half of the full step: attention over the full cache, logits and softmax statistics to the workspace.
+// fold_out: the attention kernel also finishes out (otherwise the selection kernel does).
+static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* active,
+                                      void* out, int32_t max_len_hint, cudaStream_t st, bool score_only,
+                                      bool fold_out) {
+  if (!ctx || !q || !cache_ok(full) || (!out && !score_only)) return RKV_ERR_INVALID_ARG;
   int n_max = max_len_hint == 0 ? ctx->cfg.max_len : max_len_hint;
   if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
-  if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   int chunk = 0, gx = 1;
-  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, nullptr, score_only);
+  ctx->pending_full.valid = false;
+  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, nullptr, score_only,
+                               fold_out);
   if (s != RKV_OK) return s;
+  ctx->pending_full = {true, chunk, gx, n_max, full->k, active};
+  return RKV_OK;
+}
+
+// Second half: scores and top-K from what the first half left in the workspace; folds out unless it is NULL.
+static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small,
+                              int32_t k_max, const int32_t* active, void* out, float* scores, int64_t score_stride,
+                              int32_t* topk_idx, void* q_last_full, cudaStream_t st) {
+  if (!ctx || !cache_ok(full) || !k_small || !topk_idx || (q_last_full != nullptr && q == nullptr))
+    return RKV_ERR_INVALID_ARG;
+  if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+  if (!ctx->pending_full.valid) return RKV_ERR_INVALID_ARG;   // no attention pass to take the logits from
+  const int n_max = ctx->pending_full.n_max, chunk = ctx->pending_full.chunk, gx = ctx->pending_full.gx;
+  if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
+  ctx->pending_full.valid = false;
   SelectParams sp;
   memset(&sp, 0, sizeof(sp));
   sp.logits = ctx->logits;
@@ -400,8 +417,24 @@ static rkv_status full_step_impl(rkv_ctx* ctx, const void* q, const rkv_cache* f
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
   ctx->launches += 1;
-  rkv::note_call_writes(st, nullptr, nullptr);
+  rkv::note_launch(st, nullptr, nullptr);
   return RKV_OK;
+}
+
+static rkv_status full_step_impl(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small,
+                                 int32_t k_max, const int32_t* active, void* out, float* scores, int64_t score_stride,
+                                 int32_t* topk_idx, void* q_last_full, int32_t max_len_hint, void* stream,
+                                 bool score_only) {
+  // everything the second half would reject is rejected before the first half launches
+  if (!ctx || !q || !cache_ok(full) || !k_small || (!out && !score_only) || !topk_idx) return RKV_ERR_INVALID_ARG;
+  if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
+  const int n_max = max_len_hint == 0 ? ctx->cfg.max_len : max_len_hint;
+  if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
+  if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rkv_status s = full_attention_part(ctx, q, full, active, out, max_len_hint, st, score_only, false);
+  if (s != RKV_OK) return s;
+  return select_part(ctx, q, full, k_small, k_max, active, out, scores, score_stride, topk_idx, q_last_full, st);
 }
 
 rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
@@ -418,6 +451,21 @@ rkv_status rkv_score_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, co
                         max_len_hint, stream, true);
 }
 
+rkv_status rkv_full_attention(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* active, void* out,
+                              int32_t max_len_hint, void* stream) {
+  return full_attention_part(ctx, q, full, active, out, max_len_hint, static_cast<cudaStream_t>(stream), false, true);
+}
+
+rkv_status rkv_select_topk(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
+                           const int32_t* active, float* scores, int64_t score_stride, int32_t* topk_idx,
+                           void* q_last_full, void* stream) {
+  if (ctx != nullptr && ctx->pending_full.valid && full != nullptr &&
+      (ctx->pending_full.full_k != full->k || ctx->pending_full.active != active))
+    return RKV_ERR_INVALID_ARG;   // not the cache / mask of the attention pass it completes
+  return select_part(ctx, q, full, k_small, k_max, active, nullptr, scores, score_stride, topk_idx, q_last_full,
+                     static_cast<cudaStream_t>(stream));
+}
+
 rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t* k_small, int32_t k_max,
                             const rkv_cache* full, const rkv_cache* small_cache, const int32_t* active,
                             void* stream) {
@@ -431,7 +479,7 @@ rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "gather launch");
   ctx->launches += 1;
-  rkv::note_call_writes(static_cast<cudaStream_t>(stream), small_cache, nullptr);
+  rkv::note_launch(static_cast<cudaStream_t>(stream), small_cache, nullptr);
   return RKV_OK;
 }
 
@@ -480,7 +528,7 @@ rkv_status rkv_gather_small_evict(rkv_ctx* ctx, const int32_t* topk_idx, const i
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "eviction-order launch");
   ctx->launches += 1;
-  rkv::note_call_writes(static_cast<cudaStream_t>(stream), nullptr, nullptr);
+  rkv::note_launch(static_cast<cudaStream_t>(stream), nullptr, nullptr);
   return RKV_OK;
 }
 
@@ -514,7 +562,7 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const 
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "append launch");
   ctx->launches += 1;
-  rkv::note_call_writes(static_cast<cudaStream_t>(stream), full, small_cache);
+  rkv::note_launch(static_cast<cudaStream_t>(stream), full, small_cache);
   return RKV_OK;
 }
 
@@ -529,7 +577,7 @@ rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_las
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "trigger launch");
   ctx->launches += 1;
-  rkv::note_call_writes(static_cast<cudaStream_t>(stream), nullptr, nullptr);
+  rkv::note_launch(static_cast<cudaStream_t>(stream), nullptr, nullptr);
   return RKV_OK;
 }
 

@@ -50,6 +50,7 @@ struct AttnParams {
   int32_t max_len;            // clamp for len[b]
   int32_t spec;               // 1: every CTA has work by construction, first tiles may be requested before len is read
   int32_t early;              // 1 (clustered step with spec): request them before the dependency wait as well
+  int32_t fold_out;           // full step: 1 = the last CTA of each (sequence, KV head) folds the partials and writes out
   float scale;
   // fused append (clustered partial step only): the new token's rows and where they go
   const void* k_new;          // bf16 [B][Hkv][128]
@@ -122,7 +123,9 @@ cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshol
 // optional thread-block cluster along x.  Every kernel calls pdl_launch() only AFTER its own pdl_wait():
 // a kernel can then begin no earlier than the moment its predecessor's own dependency has resolved, so at
 // most one earlier launch of this library is still running while a kernel executes the part above its wait.
-// The partial step's early cache read (AttnParams::early, last_call_wrote below) relies on exactly that.
+// The partial step's early cache read (AttnParams::early, early_read_safe below) relies on exactly that.
+// (Releasing at the top would also let an attention kernel's CTAs occupy every SM while its predecessor
+// drains, shutting out work that another stream wants to run beside it.)
 extern bool g_use_pdl;
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
@@ -158,10 +161,12 @@ __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.laun
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
-// K/V buffers written by the library's most recent call on each stream (host-side record).  A call notes what
-// it writes; the partial step asks whether its stream predecessor wrote the cache it is about to read.
-void note_call_writes(cudaStream_t st, const rkv_cache* a, const rkv_cache* b);   // either may be NULL
-bool last_call_wrote(cudaStream_t st, const rkv_cache* c);
+// The library's most recent launch on each stream (host-side record): the K/V buffers it writes (either may be
+// NULL).  early_read_safe: the launch before this one on the stream writes no row of cache c, or nothing of
+// this library was ever launched on the stream (kernels of other origin complete before a kernel of this
+// library starts).
+void note_launch(cudaStream_t st, const rkv_cache* a, const rkv_cache* b);
+bool early_read_safe(cudaStream_t st, const rkv_cache* c);
 
 cudaError_t prepare_attention();  // one-time function attributes (dynamic shared memory sizes)
 cudaError_t prepare_select();
@@ -210,6 +215,8 @@ struct rkv_ctx {
   int small_min_chunk;
   int small_cluster;   // 1: the partial step merges its splits inside a thread-block cluster when the length allows
   int early_read;      // 1: the clustered partial step may request its cache rows before its dependency wait
+  // geometry of the last rkv_full_attention, for the rkv_select_topk that completes it
+  struct { bool valid; int chunk, gx, n_max; const void* full_k; const int32_t* active; } pending_full;
   int gp;              // floats per position in the logit scratch
   std::string last_error;
   std::map<std::pair<uint64_t, int64_t>, CUtensorMap> tmaps;   // (base address, rows) -> tensor map

@@ -158,6 +158,6 @@ extern "C" rkv_status rkv_small_step_noalloc(const rkv_config* cfg, const void* 
   p.scale = cfg->softmax_scale == 0.f ? 1.0f / sqrtf((float)cfg->head_dim) : cfg->softmax_scale;
   e = rkv::launch_attention(p, tm_k, tm_v, cfg->n_seq, grid_x, false, st);
   if (e != cudaSuccess) return fail(err_msg, err_cap, RKV_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
-  rkv::note_call_writes(st, nullptr, nullptr);   // host-side record only: this launch writes no cache rows
+  rkv::note_launch(st, nullptr, nullptr);   // host-side record only: this launch writes no cache rows
   return RKV_OK;
 }

@@ -63,6 +63,18 @@ class LayerState:
         self.ctx.gather_small(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c, active=active)
         return self.out
 
+    def refresh_attention(self, q, active=None, max_len_hint=0, stream=None):
+        """First half of a refresh: attention over the full cache; out is final when this call's kernel ends."""
+        self.ctx.full_attention(q, self.full_c, self.out, active=active, max_len_hint=max_len_hint, stream=stream)
+        return self.out
+
+    def refresh_select(self, q, active=None, stream=None):
+        """Second half: scores, top-K and the rebuild of the small cache from what refresh_attention left."""
+        self.ctx.select_topk(q, self.full_c, self.k_small, self.k_max, self.topk_idx, active=active,
+                             scores=self.scores, q_last_full=self.q_last_full, stream=stream)
+        self.ctx.gather_small(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c, active=active,
+                              stream=stream)
+
     def refresh_scores_only(self, q, active=None, max_len_hint=0, small_hint=0):
         """Score-only refresh: scores and top-K from K alone, rebuild of the small cache, attention over the new one."""
         self.ctx.score_step(q, self.full_c, self.k_small, self.k_max, self.topk_idx, active=active, scores=self.scores,

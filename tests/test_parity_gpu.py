@@ -124,6 +124,44 @@ def test_full_step_matches_oracle(mods, lens, k_small, n_q, n_kv):
                 assert np.array_equal(small_h[g, :take], full_h[g, idx_host[b, g, :take]])
 
 
+@pytest.mark.parametrize("lens,k_small,n_q,n_kv", CASES)
+def test_full_step_in_two_halves_matches_oracle(mods, lens, k_small, n_q, n_kv):
+    """rkv_full_attention + rkv_select_topk (+ gather): the attention kernel finishes out itself, the selection
+    works from the workspace.  Same checks as the one-call full step, and the same indices and scores as it."""
+    rkv, runner, synth = mods
+    ctx, st, cache, q = make_layer(mods, lens, k_small, n_q, n_kv, seed=len(lens) * 131 + n_q, poison=True)
+    st.out.fill_(7.0)
+    st.refresh_attention(q)
+    torch.cuda.synchronize()
+    for b, n in enumerate(lens):          # out is final before the selection has run
+        want = oracle_full(cache, b, n, q[b], n_kv, k_small[b])[0]
+        check_out(st.out[b], want, f"attention half, seq {b}")
+    st.refresh_select(q)
+    assert ctx.device_status() == 0
+    check_full_against_oracle(st, cache, q, lens, k_small, n_kv)
+    idx_two, scores_two = st.topk_idx.clone(), st.scores.clone()
+    small_k = st.small.k.clone()
+    st.refresh(q)
+    assert torch.equal(idx_two, st.topk_idx) and torch.equal(scores_two, st.scores) and torch.equal(small_k, st.small.k)
+    assert torch.equal(st.q_last_full, q)
+
+
+def test_select_topk_needs_its_attention_pass(mods):
+    rkv, runner, synth = mods
+    ctx, st, cache, q = make_layer(mods, [300], [16], 8, 2)
+    with pytest.raises(rkv.RkvError):
+        st.refresh_select(q)                          # nothing to complete
+    st.refresh_attention(q)
+    other = synth.alloc_cache([310], [300], 2, torch.device("cuda"))
+    with pytest.raises(rkv.RkvError):                 # another cache than the attention pass read
+        ctx.select_topk(q, rkv.cache_struct(other.k, other.v, other.row_offset, other.cap, other.len), st.k_small,
+                        st.k_max, st.topk_idx)
+    st.refresh_select(q)                              # the right one still works
+    with pytest.raises(rkv.RkvError):
+        st.refresh_select(q)                          # and is used up
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("agg,name", [(1, "mean"), (2, "first")])
 def test_aggregation_modes(mods, agg, name):
     lens, k_small = [500, 129], [50, 20]
