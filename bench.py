@@ -309,34 +309,14 @@ def run_ours(args):
         layers.append(st)
 
     overlap = not args.no_overlap
-    stream2 = torch.cuda.Stream(priority=-1)
-    ev_attn = [torch.cuda.Event() for _ in range(NL)]
-    ev_sel = [torch.cuda.Event() for _ in range(NL)]
-
-    def full_token_overlapped():
-        """Full-step token, layers in order.  What the next layer needs from a layer is its attention output, which
-        is final when rkv_full_attention's kernel ends; the layer's selection and the rebuild of its small cache
-        (first read by the NEXT token) are off that path.  The attention passes of all layers follow each other
-        in the main stream; each layer's selection and rebuild run in a second stream behind its attention and
-        overlap the next layers' attention (the contexts alternate, so a workspace is reused only after the
-        selection that reads it has ended)."""
-        main = torch.cuda.current_stream()
-        for l, st in enumerate(layers):
-            if l >= 2:
-                main.wait_event(ev_sel[l - 2])
-            st.append(k_stage[l], v_stage[l])
-            st.refresh_attention(q_stage[l], max_len_hint=full_hint)
-            ev_attn[l].record(main)
-            stream2.wait_event(ev_attn[l])
-            with torch.cuda.stream(stream2):
-                st.refresh_select(q_stage[l])
-                ev_sel[l].record(stream2)
-        for l in range(max(NL - 2, 0), NL):
-            main.wait_event(ev_sel[l])
+    overlapped = runner.OverlappedRefresh(layers) if overlap and NL > 1 else None
+    overlap = overlapped is not None
 
     def token(kind: str):
         if kind == "full" and overlap:
-            return full_token_overlapped()
+            # every layer's attention in this stream; its selection and rebuild behind it in a second one
+            return overlapped.run(lambda l: q_stage[l], lambda l: k_stage[l], lambda l: v_stage[l],
+                                  max_len_hint=full_hint)
         for l, st in enumerate(layers):
             q, kn, vn = q_stage[l], k_stage[l], v_stage[l]
             if kind in ("full", "full_seq"):

@@ -134,10 +134,11 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*ho
  * step).  A caller that wants the attention output early - and the selection and the rebuild of C_p
  * off the layer's critical path, e.g. on a second stream under the next layer's work - calls
  *   rkv_full_attention   attention over C_f: out is complete when this call's one kernel ends; the
- *                        logits and softmax statistics stay in the context's workspace;
+ *                        logits and softmax statistics stay in the context's workspace
+ *                        (rkv_append_full_attention: the same behind the token's append);
  *   rkv_select_topk      scores, topk_idx, q_last_full from that workspace (same values as
  *                        rkv_full_step; out differs from rkv_full_step's by summation order only).
- * rkv_select_topk completes the LAST rkv_full_attention of the same context and must be given the same
+ * rkv_select_topk completes the LAST rkv_[append_]full_attention of the same context and must be given the same
  * cache and mask (otherwise RKV_ERR_INVALID_ARG; also when there is no attention pass to complete).  The
  * workspace holds one pass: no other rkv_full_step / rkv_score_step / rkv_full_attention on this
  * context may run between the two (stream order, or an event, must put them after rkv_select_topk);
@@ -146,6 +147,15 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*ho
  */
 rkv_status rkv_full_attention(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
                               const int32_t* active, void* out, int32_t max_len_hint, void* stream);
+/* The same with the token's new rows appended to C_f first, in the same kernel (one launch; the result is
+ * that of rkv_append(ctx, k_new, v_new, full, NULL) followed by rkv_full_attention): every sequence's
+ * cache grows by one row - inactive ones too, as in rkv_append - and the attention of the active ones
+ * covers the new row.  max_len_hint bounds the lengths AFTER the append.  A cache already at capacity
+ * sets RKV_DEV_APPEND_OVERFLOW and is attended as it is.  (Sec. 2.1: new KV pairs are appended to both
+ * caches; the full step that follows rebuilds C_p, so only C_f needs the row here.) */
+rkv_status rkv_append_full_attention(rkv_ctx* ctx, const void* q, const void* k_new, const void* v_new,
+                                     const rkv_cache* full /*host struct*/, const int32_t* active, void* out,
+                                     int32_t max_len_hint, void* stream);
 rkv_status rkv_select_topk(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
                            const int32_t* k_small, int32_t k_max, const int32_t* active, float* scores,
                            int64_t score_stride, int32_t* topk_idx, void* q_last_full, void* stream);

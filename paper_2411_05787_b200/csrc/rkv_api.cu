@@ -200,8 +200,8 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   // Early cache read: only when the launch before this one on the stream leaves the attended cache alone (a
   // gather or an append into it forbids it; so does an unknown history).
   p.early = (cluster && p.spec != 0 && ctx->early_read && rkv::early_read_safe(st, cache)) ? 1 : 0;
-  if (app != nullptr) {   // only the clustered partial step takes the append with it
-    if (!cluster) return RKV_ERR_INVALID_ARG;
+  if (app != nullptr) {   // the clustered partial step and the full step's attention pass can take the append with them
+    if (!cluster && !(logits && !score_only)) return RKV_ERR_INVALID_ARG;
     p.k_new = app->k_new;
     p.v_new = app->v_new;
     p.small_k = cache->k;
@@ -228,7 +228,7 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
     const bool wide = cluster && (int64_t)gx * ctx->cfg.n_kv_heads * ctx->cfg.n_seq * 2 <= ctx->sm_count;
     e = cluster      ? rkv::launch_attention_cluster(p, tm_k, tm_v, ctx->cfg.n_seq, gx, app != nullptr, wide, st)
         : score_only ? rkv::launch_attention_scores(p, tm_k, tm_v, ctx->cfg.n_seq, gx, st)
-                     : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st);
+                     : rkv::launch_attention(p, tm_k, tm_v, ctx->cfg.n_seq, gx, logits, st, app != nullptr);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
   ctx->launches += 1;
@@ -353,13 +353,13 @@ rkv_status rkv_destroy(rkv_ctx* ctx) {
 // fold_out: the attention kernel also finishes out (otherwise the selection kernel does).
 static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* active,
                                       void* out, int32_t max_len_hint, cudaStream_t st, bool score_only,
-                                      bool fold_out) {
+                                      bool fold_out, const AppendArgs* app = nullptr) {
   if (!ctx || !q || !cache_ok(full) || (!out && !score_only)) return RKV_ERR_INVALID_ARG;
   int n_max = max_len_hint == 0 ? ctx->cfg.max_len : max_len_hint;
   if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
   int chunk = 0, gx = 1;
   ctx->pending_full.valid = false;
-  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, nullptr, score_only,
+  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, app, score_only,
                                fold_out);
   if (s != RKV_OK) return s;
   ctx->pending_full = {true, chunk, gx, n_max, full->k, active};
@@ -454,6 +454,15 @@ rkv_status rkv_score_step(rkv_ctx* ctx, const void* q, const rkv_cache* full, co
 rkv_status rkv_full_attention(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* active, void* out,
                               int32_t max_len_hint, void* stream) {
   return full_attention_part(ctx, q, full, active, out, max_len_hint, static_cast<cudaStream_t>(stream), false, true);
+}
+
+rkv_status rkv_append_full_attention(rkv_ctx* ctx, const void* q, const void* k_new, const void* v_new,
+                                     const rkv_cache* full, const int32_t* active, void* out, int32_t max_len_hint,
+                                     void* stream) {
+  if (!k_new || !v_new) return RKV_ERR_INVALID_ARG;
+  const AppendArgs app = {k_new, v_new, nullptr, nullptr, nullptr, nullptr, 0};   // one cache: the attended one
+  return full_attention_part(ctx, q, full, active, out, max_len_hint, static_cast<cudaStream_t>(stream), false, true,
+                             &app);
 }
 
 rkv_status rkv_select_topk(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,

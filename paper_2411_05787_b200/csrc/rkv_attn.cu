@@ -43,7 +43,8 @@ constexpr int kOPad = 132;  // floats per head row in the merge buffer (bank spr
 constexpr int kQPad = 68;   // 32-bit words per query row in shared memory (64 + 4: the fragment reads spread over all banks)
 constexpr int kRecvFloats = kMaxGroup * kHeadDim + kAttnCluster * kMaxGroup * 2;   // pushed slices + (m, l) pairs
 
-enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2, kModeClusterAppend = 3, kModeScore = 4 };
+enum : int { kModeFull = 0, kModeTicket = 1, kModeCluster = 2, kModeClusterAppend = 3, kModeScore = 4,
+              kModeFullAppend = 5 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -166,10 +167,10 @@ template <int kMode, bool kWideT = false>
 __global__ void __launch_bounds__(Ring<kMode, kWideT>::kThreads, Ring<kMode, kWideT>::kMinBlocks)
 attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
             const AttnParams p) {
-  constexpr bool kLogits = (kMode == kModeFull || kMode == kModeScore);
+  constexpr bool kLogits = (kMode == kModeFull || kMode == kModeScore || kMode == kModeFullAppend);
   constexpr bool kScoreOnly = (kMode == kModeScore);   // logits and softmax statistics only: V is never read
   constexpr bool kCluster = (kMode == kModeCluster || kMode == kModeClusterAppend);
-  constexpr bool kAppend = (kMode == kModeClusterAppend);
+  constexpr bool kAppend = (kMode == kModeClusterAppend || kMode == kModeFullAppend);
   constexpr int kStg = Ring<kMode, kWideT>::kStg;
   constexpr int kMW = Ring<kMode, kWideT>::kMmaWarps;      // MMA warps; warp kMW is the copy warp
   // Rows of a tile per MMA warp.  The bandwidth-bound forms use 16 (four warps per tile).  The clustered
@@ -322,12 +323,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       qb[ks][1] = qd < G ? sm_q[qd * kQPad + 8 * ks + 4 + (lane & 3)] : 0u;
     }
   }
-  // Fused append: the lengths are bumped by the last (sequence, KV head) cluster to get here.  Every cluster
-  // has read the old lengths before it takes its ticket, so nobody can still see them change.
+  // Fused append: the lengths are bumped by the last ticket holder of the sequence.  A ticket is taken only
+  // after the old lengths have been read by everyone it stands for - one per cluster, taken behind the cluster
+  // barrier, or (streaming form, no barrier) one per CTA, taken right here - so nobody can still see them change.
+  bool ticket_due = kAppend && tid == 0 && (!kCluster || split == 0);
   auto take_len_ticket = [&] {
-    if (kAppend && split == 0 && tid == 0) {
+    if (ticket_due) {
+      ticket_due = false;
+      const int holders = kCluster ? p.n_kv_heads : p.n_kv_heads * (int)gridDim.x;
       const int old = atomicAdd(p.len_tickets + b, 1);
-      if (old == p.n_kv_heads - 1) {
+      if (old == holders - 1) {
         if (new_len_s >= 0) p.small_len[b] = new_len_s;
         if (new_len_f >= 0) p.full_len[b] = new_len_f;
         if (bump_evict) p.evict_count[b] += 1;   // the same decision in every cluster of the sequence
@@ -335,6 +340,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       }
     }
   };
+  if (!kCluster) take_len_ticket();
   if (act == 0) {   // the same for every CTA of a cluster
     take_len_ticket();
     return;
@@ -767,6 +773,8 @@ cudaError_t prepare_attention() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_kernel<kModeScore>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_kernel<kModeFullAppend>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_kernel<kModeCluster, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(attn_kernel<kModeClusterAppend, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
@@ -780,8 +788,11 @@ cudaError_t prepare_attention() {
 }
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                             int n_seq, int grid_x, bool write_logits, cudaStream_t st) {
+                             int n_seq, int grid_x, bool write_logits, cudaStream_t st, bool append) {
   dim3 grid(grid_x, p.n_kv_heads, n_seq);
+  if (write_logits && append)
+    return launch_ex(attn_kernel<kModeFullAppend>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v,
+                     p);
   if (write_logits)
     return launch_ex(attn_kernel<kModeFull>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);
   return launch_ex(attn_kernel<kModeTicket>, grid, dim3(kAttnThreads), attention_smem_bytes(), st, 1, tm_k, tm_v, p);

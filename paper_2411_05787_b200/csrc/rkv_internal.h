@@ -101,7 +101,7 @@ struct CacheDev {
 };
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                             int n_seq, int grid_x, bool write_logits, cudaStream_t st);
+                             int n_seq, int grid_x, bool write_logits, cudaStream_t st, bool append = false);
 cudaError_t launch_attention_cluster(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                      int n_seq, int cluster, bool append, bool wide, cudaStream_t st);
 cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v,

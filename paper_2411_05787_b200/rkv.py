@@ -22,7 +22,8 @@ EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", 
            "rkv_small_step", "rkv_append", "rkv_should_refresh", "rkv_get_device_status",
            "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
            "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step", "rkv_score_step",
-           "rkv_gather_small_evict", "rkv_append_small_step_evict", "rkv_full_attention", "rkv_select_topk"]
+           "rkv_gather_small_evict", "rkv_append_small_step_evict", "rkv_full_attention", "rkv_select_topk",
+           "rkv_append_full_attention"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER, OPT_EARLY_CACHE_READ = 1, 2, 3, 4
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger"]
@@ -59,6 +60,8 @@ def _load() -> ctypes.CDLL:
     lib.rkv_score_step.restype = i32
     lib.rkv_full_attention.argtypes = [vp, vp, cachep, vp, vp, i32, vp]
     lib.rkv_full_attention.restype = i32
+    lib.rkv_append_full_attention.argtypes = [vp, vp, vp, vp, cachep, vp, vp, i32, vp]
+    lib.rkv_append_full_attention.restype = i32
     lib.rkv_select_topk.argtypes = [vp, vp, cachep, vp, i32, vp, vp, i64, vp, vp, vp]
     lib.rkv_select_topk.restype = i32
     lib.rkv_gather_small.argtypes = [vp, vp, vp, i32, cachep, cachep, vp, vp]
@@ -186,6 +189,10 @@ class Context:
     def full_attention(self, q, full: RkvCache, out, active=None, max_len_hint=0, stream=None):
         self._check(lib.rkv_full_attention(self._h, _ptr(q), ctypes.byref(full), _ptr(active), _ptr(out),
                                            max_len_hint, _stream(stream)))
+
+    def append_full_attention(self, q, k_new, v_new, full: RkvCache, out, active=None, max_len_hint=0, stream=None):
+        self._check(lib.rkv_append_full_attention(self._h, _ptr(q), _ptr(k_new), _ptr(v_new), ctypes.byref(full),
+                                                  _ptr(active), _ptr(out), max_len_hint, _stream(stream)))
 
     def select_topk(self, q, full: RkvCache, k_small, k_max, topk_idx, active=None, scores=None, q_last_full=None,
                     stream=None):

@@ -68,6 +68,12 @@ class LayerState:
         self.ctx.full_attention(q, self.full_c, self.out, active=active, max_len_hint=max_len_hint, stream=stream)
         return self.out
 
+    def append_refresh_attention(self, q, k_new, v_new, active=None, max_len_hint=0, stream=None):
+        """Append to the full cache and attend over it, one launch (the refresh rebuilds the small cache anyway)."""
+        self.ctx.append_full_attention(q, k_new, v_new, self.full_c, self.out, active=active,
+                                       max_len_hint=max_len_hint, stream=stream)
+        return self.out
+
     def refresh_select(self, q, active=None, stream=None):
         """Second half: scores, top-K and the rebuild of the small cache from what refresh_attention left."""
         self.ctx.select_topk(q, self.full_c, self.k_small, self.k_max, self.topk_idx, active=active,
@@ -99,3 +105,43 @@ class LayerState:
     def check_trigger(self, q, threshold):
         self.ctx.should_refresh(q, self.q_last_full, threshold, self.flag, self.sim, keep=self.not_flag)
         return self.flag
+
+
+class OverlappedRefresh:
+    """Full-step token over a stack of layers with the selection off the layers' critical path.
+
+    What layer l + 1 needs from layer l is its attention output, which is final when rkv_full_attention's kernel
+    ends; the selection and the rebuild of the small cache are first needed by the NEXT token.  The attention
+    passes of all layers follow each other in the calling stream; each layer's selection and rebuild run in a
+    second stream behind its attention and overlap the next layers' attention.  Consecutive layers must use
+    different contexts (a context's workspace holds one attention pass): with two contexts that alternate, a
+    workspace is reused two layers later, after an event has said that the selection reading it has ended."""
+
+    def __init__(self, layers, priority=-1):
+        self.layers = layers
+        for a, b in zip(layers, layers[1:]):
+            if a.ctx is b.ctx:
+                raise ValueError("consecutive layers must not share a context")
+        for a, c in zip(layers, layers[2:]):
+            if a.ctx is not c.ctx:
+                raise ValueError("layers two apart must share a context (two contexts, alternating)")
+        self.side = torch.cuda.Stream(priority=priority)
+        self.ev_attn = [torch.cuda.Event() for _ in layers]
+        self.ev_sel = [torch.cuda.Event() for _ in layers]
+
+    def run(self, q_of, k_new_of, v_new_of, max_len_hint=0):
+        """q_of(l), k_new_of(l), v_new_of(l): the layer's inputs.  Appends, attends, selects, rebuilds."""
+        main = torch.cuda.current_stream()
+        n = len(self.layers)
+        for l, st in enumerate(self.layers):
+            if l >= 2:
+                main.wait_event(self.ev_sel[l - 2])
+            st.append_refresh_attention(q_of(l), k_new_of(l), v_new_of(l), max_len_hint=max_len_hint)
+            self.ev_attn[l].record(main)
+            self.side.wait_event(self.ev_attn[l])
+            with torch.cuda.stream(self.side):
+                st.refresh_select(q_of(l))
+                self.ev_sel[l].record(self.side)
+        for l in range(max(n - 2, 0), n):
+            main.wait_event(self.ev_sel[l])
+

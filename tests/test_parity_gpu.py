@@ -146,6 +146,56 @@ def test_full_step_in_two_halves_matches_oracle(mods, lens, k_small, n_q, n_kv):
     assert torch.equal(st.q_last_full, q)
 
 
+@pytest.mark.parametrize("n_full", [0, 1, 63, 64, 1000, 2047, 2048, 4159])
+def test_fused_append_full_attention_equals_append_then_attention(mods, n_full):
+    """rkv_append_full_attention against rkv_append + rkv_full_attention on twin caches: same rows, lengths, flags,
+    output bits, and - after rkv_select_topk - the same scores and indices; the active sequences also against the
+    oracle.  The new row lands at tile and chunk boundaries, in an empty cache and (third step) in a full one."""
+    rkv, runner, synth = mods
+    dev = torch.device("cuda")
+    n_q, n_kv, B, K = 28, 4, 3, 48
+    lens, caps = [n_full, n_full // 2, 5], [n_full + 2, n_full // 2 + 3, 7]
+    g = torch.Generator(device=dev); g.manual_seed(900 + n_full)
+    fa = synth.alloc_cache(caps, lens, n_kv, dev)
+    fb = synth.alloc_cache(caps, lens, n_kv, dev)
+    for t in (fa.k, fa.v):
+        t.copy_(torch.randn(t.shape, generator=g, device=dev).to(torch.bfloat16))
+    fb.k.copy_(fa.k); fb.v.copy_(fa.v)
+    ctx_a = rkv.Context(B, n_q, n_kv, max(caps), K + 4)
+    ctx_b = rkv.Context(B, n_q, n_kv, max(caps), K + 4)
+    cs = lambda c: rkv.cache_struct(c.k, c.v, c.row_offset, c.cap, c.len)
+    sa, sb = cs(fa), cs(fb)
+    k_small = torch.tensor([K, K, 3], dtype=torch.int32, device=dev)
+    active = torch.tensor([1, 0, 1], dtype=torch.int32, device=dev)
+    mk = lambda: (torch.zeros((B, n_q, 128), dtype=torch.bfloat16, device=dev),
+                  torch.full((B, n_kv, K), -7, dtype=torch.int32, device=dev),
+                  torch.zeros((B, n_kv, max(caps)), dtype=torch.float32, device=dev))
+    for step in range(3):
+        q = torch.randn((B, n_q, 128), generator=g, device=dev).to(torch.bfloat16)
+        kn = torch.randn((B, n_kv, 128), generator=g, device=dev).to(torch.bfloat16)
+        vn = torch.randn((B, n_kv, 128), generator=g, device=dev).to(torch.bfloat16)
+        (out_a, idx_a, sc_a), (out_b, idx_b, sc_b) = mk(), mk()
+        out_a.fill_(3.0); out_b.fill_(3.0)
+        ctx_a.append_full_attention(q, kn, vn, sa, out_a, active=active)
+        ctx_a.select_topk(None, sa, k_small, K, idx_a, active=active, scores=sc_a)
+        bits_a = ctx_a.device_status()
+        ctx_b.append(kn, vn, sb, None)
+        ctx_b.full_attention(q, sb, out_b, active=active)
+        ctx_b.select_topk(None, sb, k_small, K, idx_b, active=active, scores=sc_b)
+        bits_b = ctx_b.device_status()
+        assert bits_a == bits_b, (step, bits_a, bits_b)
+        assert fa.len.tolist() == fb.len.tolist()
+        assert torch.equal(fa.k, fb.k) and torch.equal(fa.v, fb.v)
+        assert torch.equal(out_a, out_b) and torch.equal(idx_a, idx_b) and torch.equal(sc_a, sc_b), f"step {step}"
+        assert (out_a[1] == 3.0).all() and (idx_a[1] == -7).all()   # inactive: untouched, but its cache grew
+        for b in (0, 2):
+            n = int(fa.len[b])
+            want = oracle_full(fa, b, n, q[b], n_kv, int(k_small[b]))[0]
+            check_out(out_a[b], want, f"fused full step {step} seq {b}")
+    # three appends: sequence 0 had room for two, sequence 1 for three, sequence 2 for two
+    assert fa.len.tolist() == [n_full + 2, n_full // 2 + 3, 7]
+
+
 def test_select_topk_needs_its_attention_pass(mods):
     rkv, runner, synth = mods
     ctx, st, cache, q = make_layer(mods, [300], [16], 8, 2)
@@ -761,16 +811,19 @@ def test_largest_supported_length(mods):
 
 
 def test_bench_configuration_graph_replay_shared_context(mods):
-    """The launch configuration bench.py times, at config 2's full size: several layers share one context, a token's
-    calls (rkv_append_small_step, or rkv_append + rkv_full_step + rkv_gather_small) are replayed from CUDA graphs
-    with the inputs staged in a device buffer.  Every layer's output of every token is compared with the oracle."""
+    """The launch configuration bench.py times, at config 2's full size: the layers alternate between two
+    contexts, a token's calls are replayed from CUDA graphs with the inputs staged in a device buffer.  Partial
+    tokens: one rkv_append_small_step per layer (the early cache read is live: the launch before each is another
+    layer's).  Full-step tokens: rkv_append + rkv_full_attention in the capturing stream, rkv_select_topk +
+    rkv_gather_small behind them in a second stream (runner.OverlappedRefresh).  Every layer's output of every
+    token is compared with the oracle."""
     rkv, runner, synth = mods
     dev = torch.device("cuda")
-    NL, S, T = 2, 10, 11
+    NL, S, T = 3, 10, 21
     w = synth.scaled(synth.config2(n_layers=NL), steps=T)
     L, K, Hq, Hkv = w.lens[0], w.k_small[0], w.n_q_heads, w.n_kv_heads
     full_hint, small_hint = L + T + 1, K + S + 2
-    ctx = rkv.Context(1, Hq, Hkv, full_hint, small_hint)
+    ctxs = [rkv.Context(1, Hq, Hkv, full_hint, small_hint) for _ in range(2)]
     q_stage = torch.zeros((NL, 1, Hq, 128), dtype=torch.bfloat16, device=dev)
     k_stage = torch.zeros((NL, 1, Hkv, 128), dtype=torch.bfloat16, device=dev)
     v_stage = torch.zeros((NL, 1, Hkv, 128), dtype=torch.bfloat16, device=dev)
@@ -780,7 +833,7 @@ def test_bench_configuration_graph_replay_shared_context(mods):
         qs = synth.query_trajectory(w, l).to(dev)
         kn, vn = synth.new_token_kv(w, l)
         synth.plant_heavy(w, cache, l, qs[0])
-        st = runner.LayerState(ctx, cache, [K], S + 2, Hq, Hkv)
+        st = runner.LayerState(ctxs[l % 2], cache, [K], S + 2, Hq, Hkv)
         layers.append(st)
         inputs.append((qs, kn.to(dev), vn.to(dev)))
         states.append(O.SequenceState(host_heads(cache, 0, Hkv, "k").copy(), host_heads(cache, 0, Hkv, "v").copy(), L, K))
@@ -789,13 +842,14 @@ def test_bench_configuration_graph_replay_shared_context(mods):
         for l in range(NL):
             q_stage[l].copy_(inputs[l][0][t]); k_stage[l].copy_(inputs[l][1][t]); v_stage[l].copy_(inputs[l][2][t])
 
+    overlapped = runner.OverlappedRefresh(layers)
+
     def token(kind):
+        if kind == "full":
+            return overlapped.run(lambda l: q_stage[l], lambda l: k_stage[l], lambda l: v_stage[l],
+                                  max_len_hint=full_hint)
         for l, st in enumerate(layers):
-            if kind == "full":
-                st.append(k_stage[l], v_stage[l])
-                st.refresh(q_stage[l], max_len_hint=full_hint)
-            else:
-                st.append_partial(q_stage[l], k_stage[l], v_stage[l], max_len_hint=small_hint)
+            st.append_partial(q_stage[l], k_stage[l], v_stage[l], max_len_hint=small_hint)
 
     class W1:      # what follow_gpu_selection needs to know about the workload
         n_kv_heads, k_small = Hkv, [K]
@@ -827,5 +881,5 @@ def test_bench_configuration_graph_replay_shared_context(mods):
                 follow_gpu_selection(st, states[l], 0, o_score, W1)
             else:
                 check_out(st.out[0], states[l].small(bits(inputs[l][0][t, 0])), f"partial token {t} layer {l}")
-    assert ctx.device_status() == 0
+    assert all(c.device_status() == 0 for c in ctxs)
     assert all(int(st.full.len[0]) == L + T and int(st.small.len[0]) == K + 1 for st in layers)
