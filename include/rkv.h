@@ -133,8 +133,9 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*ho
  * what the decoder needs next; the refreshed partial cache is first read by the NEXT token's partial
  * step).  A caller that wants the attention output early - and the selection and the rebuild of C_p
  * off the layer's critical path, e.g. on a second stream under the next layer's work - calls
- *   rkv_full_attention   attention over C_f: out is complete when this call's one kernel ends; the
- *                        logits and softmax statistics stay in the context's workspace
+ *   rkv_full_attention   attention over C_f: out is complete when this call's two kernels end (the
+ *                        streaming pass, then a short merge of its split partials); the logits
+ *                        and softmax statistics stay in the context's workspace
  *                        (rkv_append_full_attention: the same behind the token's append);
  *   rkv_select_topk      scores, topk_idx, q_last_full from that workspace (same values as
  *                        rkv_full_step; out differs from rkv_full_step's by summation order only).
@@ -350,7 +351,8 @@ rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
 #define RKV_KERNEL_GATHER 3     /* rkv_gather_small                                                  */
 #define RKV_KERNEL_APPEND 4     /* rkv_append                                                        */
 #define RKV_KERNEL_TRIGGER 5    /* rkv_should_refresh                                                */
-#define RKV_KERNEL_KINDS 6
+#define RKV_KERNEL_FOLD 6       /* output from the split partials        (rkv_[append_]full_attention, 2nd kernel) */
+#define RKV_KERNEL_KINDS 7
 rkv_status rkv_set_profiling(rkv_ctx* ctx, int32_t on);
 rkv_status rkv_get_profile(rkv_ctx* ctx, double* total_us /*host*/, int64_t* launches /*host*/);
 

@@ -154,7 +154,7 @@ bool cluster_eligible(const rkv_ctx* ctx, int n_max) { return ctx->small_cluster
 
 rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, const int32_t* active, void* out,
                          int n_max, int limit, bool logits, cudaStream_t st, int* chunk_out, int* gx_out,
-                         const AppendArgs* app = nullptr, bool score_only = false, bool fold_out = false) {
+                         const AppendArgs* app = nullptr, bool score_only = false) {
   if (!aligned16(q) || !aligned16(out) || (app != nullptr && (!aligned16(app->k_new) || !aligned16(app->v_new))))
     return RKV_ERR_INVALID_ARG;   // the kernels read and write these 16 bytes at a time
   CUtensorMap tm_k, tm_v;
@@ -196,7 +196,6 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   p.scale = ctx->cfg.softmax_scale;
   // without a mask: a cluster per head always has work; a streaming grid has when it serves a single sequence
   p.spec = (active == nullptr && (cluster || (logits && ctx->cfg.n_seq == 1))) ? 1 : 0;
-  p.fold_out = (logits && !score_only && fold_out) ? 1 : 0;
   // Early cache read: only when the launch before this one on the stream leaves the attended cache alone (a
   // gather or an append into it forbids it; so does an unknown history).
   p.early = (cluster && p.spec != 0 && ctx->early_read && rkv::early_read_safe(st, cache)) ? 1 : 0;
@@ -350,7 +349,7 @@ rkv_status rkv_destroy(rkv_ctx* ctx) {
 }
 
 // First half of the full step: attention over the full cache, logits and softmax statistics to the workspace.
-// fold_out: the attention kernel also finishes out (otherwise the selection kernel does).
+// fold_out: a second kernel finishes out from the partials right away (otherwise the selection kernel does).
 static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* active,
                                       void* out, int32_t max_len_hint, cudaStream_t st, bool score_only,
                                       bool fold_out, const AppendArgs* app = nullptr) {
@@ -359,9 +358,19 @@ static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cac
   if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
   int chunk = 0, gx = 1;
   ctx->pending_full.valid = false;
-  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, app, score_only,
-                               fold_out);
+  rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, app, score_only);
   if (s != RKV_OK) return s;
+  if (fold_out && !score_only) {
+    cudaError_t e;
+    {
+      LaunchScope scope(ctx, st, RKV_KERNEL_FOLD);
+      e = rkv::launch_fold(ctx->partials, ctx->ml_t, full->len, full->cap, active, out, ctx->cfg.n_seq,
+                           ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, chunk, ctx->max_splits, n_max, st);
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "fold launch");
+    ctx->launches += 1;
+    rkv::note_launch(st, nullptr, nullptr);
+  }
   ctx->pending_full = {true, chunk, gx, n_max, full->k, active};
   return RKV_OK;
 }

@@ -730,7 +730,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         t[(int64_t)(kMaxGroup + d) * p.max_splits] = Ld;
       }
     }
-    if (kLogits && (kScoreOnly || p.fold_out == 0)) return;   // full step: the selection kernel folds the partials
+    if (kLogits) return;   // full step: the selection kernel (or the fold kernel) finishes out from the partials
     __threadfence();
     consumer_bar();
     if (tid == 0) {

@@ -50,7 +50,6 @@ struct AttnParams {
   int32_t max_len;            // clamp for len[b]
   int32_t spec;               // 1: every CTA has work by construction, first tiles may be requested before len is read
   int32_t early;              // 1 (clustered step with spec): request them before the dependency wait as well
-  int32_t fold_out;           // full step: 1 = the last CTA of each (sequence, KV head) folds the partials and writes out
   float scale;
   // fused append (clustered partial step only): the new token's rows and where they go
   const void* k_new;          // bf16 [B][Hkv][128]
@@ -116,6 +115,9 @@ cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k
 cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, CacheDev small_cache,
                           bool has_full, bool has_small, int n_seq, int n_kv_heads, int32_t* status,
                           cudaStream_t st);
+cudaError_t launch_fold(const float* partials, const float* ml_t, const int32_t* len, const int32_t* cap,
+                        const int32_t* active, void* out, int n_seq, int n_q_heads, int n_kv_heads, int chunk,
+                        int max_splits, int max_len, cudaStream_t st);
 cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, int32_t* keep,
                            float* sim, int n_seq, int n_q_heads, cudaStream_t st);
 // Launch with optional programmatic dependent launch (the kernel may start while its predecessor on

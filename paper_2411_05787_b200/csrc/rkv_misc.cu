@@ -156,6 +156,80 @@ __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __res
   }
 }
 
+// Attention output of the full step from the split partials its streaming pass left in the workspace (the
+// flash-decoding merge: M = max_s m_s, w_s = exp(m_s - M), out = sum_s w_s O_s / sum_s w_s l_s).  A kernel of its
+// own, for rkv_full_attention: hundreds of small blocks finish in about one memory round trip, where the last
+// CTA of the streaming pass would need several microseconds of dependent round trips on an otherwise idle GPU.
+// One block per (sequence, KV head, head of the group, quarter of the channels); warp w takes the splits
+// s = w (mod 4), lane c the channel; every load is issued before the first is used.
+__global__ void __launch_bounds__(128) fold_kernel(const float* __restrict__ partials, const float* __restrict__ ml_t,
+                                                   const int32_t* __restrict__ len, const int32_t* __restrict__ cap,
+                                                   const int32_t* __restrict__ active, __nv_bfloat16* __restrict__ out,
+                                                   int n_q_heads, int n_kv_heads, int group, int chunk, int max_splits,
+                                                   int max_len) {
+  constexpr int kU = 8;   // splits per warp in the first batch of loads (4 * kU = 32 splits)
+  constexpr float kLog2e = 1.4426950408889634f;
+  const int h = blockIdx.x >> 2, c = (blockIdx.x & 3) * 32 + (threadIdx.x & 31);
+  const int g = blockIdx.y, b = blockIdx.z, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ float sm_e[kMaxSplits];
+  __shared__ float sm_red[4][32];
+  __shared__ float sm_L;
+  pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
+  if (active != nullptr && __ldcg(active + b) == 0) return;
+  int n = __ldcg(len + b);
+  const int cp = __ldg(cap + b), lim = cp < max_len ? cp : max_len;
+  n = n < lim ? n : lim;            // the clamp of the streaming pass
+  if (n <= 0) return;               // nothing cached: the streaming pass has written zeros
+  const int n_splits = (n + chunk - 1) / chunk;
+  const int64_t bg = (int64_t)b * n_kv_heads + g;
+  const float* po = partials + bg * max_splits * PartialLayout::kFloats + h * kHeadDim + c;
+  float v[kU];
+#pragma unroll
+  for (int k = 0; k < kU; ++k) {
+    const int s = warp + 4 * k;
+    v[k] = s < n_splits ? __ldcg(po + (int64_t)s * PartialLayout::kFloats) : 0.f;
+  }
+  if (warp == 0) {   // weights of all splits (at most kMaxSplits = 4 per lane), their sum of denominators
+    const float* pm = ml_t + bg * 16 * max_splits + (int64_t)h * max_splits;
+    const float* pl = pm + (int64_t)kMaxGroup * max_splits;
+    float m[4], l[4], M = -INFINITY, L = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int s = lane + 32 * i;
+      m[i] = s < n_splits ? __ldcg(pm + s) : -INFINITY;
+      l[i] = s < n_splits ? __ldcg(pl + s) : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) M = fmaxf(M, m[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float e = (m[i] == -INFINITY) ? 0.f : exp2f((m[i] - M) * kLog2e);
+      L = fmaf(l[i], e, L);
+      sm_e[lane + 32 * i] = e;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+    if (lane == 0) sm_L = L;
+  }
+  __syncthreads();
+  float acc = 0.f;
+#pragma unroll
+  for (int k = 0; k < kU; ++k) {
+    const int s = warp + 4 * k;
+    if (s < n_splits) acc = fmaf(v[k], sm_e[s], acc);
+  }
+  for (int s = warp + 4 * kU; s < n_splits; s += 4) acc = fmaf(__ldcg(po + (int64_t)s * PartialLayout::kFloats), sm_e[s], acc);
+  sm_red[warp][lane] = acc;
+  __syncthreads();
+  if (warp == 0) {
+    const float sum = (sm_red[0][lane] + sm_red[1][lane]) + (sm_red[2][lane] + sm_red[3][lane]);
+    out[((int64_t)b * n_q_heads + (int64_t)g * group + h) * kHeadDim + c] = __float2bfloat16(sum / sm_L);
+  }
+}
+
 // Eviction order of a freshly rebuilt small cache (Sec. 2.2 "Decoding with partial cache": to keep C_p at a fixed
 // size, the entry with the lowest attention score of the last full step is dropped for each new token).  One block
 // per (sequence, KV head): bitonic sort of (key, slot) pairs, largest key = lowest score first, the higher slot
@@ -229,6 +303,14 @@ cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, C
   return launch_ex(append_kernel, dim3(n_seq), dim3(128), 0, st, 1, static_cast<const uint4*>(k_new),
                    static_cast<const uint4*>(v_new), full, small_cache, has_full ? 1 : 0, has_small ? 1 : 0,
                    n_kv_heads, status);
+}
+
+cudaError_t launch_fold(const float* partials, const float* ml_t, const int32_t* len, const int32_t* cap,
+                        const int32_t* active, void* out, int n_seq, int n_q_heads, int n_kv_heads, int chunk,
+                        int max_splits, int max_len, cudaStream_t st) {
+  const int group = n_q_heads / n_kv_heads;
+  return launch_ex(fold_kernel, dim3(4 * group, n_kv_heads, n_seq), dim3(128), 0, st, 1, partials, ml_t, len, cap,
+                   active, static_cast<__nv_bfloat16*>(out), n_q_heads, n_kv_heads, group, chunk, max_splits, max_len);
 }
 
 cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, int32_t* keep,
