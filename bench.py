@@ -30,9 +30,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 # DRAM traffic of one full-step attention launch per algorithmic K/V byte, from the ncu capture of the cfg-2
-# launch summarised in profiles/attn_kernel_full_step_cfg2_L32768.md (134.27 MB read + 3.54 MB written for
+# launch summarised in profiles/attn_kernel_full_step_cfg2_L32768.md (134.52 MB read + 3.60 MB written for
 # 134.22 MB of K/V); traffic grows with the positions streamed.  Set to None when the kernel changes.
-ATTN_FULL_TRAFFIC_PER_KV_BYTE = 137.81 / 134.22
+ATTN_FULL_TRAFFIC_PER_KV_BYTE = 138.12 / 134.22
 
 METRIC = "decode attention us/token (all layers, refresh schedule of the workload; full step and small step also reported)"
 UNIT = "us/token"
@@ -481,8 +481,8 @@ def run_ours(args):
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": NL * B * row * 2,
                 "d2h_bytes_per_step": NL * B * Hq * 128 * 2},
         "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "attn_kernel<full> (full-cache attention + score logits; with the "
-                                               "token's append and the output fold when the selection is overlapped)",
+        "roofline": {"bound": "hbm", "kernel": "attn_kernel<full> (full-cache attention + score logits, the token's "
+                                               "append fused in)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": peak_src,
                      "traffic": (kv_bytes_full * ATTN_FULL_TRAFFIC_PER_KV_BYTE

@@ -325,7 +325,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   }
   // Fused append: the lengths are bumped by the last ticket holder of the sequence.  A ticket is taken only
   // after the old lengths have been read by everyone it stands for - one per cluster, taken behind the cluster
-  // barrier, or (streaming form, no barrier) one per CTA, taken right here - so nobody can still see them change.
+  // barrier, or (streaming form, no barrier) one per CTA, taken when the CTA is done - so nobody can still see
+  // them change.
   bool ticket_due = kAppend && tid == 0 && (!kCluster || split == 0);
   auto take_len_ticket = [&] {
     if (ticket_due) {
@@ -340,7 +341,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       }
     }
   };
-  if (!kCluster) take_len_ticket();
   if (act == 0) {   // the same for every CTA of a cluster
     take_len_ticket();
     return;
@@ -371,6 +371,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         for (int t = 0; t < n_spec; ++t) mbar_wait(bar_full + 8 * t, 0);
       __syncthreads();
     }
+    take_len_ticket();
     return;
   }
   const int end = (start + p.chunk < n) ? start + p.chunk : n;
@@ -730,6 +731,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         t[(int64_t)(kMaxGroup + d) * p.max_splits] = Ld;
       }
     }
+    take_len_ticket();     // streaming form with the append: at the very end, off the CTA's critical path
     if (kLogits) return;   // full step: the selection kernel (or the fold kernel) finishes out from the partials
     __threadfence();
     consumer_bar();
