@@ -317,6 +317,10 @@ def run_ours(args):
             # every layer's attention in this stream; its selection and rebuild behind it in a second one
             return overlapped.run(lambda l: q_stage[l], lambda l: k_stage[l], lambda l: v_stage[l],
                                   max_len_hint=full_hint)
+        if kind == "check" and overlap:
+            return overlapped.run_checked(lambda l: q_stage[l], lambda l: k_stage[l], lambda l: v_stage[l],
+                                          w.threshold, small_hint=small_hint, full_hint=full_hint,
+                                          after_trigger=lambda l, st: flag_total[l].add_(st.flag))
         for l, st in enumerate(layers):
             q, kn, vn = q_stage[l], k_stage[l], v_stage[l]
             if kind in ("full", "full_seq"):

@@ -145,3 +145,26 @@ class OverlappedRefresh:
         for l in range(max(n - 2, 0), n):
             main.wait_event(self.ev_sel[l])
 
+    def run_checked(self, q_of, k_new_of, v_new_of, threshold, small_hint=0, full_hint=0, after_trigger=None):
+        """Token of the dynamic schedule at a check position: per layer the trigger, then both branches under its
+        device masks - the partial step (which appends to both caches for every sequence) for the sequences that
+        keep their small cache, the full step for those that refresh - with the full step's selection and rebuild
+        behind the attention in the second stream, as in run()."""
+        main = torch.cuda.current_stream()
+        n = len(self.layers)
+        for l, st in enumerate(self.layers):
+            if l >= 2:
+                main.wait_event(self.ev_sel[l - 2])
+            st.check_trigger(q_of(l), threshold)
+            if after_trigger is not None:
+                after_trigger(l, st)
+            st.append_partial(q_of(l), k_new_of(l), v_new_of(l), active=st.not_flag, max_len_hint=small_hint)
+            st.refresh_attention(q_of(l), active=st.flag, max_len_hint=full_hint)
+            self.ev_attn[l].record(main)
+            self.side.wait_event(self.ev_attn[l])
+            with torch.cuda.stream(self.side):
+                st.refresh_select(q_of(l), active=st.flag)
+                self.ev_sel[l].record(self.side)
+        for l in range(max(n - 2, 0), n):
+            main.wait_event(self.ev_sel[l])
+

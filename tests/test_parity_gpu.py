@@ -558,8 +558,11 @@ def test_host_side_argument_errors(mods):
 
 
 # ----------------------------------------------------------------------------- the five workload configs
-def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False, evict=0):
-    """Run workload `w` for one layer on the GPU and step the oracle beside it on the same bytes."""
+def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False, evict=0, overlapped=False):
+    """Run workload `w` for one layer on the GPU and step the oracle beside it on the same bytes.
+
+    overlapped: full-step and check tokens go through runner.OverlappedRefresh (attention in the calling stream,
+    selection and rebuild behind it in a second one), the way bench.py launches them."""
     rkv, runner, synth = mods
     dev = torch.device("cuda")
     cache = synth.fill_layer(w, layer, dev)
@@ -574,6 +577,7 @@ def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False, evict=
         st.enable_eviction(evict)
         st.refresh, st.append_partial = st.refresh_evict, st.append_partial_evict
         fused = True
+    ov = runner.OverlappedRefresh([st]) if overlapped else None
     seqs = list(range(w.batch)) if seqs is None else seqs
     # oracle state per checked sequence, on copies of the same bytes
     states = {}
@@ -597,7 +601,9 @@ def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False, evict=
             states[b].append(bits(kn[t, b]), bits(vn[t, b]))
         if w.schedule == "fixed":
             full_now = [O.fixed_stride_is_full(t, w.stride)] * w.batch
-            if full_now[0]:
+            if full_now[0] and ov is not None:
+                ov.run(lambda l: qs[t], lambda l: kn[t], lambda l: vn[t])
+            elif full_now[0]:
                 st.append(kn[t], vn[t])
                 st.refresh(qs[t])
             elif fused:
@@ -608,16 +614,21 @@ def run_trajectory(mods, w, layer, seqs=None, check_every=1, fused=False, evict=
         else:
             full_now = [False] * w.batch
             if t % w.stride == 0:
-                st.check_trigger(qs[t], w.threshold)
-                flags = st.flag.cpu().numpy()
-                assert torch.equal(st.not_flag, 1 - st.flag)      # the trigger wrote both masks
-                if fused:      # appends for every sequence, attends for those that keep the partial cache
-                    st.append_partial(qs[t], kn[t], vn[t], active=st.not_flag)
-                    st.refresh(qs[t], active=st.flag)
+                if ov is not None:      # trigger, both branches under its masks, selection in the second stream
+                    ov.run_checked(lambda l: qs[t], lambda l: kn[t], lambda l: vn[t], w.threshold)
+                    torch.cuda.synchronize()
+                    flags = st.flag.cpu().numpy()
                 else:
-                    st.append(kn[t], vn[t])
-                    st.refresh(qs[t], active=st.flag)
-                    st.partial(qs[t], active=st.not_flag)
+                    st.check_trigger(qs[t], w.threshold)
+                    flags = st.flag.cpu().numpy()
+                    if fused:      # appends for every sequence, attends for those that keep the partial cache
+                        st.append_partial(qs[t], kn[t], vn[t], active=st.not_flag)
+                        st.refresh(qs[t], active=st.flag)
+                    else:
+                        st.append(kn[t], vn[t])
+                        st.refresh(qs[t], active=st.flag)
+                        st.partial(qs[t], active=st.not_flag)
+                assert torch.equal(st.not_flag, 1 - st.flag)      # the trigger wrote both masks
                 full_now = [bool(f) for f in flags]
                 for b in seqs:
                     want, cos = O.should_refresh(O.bf16_bits_to_f64(bits(qs[t, b])), states[b].q_last_full, w.threshold)
@@ -683,11 +694,11 @@ def follow_gpu_selection(st, state, b, o_score, w):
             assert np.array_equal(gpu_small[g, :take], small[g])
 
 
-@pytest.mark.parametrize("fused", [False, True])
-def test_config1_every_step_every_head(mods, fused):
+@pytest.mark.parametrize("fused,overlapped", [(False, False), (True, False), (True, True)])
+def test_config1_every_step_every_head(mods, fused, overlapped):
     rkv, runner, synth = mods
     w = synth.config1()
-    n_full = run_trajectory(mods, w, 0, fused=fused)
+    n_full = run_trajectory(mods, w, 0, fused=fused, overlapped=overlapped)
     assert n_full[0] == 4      # full steps at t = 4, 8, 12, 16
 
 
@@ -764,12 +775,12 @@ def test_config2_shape_one_layer_full_size(mods):
     assert n_full[0] == 1
 
 
-@pytest.mark.parametrize("fused", [False, True])
-def test_config3_shape_dynamic_flags(mods, fused):
+@pytest.mark.parametrize("fused,overlapped", [(False, False), (True, False), (True, True)])
+def test_config3_shape_dynamic_flags(mods, fused, overlapped):
     """Qwen2-7B shape (G=7), batch 4, dynamic refresh; reduced context for the per-step oracle, full K ratio."""
     rkv, runner, synth = mods
     w = synth.scaled(synth.config3(n_layers=1, ctx=8192), steps=40)
-    n_full = run_trajectory(mods, w, 0, fused=fused)
+    n_full = run_trajectory(mods, w, 0, fused=fused, overlapped=overlapped)
     # fast-drifting sequences refresh more often than slow ones
     assert n_full[0] >= n_full[3]
     assert n_full[0] >= 1
