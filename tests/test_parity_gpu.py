@@ -555,6 +555,16 @@ def test_host_side_argument_errors(mods):
         rkv.Context(1, 8, 2, 100, 10, pool_kernel=33)
     with pytest.raises(rkv.RkvError):
         rkv.Context(1, 8, 2, 200000, 10, pool_kernel=7)      # with pooling the length limit is 163840
+    # bf16 tensors start on a 16-byte boundary: a query (or output) view that begins 2 bytes in is refused
+    skew = torch.zeros(q.numel() + 8, dtype=torch.bfloat16, device=q.device)
+    q_off = skew[1: 1 + q.numel()].view_as(q)
+    out_off = skew[1: 1 + st.out.numel()].view_as(st.out)
+    with pytest.raises(rkv.RkvError):
+        ctx.full_step(q_off, st.full_c, st.k_small, st.k_max, st.out, st.topk_idx)
+    with pytest.raises(rkv.RkvError):
+        ctx.small_step(q, st.small_c, out_off)
+    st.refresh(q)                                            # the context is still usable
+    assert ctx.device_status() == 0
 
 
 # ----------------------------------------------------------------------------- the five workload configs
