@@ -10,23 +10,28 @@
 //
 // Shape of the kernel: one CTA per (sequence, KV head, chunk of positions).
 // A copy warp streams 64-position tiles of K and V into a shared-memory ring (3 stages,
-// 6 in the clustered partial step) with tensor-map TMA loads, one per K or V tile (128-byte swizzle, completion on
-// mbarriers).  Four MMA warps each own 16 positions of a tile: S^T = K Q^T and
-// O^T += V^T P^T with m16n8k16 bf16 tensor-core MMAs (fp32 accumulate), where
-// the N=8 dimension holds all query heads of the group, so K/V are read once
-// per group.  Online softmax lives in registers.  Three ways to merge the splits:
-//   full step      partials go to the workspace, the selection kernel folds them (the score-only
-//                  variant of the full step streams K alone: logits and softmax statistics, no output);
+// 6 in the wide form of the clustered partial step) with tensor-map TMA loads, one per K or
+// V tile (128-byte swizzle, completion on mbarriers).  The MMA warps own bands of a tile
+// (16 positions; 32 in the wide form): S^T = K Q^T and O^T += V^T P^T with m16n8k16 bf16
+// tensor-core MMAs (fp32 accumulate), where the N=8 dimension holds all query heads of the
+// group, so K/V are read once per group.  Online softmax lives in registers; the warps of a
+// CTA merge by a sum of accumulators pre-scaled to the CTA-wide maximum.  Three ways to
+// merge the splits:
+//   full step      partials go to the workspace; the selection kernel folds them, or - for
+//                  rkv_full_attention - a small fold kernel right behind this one (the
+//                  score-only variant streams K alone: logits and softmax statistics);
 //   partial step   (a) the CTAs of one (sequence, KV head) form a thread-block cluster:
 //                  each pushes its slice of the partial output into the peer that owns
 //                  that slice through distributed shared memory, one cluster barrier,
 //                  each CTA finishes 128/C channels of every head;
 //                  (b) long small caches: partials to the workspace, folded by the last
 //                  CTA of each (sequence, KV head) to arrive (atomic ticket, no spin).
-// The clustered partial step can also take the append with it (Sec. 2.2: the partial
-// step stores the input token's K/V in C_p, and C_f receives it too): the new rows are
-// written to both caches, patched into the shared-memory tile that covers the new
-// position, and the lengths are bumped by the last cluster of a sequence to finish.
+// The clustered partial step and the full step's pass can take the append with them
+// (Sec. 2.2: the input token's K/V is stored in C_p, and C_f receives it too): the new rows
+// are written to the cache(s), patched into the shared-memory tile that covers the new
+// position, and the lengths are bumped by the last ticket holder of a sequence.
+// The clustered partial step may also request its tiles before its stream dependency has
+// resolved (AttnParams::early): see the comment at the dependency wait.
 #include <cuda_bf16.h>
 
 #include "rkv_fold.cuh"
@@ -149,7 +154,7 @@ __device__ __forceinline__ void cluster_sync_alive() {
 
 // Stage ring: normally two CTAs per SM with three 32 KiB stages each.  The clustered partial step with few
 // clusters (batch 1) is a pure latency chain on half-empty SMs: its "wide" form takes the whole SM, keeps six
-// tiles in flight and splits the tiles over two groups of MMA warps.  With many clusters the narrow form wins
+// tiles in flight and splits the tiles over five pairs of MMA warps.  With many clusters the narrow form wins
 // (two CTAs per SM place clusters more freely and overlap each other's latencies).
 template <int kMode, bool kWideT>
 struct Ring {
@@ -176,7 +181,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // Rows of a tile per MMA warp.  The bandwidth-bound forms use 16 (four warps per tile).  The clustered
   // partial step is bound by the length of one warp's instruction chain: there a warp takes 32 rows, two
   // independent 16-row blocks that share one softmax update, and two warps cover a tile.
-  constexpr int kNB = kWideT ? 2 : 1;               // 16-row blocks per warp
+  constexpr int kNB = Ring<kMode, kWideT>::kWide ? 2 : 1;   // 16-row blocks per warp
   constexpr int kBand = 16 * kNB;
   constexpr int kWT = kTile / kBand;                // warps per tile
   constexpr int kGroups = kMW / kWT;                // groups of warps that take alternate tiles
