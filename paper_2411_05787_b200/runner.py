@@ -117,7 +117,7 @@ class OverlappedRefresh:
     different contexts (a context's workspace holds one attention pass): with two contexts that alternate, a
     workspace is reused two layers later, after an event has said that the selection reading it has ended."""
 
-    def __init__(self, layers, priority=-1):
+    def __init__(self, layers, priority=0):
         self.layers = layers
         for a, b in zip(layers, layers[1:]):
             if a.ctx is b.ctx:
