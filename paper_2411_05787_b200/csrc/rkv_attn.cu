@@ -10,7 +10,7 @@
 //
 // Shape of the kernel: one CTA per (sequence, KV head, chunk of positions).
 // A copy warp streams 64-position tiles of K and V into a shared-memory ring (3 stages,
-// 6 in the wide form of the clustered partial step) with tensor-map TMA loads, one per K or
+// 5 in the wide form of the clustered partial step) with tensor-map TMA loads, one per K or
 // V tile (128-byte swizzle, completion on mbarriers).  The MMA warps own bands of a tile
 // (16 positions; 32 in the wide form): S^T = K Q^T and O^T += V^T P^T with m16n8k16 bf16
 // tensor-core MMAs (fp32 accumulate), where the N=8 dimension holds all query heads of the
@@ -153,13 +153,16 @@ __device__ __forceinline__ void cluster_sync_alive() {
 }
 
 // Stage ring: normally two CTAs per SM with three 32 KiB stages each.  The clustered partial step with few
-// clusters (batch 1) is a pure latency chain on half-empty SMs: its "wide" form takes the whole SM, keeps six
+// clusters (batch 1) is a pure latency chain on half-empty SMs: its "wide" form takes the whole SM, keeps five
 // tiles in flight and splits the tiles over five pairs of MMA warps.  With many clusters the narrow form wins
 // (two CTAs per SM place clusters more freely and overlap each other's latencies).
 template <int kMode, bool kWideT>
 struct Ring {
   static constexpr bool kWide = kWideT && (kMode == kModeCluster || kMode == kModeClusterAppend);
-  static constexpr int kStg = kWide ? 6 : kStages;
+  // (stages = groups of MMA warps in the wide form: tile t and the tile t + kStg that reuses its stage must
+  // belong to the same group, because a warp may only wait for a stage's second phase after it has seen the
+  // first - a parity wait on a phase the warp has skipped returns at once)
+  static constexpr int kStg = kWide ? 5 : kStages;
   static constexpr int kMinBlocks = kWide ? 1 : 2;
   // The clustered partial step is bound by the length of one warp's MMA / softmax instruction chain, not by
   // bandwidth: five pairs of MMA warps take alternate tiles, so that a chunk of up to five tiles (a small
@@ -185,6 +188,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   constexpr int kBand = 16 * kNB;
   constexpr int kWT = kTile / kBand;                // warps per tile
   constexpr int kGroups = kMW / kWT;                // groups of warps that take alternate tiles
+  static_assert(kStg % kGroups == 0, "a stage must always be consumed by the same group of warps");
   auto consumer_bar = [] { consumer_bar_n<32 * kMW>(); };
   extern __shared__ uint8_t smem_raw[];
   __shared__ int s_last;

@@ -279,6 +279,33 @@ def test_small_step_every_cluster_shape(mods, n_small):
         check_out(out[b], want, f"small step n={n}")
 
 
+@pytest.mark.parametrize("n_small,n_q,n_kv", [(2560, 32, 8), (3073, 32, 8), (4096 + 9, 32, 8), (8000, 32, 8),
+                                              (5000, 28, 4), (8180, 8, 1)])
+def test_small_step_long_small_cache_one_sequence(mods, n_small, n_q, n_kv):
+    """One sequence, few KV heads: the latency-bound form of the clustered step (one CTA per SM, groups of MMA warps
+    on alternate tiles) with chunks longer than its ring, so every stage is used more than once; plain and with
+    the append fused in, against the oracle."""
+    rkv, runner, synth = mods
+    ctx, st, cache, q = make_layer(mods, [n_small], [n_small], n_q, n_kv, seed=300 + n_small, poison=True)
+    st.refresh(q)                                   # K = L: the small cache is the whole cache
+    out = st.partial(q).clone()
+    want, _, _, _ = oracle_full(cache, 0, n_small, q[0], n_kv, n_small)
+    check_out(out[0], want, f"small step n={n_small}")
+    g = torch.Generator(device=q.device); g.manual_seed(n_small)
+    for step in range(2):
+        q2 = torch.randn(q.shape, generator=g, device=q.device).to(torch.bfloat16)
+        kn = torch.randn((1, n_kv, 128), generator=g, device=q.device).to(torch.bfloat16)
+        vn = torch.randn((1, n_kv, 128), generator=g, device=q.device).to(torch.bfloat16)
+        out2 = st.append_partial(q2, kn, vn).clone()
+        n = int(st.small.len[0])
+        assert n == n_small + step + 1
+        k = O.bf16_bits_to_f64(host_heads(st.small, 0, n_kv, "k")[:, :n])
+        v = O.bf16_bits_to_f64(host_heads(st.small, 0, n_kv, "v")[:, :n])
+        want2, _, _ = O.decode_attention(O.bf16_bits_to_f64(bits(q2[0])), k, v)
+        check_out(out2[0], want2, f"fused step {step} n={n}")
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("n_small", [0, 1, 63, 64, 127, 128, 320, 639, 640, 2047])
 def test_fused_append_small_step_equals_append_then_small_step(mods, n_small):
     """rkv_append_small_step against the two separate calls on twin caches: same rows, lengths, flags, output.
