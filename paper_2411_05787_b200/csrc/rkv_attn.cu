@@ -22,8 +22,9 @@
 //                  score-only variant streams K alone: logits and softmax statistics);
 //   partial step   (a) the CTAs of one (sequence, KV head) form a thread-block cluster:
 //                  each pushes its slice of the partial output into the peer that owns
-//                  that slice through distributed shared memory, one cluster barrier,
-//                  each CTA finishes 128/C channels of every head;
+//                  that slice through distributed shared memory, with stores that credit
+//                  an mbarrier of the receiver (no cluster barrier behind the dependency
+//                  wait); each CTA finishes 128/C channels of every head;
 //                  (b) long small caches: partials to the workspace, folded by the last
 //                  CTA of each (sequence, KV head) to arrive (atomic ticket, no spin).
 // The clustered partial step and the full step's pass can take the append with them
@@ -140,14 +141,18 @@ __device__ __forceinline__ void st_shared_v2(uint32_t addr, uint2 v) {
 __device__ __forceinline__ void st_keep_f2(float* addr, float a, float b, uint64_t policy) {
   asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(addr), "f"(a), "f"(b), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void st_cluster_f32x4(uint32_t addr, float4 v) {
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+// Store into a peer CTA's shared memory that also credits the bytes to an mbarrier of that peer: data and the
+// "it has arrived" signal travel together, one way.
+__device__ __forceinline__ void st_async_f32x4(uint32_t addr, float4 v, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+               "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar)
                : "memory");
 }
-__device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+__device__ __forceinline__ void st_async_f32x2(uint32_t addr, float a, float b, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(addr),
+               "f"(a), "f"(b), "r"(remote_bar)
+               : "memory");
 }
-// Cluster barrier (all five warps of every CTA of the cluster arrive).
 __device__ __forceinline__ void cluster_sync_alive() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -200,11 +205,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t bar_full = smem_base + kStg * kStageBytes;
   const uint32_t bar_empty = bar_full + 8 * kStg;
+  const uint32_t bar_recv = bar_empty + 8 * kStg;   // cluster mode: completes when every peer's slice has arrived
   if (tid == 0) {
     for (int s = 0; s < kStg; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, kWT);   // one arrival per MMA warp that reads the tile
     }
+    if (kCluster) mbar_init(bar_recv, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid == 32 * kMW) {
@@ -222,6 +229,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   const int cap = __ldg(p.cap + b);
   const int64_t roff = __ldg(p.row_offset + b);
   __syncthreads();   // barrier initialisation (above) is visible to every warp
+  if (kCluster) {
+    // The receive barrier expects, from every CTA of the cluster, its slice of the partial outputs (G heads x
+    // 128 / C channels) and its (m, l) of all eight head slots.  It is armed before the one cluster-wide barrier
+    // of the kernel, which sits up here, above the dependency wait, where it costs nothing: behind it every
+    // peer's receive barrier exists, and the merge needs no further barrier - the pushes carry their own signal.
+    if (gridDim.x > 1) {
+      if (tid == 0) mbar_expect_tx(bar_recv, (uint32_t)(p.group * kHeadDim * 4 + (int)gridDim.x * kMaxGroup * 8));
+      cluster_sync_alive();
+    }
+  }
 
   // One tile = K (and V) rows [y, y + 64) into stage t % kStg, completion on that stage's barrier.
   auto issue_tile = [&](int t, int64_t row_first, uint64_t policy) {
@@ -401,10 +418,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         }
         issue_tile(t, row0, policy);
       }
-    }
-    if (kCluster) {   // stay until the peers have pushed: every warp of the cluster meets at one barrier
-      __syncwarp();
-      cluster_sync_alive();
     }
     return;
   }
@@ -642,6 +655,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     const int C = (int)gridDim.x;                       // cluster size = CTAs per (sequence, KV head): 1, 2, 4 or 8
     const int c_sh = __ffs(C) - 1;                      // C is a power of two: shifts instead of divisions below
     const int dchunk = kHeadDim >> c_sh;                // channels of every head that one CTA finishes
+    if (C == 1) {   // a "cluster" of one: nothing to exchange (and no remote stores from a launch without clusters)
+      take_len_ticket();
+      if (!ok) return;
+#pragma unroll
+      for (int it = 0; it < kIt; ++it) {
+        const int item = tid + it * kNT;
+        if (item < n_items) {
+          const int h = item >> 5, d4 = (item & 31) * 4;
+          float Mh, Lh;
+          head_ml(h, Mh, Lh);
+          const float inv = __fdividef(1.f, Lh);
+          uint2 o2;
+          o2.x = pack_bf16(acc4[it].x * inv, acc4[it].y * inv);
+          o2.y = pack_bf16(acc4[it].z * inv, acc4[it].w * inv);
+          *reinterpret_cast<uint2*>(out + h * kHeadDim + d4) = o2;
+        }
+      }
+      return;
+    }
     float* recv = reinterpret_cast<float*>(smem_gen + kStg * kStageBytes + 16 * kStg + 16);
     float* recv_ml = recv + kMaxGroup * kHeadDim;       // [source CTA][head][2]
     const uint32_t recv_u32 = smem_u32(recv), recv_ml_u32 = smem_u32(recv_ml);
@@ -651,16 +683,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       if (item < n_items) {   // four channels never straddle two owners: dchunk is a multiple of 16
         const int h = item >> 5, d4 = (item & 31) * 4;
         const int owner = d4 >> (7 - c_sh), dd = d4 & (dchunk - 1);
-        st_cluster_f32x4(map_rank(recv_u32 + 4u * ((split * kMaxGroup + h) * dchunk + dd), owner), acc4[it]);
+        st_async_f32x4(map_rank(recv_u32 + 4u * ((split * kMaxGroup + h) * dchunk + dd), owner), acc4[it],
+                       map_rank(bar_recv, owner));
       }
     }
     if (tid < kMaxGroup * C) {   // (m, l) of head tid % 8 to peer tid / 8
       const int h = tid & 7, peer = tid >> 3;
       float Md, Ld;
       head_ml(h, Md, Ld);
-      st_cluster_f32x2(map_rank(recv_ml_u32 + 4u * ((split * kMaxGroup + h) * 2), peer), Md, Ld);
+      st_async_f32x2(map_rank(recv_ml_u32 + 4u * ((split * kMaxGroup + h) * 2), peer), Md, Ld, map_rank(bar_recv, peer));
     }
-    cluster_sync_alive();
+    if (!mbar_wait(bar_recv, 0)) {   // every peer's slice is here (bounded: a lost peer cannot hang the GPU)
+      if (lane == 0) atomicOr(p.status, kDevTimeoutBit);
+      ok = false;
+    }
     take_len_ticket();
     if (!ok) return;
     // This CTA finishes dchunk channels of every head: G * dchunk / 4 items of four channels, and C adjacent
