@@ -931,3 +931,90 @@ def test_bench_configuration_graph_replay_shared_context(mods):
                 check_out(st.out[0], states[l].small(bits(inputs[l][0][t, 0])), f"partial token {t} layer {l}")
     assert all(c.device_status() == 0 for c in ctxs)
     assert all(int(st.full.len[0]) == L + T and int(st.small.len[0]) == K + 1 for st in layers)
+
+
+def test_bench_configuration_dynamic_schedule_graph_replay(mods):
+    """The dynamic schedule as bench.py launches it (config-3 shape, reduced context): three layers that alternate
+    between two contexts; plain tokens = one rkv_append_small_step per layer; every fifth token the trigger, both
+    branches under its masks and the selection in the second stream (runner.OverlappedRefresh.run_checked); both
+    kinds replayed from CUDA graphs with the inputs staged in a device buffer.  Every layer, sequence and token
+    against the oracle."""
+    rkv, runner, synth = mods
+    dev = torch.device("cuda")
+    NL, T = 3, 16
+    w = synth.scaled(synth.config3(n_layers=NL, ctx=4096), steps=T)
+    B, Hq, Hkv, QC = w.batch, w.n_q_heads, w.n_kv_heads, w.stride
+    full_hint, small_hint = max(w.lens) + T + 1, max(w.k_small) + T + 2
+    ctxs = [rkv.Context(B, Hq, Hkv, full_hint, small_hint) for _ in range(2)]
+    q_stage = torch.zeros((NL, B, Hq, 128), dtype=torch.bfloat16, device=dev)
+    k_stage = torch.zeros((NL, B, Hkv, 128), dtype=torch.bfloat16, device=dev)
+    v_stage = torch.zeros((NL, B, Hkv, 128), dtype=torch.bfloat16, device=dev)
+    layers, inputs, states = [], [], []
+    for l in range(NL):
+        cache = synth.fill_layer(w, l, dev)
+        qs = synth.query_trajectory(w, l).to(dev)
+        kn, vn = synth.new_token_kv(w, l)
+        synth.plant_heavy(w, cache, l, qs[0])
+        layers.append(runner.LayerState(ctxs[l % 2], cache, list(w.k_small), T + 2, Hq, Hkv))
+        inputs.append((qs, kn.to(dev), vn.to(dev)))
+        states.append([O.SequenceState(host_heads(cache, b, Hkv, "k").copy(), host_heads(cache, b, Hkv, "v").copy(),
+                                       w.lens[b], w.k_small[b]) for b in range(B)])
+
+    def stage(t):
+        for l in range(NL):
+            q_stage[l].copy_(inputs[l][0][t]); k_stage[l].copy_(inputs[l][1][t]); v_stage[l].copy_(inputs[l][2][t])
+
+    overlapped = runner.OverlappedRefresh(layers)
+
+    def token(kind):
+        if kind == "check":
+            return overlapped.run_checked(lambda l: q_stage[l], lambda l: k_stage[l], lambda l: v_stage[l], w.threshold,
+                                          small_hint=small_hint, full_hint=full_hint)
+        for l, st in enumerate(layers):
+            st.append_partial(q_stage[l], k_stage[l], v_stage[l], max_len_hint=small_hint)
+
+    stage(0)
+    for l, st in enumerate(layers):          # initial small caches (eager; also builds the tensor maps)
+        st.refresh(q_stage[l], max_len_hint=full_hint)
+        for b in range(B):
+            o_out, o_score, _ = states[l][b].full(bits(inputs[l][0][0, b]))
+            check_out(st.out[b], o_out, f"init layer {l} seq {b}")
+            follow_gpu_selection(st, states[l][b], b, o_score, w)
+    torch.cuda.synchronize()
+    graphs, side = {}, torch.cuda.Stream()
+    for kind in ("small", "check"):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(gr, stream=side):
+                token(kind)
+        graphs[kind] = gr
+    n_full = 0
+    for t in range(1, T + 1):
+        stage(t)
+        kind = "check" if t % QC == 0 else "small"
+        graphs[kind].replay()
+        torch.cuda.synchronize()
+        for l, st in enumerate(layers):
+            flags = st.flag.cpu().numpy()
+            for b in range(B):
+                state = states[l][b]
+                state.append(bits(inputs[l][1][t, b]), bits(inputs[l][2][t, b]))
+                qb = bits(inputs[l][0][t, b])
+                full_now = False
+                if kind == "check":
+                    want, cos = O.should_refresh(O.bf16_bits_to_f64(qb), state.q_last_full, w.threshold)
+                    if abs(cos - w.threshold) >= 1e-4:
+                        assert flags[b] == want, (t, l, b, cos)
+                    full_now = bool(flags[b])
+                if full_now:
+                    o_out, o_score, _ = state.full(qb)
+                    check_out(st.out[b], o_out, f"full step t={t} layer {l} seq {b}")
+                    follow_gpu_selection(st, state, b, o_score, w)
+                    n_full += 1
+                else:
+                    check_out(st.out[b], state.small(qb), f"partial step t={t} layer {l} seq {b}")
+    assert all(c.device_status() == 0 for c in ctxs)
+    assert n_full >= 1
+    for st in layers:
+        assert st.full.len.tolist() == [n + T for n in w.lens]
+
