@@ -260,7 +260,7 @@ def run_ours(args):
     dynamic = w.schedule == "dynamic"
     n_prof = 2 * S
     # tokens decoded over all phases: main loop, e2e loop, always-full loop, small-only loop, profiling
-    total_tokens = 2 * (args.steps + args.warmup) + 10 + 23 + 21 + 2 * S + n_prof + 8 + 2 * 24
+    total_tokens = 2 * (args.steps + args.warmup) + 10 + 23 + 21 + 4 * S + n_prof + 8 + 2 * 24
     wl = synth.scaled(w, steps=total_tokens)
     k_max = max(w.k_small)
     full_hint = max(w.lens) + total_tokens + 1
@@ -438,8 +438,10 @@ def run_ours(args):
     # no event bracket separates it from its neighbours
     ms_attn_only = timed(20, force_kind="attn_only")[0] if overlap else None
     run_tokens(1, always_full=True)                # a regular full token again: the small caches are rebuilt
-    run_tokens(1, always_full=True)
-    ms_small, _ = timed(S - 1, force_small=True)   # right after a full token: K .. K+S-2 rows
+    ms_small = 0.0
+    for _ in range(3):                             # three periods: the partial tokens between two full ones
+        run_tokens(1, always_full=True)
+        ms_small += timed(S - 1, force_small=True)[0] / 3.0   # right after a full token: K .. K+S-2 rows
     run_tokens(1, always_full=True)
     # ---- per-kernel device time: every launch bracketed by CUDA events on its stream (fixed-stride schedule,
     # two periods, every sequence active).  A spin kernel first keeps the GPU busy while the host enqueues, so
