@@ -169,6 +169,10 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   if (cluster) {   // 1, 2, 4 or 8 CTAs per (sequence, KV head), whole tiles each
     const int tiles = (n_max + rkv::kTile - 1) / rkv::kTile;
     gx = tiles >= 5 ? 8 : tiles >= 3 ? 4 : tiles >= 2 ? 2 : 1;
+    // with many (sequence, KV head) pairs one wave of CTAs is enough: fewer, longer CTAs per pair spend a smaller
+    // share of their time on the exchange inside the cluster
+    const int bg = ctx->cfg.n_seq * ctx->cfg.n_kv_heads;
+    while (gx > 1 && (int64_t)gx * bg > 2 * ctx->sm_count) gx >>= 1;
     p.chunk = ((tiles + gx - 1) / gx) * rkv::kTile;
   } else {
     p.chunk = choose_chunk(ctx, n_max, logits, &gx);
