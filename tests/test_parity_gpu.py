@@ -829,13 +829,16 @@ def test_config3_full_size_single_step(mods):
     run_trajectory(mods, w, 0, seqs=[0, 3])
 
 
-def test_config4_ragged_sampled_sequences(mods):
-    """Ragged batch of 16 (lengths 8K..128K): shortest, median and longest sequence against the oracle."""
+@pytest.mark.parametrize("fused,overlapped", [(False, False), (True, True)])
+def test_config4_ragged_sampled_sequences(mods, fused, overlapped):
+    """Ragged batch of 16 (lengths 8K..128K): shortest, median and longest sequence against the oracle; the second
+    variant in the calls bench.py makes (append fused into the partial step - two CTAs per (sequence, KV head) at
+    this batch size - and the full step in two halves on two streams)."""
     rkv, runner, synth = mods
     w = synth.scaled(synth.config4(n_layers=1), steps=11)
     order = np.argsort(w.lens)
     seqs = [int(order[0]), int(order[len(order) // 2]), int(order[-1])]
-    n_full = run_trajectory(mods, w, 0, seqs=seqs)
+    n_full = run_trajectory(mods, w, 0, seqs=seqs, fused=fused, overlapped=overlapped)
     assert all(v == 1 for v in n_full.values())
 
 
