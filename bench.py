@@ -488,6 +488,16 @@ def run_ours(args):
     kern["gather"]["gbs"] = 2 * sum(w.k_small) * Hkv * 512.0 / (kern["gather"]["avg_us"] * 1e-6) / 1e9
     full_step_us = attn_us + kern["select"]["avg_us"]
 
+    # The kernel's average launch duration: CUDA events around a region of 20 tokens in which the attention passes
+    # of all layers follow each other on one stream (each with its short fold kernel, whose time stays in the
+    # figure: a lower bound for the pass itself).  Without that loop: one launch alone between two events.
+    if ms_attn_only:
+        achieved_main = kv_bytes_full / (ms_attn_only * 1e-3 / (20 * world) / NL) / 1e9
+        how_main = ("CUDA events around 20 tokens x %d layers of rkv_append_full_attention launched back to back on one "
+                    "stream; bytes / (region / launches), the fold kernel's time included" % NL)
+    else:
+        achieved_main = achieved
+        how_main = "one launch alone between two CUDA events, averaged over the profiling pass"
     result = {
         "metric": METRIC, "value": us_per_token, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": False, "scaling": "weak",
@@ -499,14 +509,15 @@ def run_ours(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": "attn_kernel<full> (full-cache attention + score logits, the token's "
                                                "append fused in)",
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "achieved": achieved_main, "peak": peak, "unit": "GB/s", "frac": achieved_main / peak,
                      "peak_source": peak_src,
+                     "how": how_main,
+                     # one launch alone between two CUDA events (carries the launch and drain latency of a kernel
+                     # that nothing overlaps)
+                     "achieved_single_launch": achieved, "frac_single_launch": achieved / peak,
                      "traffic": (kv_bytes_full * ATTN_FULL_TRAFFIC_PER_KV_BYTE
                                  if ATTN_FULL_TRAFFIC_PER_KV_BYTE and args.workload == "cfg2" else None),
-                     "algorithmic_bytes_per_launch": kv_bytes_full,
-                     # lower bound from launches run back to back in a graph (the fold kernel's time is in it)
-                     "achieved_back_to_back": (kv_bytes_full / (ms_attn_only * 1e-3 / (20 * world) / NL) / 1e9
-                                               if ms_attn_only else None)},
+                     "algorithmic_bytes_per_launch": kv_bytes_full},
         "detail": {
             "always_full_us_per_token": full_token_us,
             "refresh_speedup_vs_always_full": full_token_us / us_per_token,
