@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(128) fold_kernel(const float* __restrict__ par
                                                    const int32_t* __restrict__ active, __nv_bfloat16* __restrict__ out,
                                                    int n_q_heads, int n_kv_heads, int group, int chunk, int max_splits,
                                                    int max_len) {
-  constexpr int kU = 8;   // splits per warp in the first batch of loads (4 * kU = 32 splits)
+  constexpr int kU = 10;  // splits per warp in the first batch of loads (4 * kU = 40 splits: one batch at batch 1, L = 32K)
   constexpr float kLog2e = 1.4426950408889634f;
   const int h = blockIdx.x >> 2, c = (blockIdx.x & 3) * 32 + (threadIdx.x & 31);
   const int g = blockIdx.y, b = blockIdx.z, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
