@@ -369,7 +369,7 @@ static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cac
     {
       LaunchScope scope(ctx, st, RKV_KERNEL_FOLD);
       e = rkv::launch_fold(ctx->partials, ctx->ml_t, full->len, full->cap, active, out, ctx->cfg.n_seq,
-                           ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, chunk, ctx->max_splits, n_max, st);
+                           ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, chunk, ctx->max_splits, n_max, gx, st);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "fold launch");
     ctx->launches += 1;

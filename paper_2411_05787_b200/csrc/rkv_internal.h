@@ -117,7 +117,7 @@ cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, C
                           cudaStream_t st);
 cudaError_t launch_fold(const float* partials, const float* ml_t, const int32_t* len, const int32_t* cap,
                         const int32_t* active, void* out, int n_seq, int n_q_heads, int n_kv_heads, int chunk,
-                        int max_splits, int max_len, cudaStream_t st);
+                        int max_splits, int max_len, int grid_splits, cudaStream_t st);
 cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, int32_t* keep,
                            float* sim, int n_seq, int n_q_heads, cudaStream_t st);
 // Launch with optional programmatic dependent launch (the kernel may start while its predecessor on

@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(128) fold_kernel(const float* __restrict__ par
                                                    const int32_t* __restrict__ len, const int32_t* __restrict__ cap,
                                                    const int32_t* __restrict__ active, __nv_bfloat16* __restrict__ out,
                                                    int n_q_heads, int n_kv_heads, int group, int chunk, int max_splits,
-                                                   int max_len) {
+                                                   int max_len, int grid_splits) {
   constexpr int kU = 10;  // splits per warp in the first batch of loads (4 * kU = 40 splits: one batch at batch 1, L = 32K)
   constexpr float kLog2e = 1.4426950408889634f;
   const int h = blockIdx.x >> 2, c = (blockIdx.x & 3) * 32 + (threadIdx.x & 31);
@@ -176,29 +176,42 @@ __global__ void __launch_bounds__(128) fold_kernel(const float* __restrict__ par
   __shared__ float sm_L;
   pdl_wait();
   pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
-  if (active != nullptr && __ldcg(active + b) == 0) return;
+  // One round trip: the sizes and every slot a CTA of the pass can have written (grid_splits of them; slots the
+  // current length does not reach hold older partials and are left out below, once the length is known).
+  const int act = active != nullptr ? __ldcg(active + b) : 1;
   int n = __ldcg(len + b);
   const int cp = __ldg(cap + b), lim = cp < max_len ? cp : max_len;
-  n = n < lim ? n : lim;            // the clamp of the streaming pass
-  if (n <= 0) return;               // nothing cached: the streaming pass has written zeros
-  const int n_splits = (n + chunk - 1) / chunk;
   const int64_t bg = (int64_t)b * n_kv_heads + g;
   const float* po = partials + bg * max_splits * PartialLayout::kFloats + h * kHeadDim + c;
   float v[kU];
 #pragma unroll
   for (int k = 0; k < kU; ++k) {
     const int s = warp + 4 * k;
-    v[k] = s < n_splits ? __ldcg(po + (int64_t)s * PartialLayout::kFloats) : 0.f;
+    v[k] = s < grid_splits ? __ldcg(po + (int64_t)s * PartialLayout::kFloats) : 0.f;
   }
-  if (warp == 0) {   // weights of all splits (at most kMaxSplits = 4 per lane), their sum of denominators
+  float m[4], l[4];
+  if (warp == 0) {   // (m, l) of all splits (at most kMaxSplits = 4 per lane)
     const float* pm = ml_t + bg * 16 * max_splits + (int64_t)h * max_splits;
     const float* pl = pm + (int64_t)kMaxGroup * max_splits;
-    float m[4], l[4], M = -INFINITY, L = 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int s = lane + 32 * i;
-      m[i] = s < n_splits ? __ldcg(pm + s) : -INFINITY;
-      l[i] = s < n_splits ? __ldcg(pl + s) : 0.f;
+      m[i] = s < grid_splits ? __ldcg(pm + s) : -INFINITY;
+      l[i] = s < grid_splits ? __ldcg(pl + s) : 0.f;
+    }
+  }
+  if (act == 0) return;
+  n = n < lim ? n : lim;            // the clamp of the streaming pass
+  if (n <= 0) return;               // nothing cached: the streaming pass has written zeros
+  const int n_splits = (n + chunk - 1) / chunk;
+  if (warp == 0) {   // weights of the splits in use, their sum of denominators
+    float M = -INFINITY, L = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (lane + 32 * i >= n_splits) {
+        m[i] = -INFINITY;
+        l[i] = 0.f;
+      }
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) M = fmaxf(M, m[i]);
@@ -307,10 +320,11 @@ cudaError_t launch_append(const void* k_new, const void* v_new, CacheDev full, C
 
 cudaError_t launch_fold(const float* partials, const float* ml_t, const int32_t* len, const int32_t* cap,
                         const int32_t* active, void* out, int n_seq, int n_q_heads, int n_kv_heads, int chunk,
-                        int max_splits, int max_len, cudaStream_t st) {
+                        int max_splits, int max_len, int grid_splits, cudaStream_t st) {
   const int group = n_q_heads / n_kv_heads;
   return launch_ex(fold_kernel, dim3(4 * group, n_kv_heads, n_seq), dim3(128), 0, st, 1, partials, ml_t, len, cap,
-                   active, static_cast<__nv_bfloat16*>(out), n_q_heads, n_kv_heads, group, chunk, max_splits, max_len);
+                   active, static_cast<__nv_bfloat16*>(out), n_q_heads, n_kv_heads, group, chunk, max_splits, max_len,
+                   grid_splits);
 }
 
 cudaError_t launch_trigger(const void* q_now, const void* q_last, float threshold, int32_t* flag, int32_t* keep,
