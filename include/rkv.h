@@ -129,7 +129,7 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*ho
                          void* q_last_full, int32_t max_len_hint, void* stream);
 
 /*
- * The two halves of rkv_full_step as calls of their own (Sec. 2.1: the full step's attention output is
+ * The two halves of rkv_full_step as calls of their own (Sec. 2.2: the full step's attention output is
  * what the decoder needs next; the refreshed partial cache is first read by the NEXT token's partial
  * step).  A caller that wants the attention output early - and the selection and the rebuild of C_p
  * off the layer's critical path, e.g. on a second stream under the next layer's work - calls
@@ -148,11 +148,11 @@ rkv_status rkv_full_step(rkv_ctx* ctx, const void* q, const rkv_cache* full /*ho
  */
 rkv_status rkv_full_attention(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
                               const int32_t* active, void* out, int32_t max_len_hint, void* stream);
-/* The same with the token's new rows appended to C_f first, in the same kernel (one launch; the result is
- * that of rkv_append(ctx, k_new, v_new, full, NULL) followed by rkv_full_attention): every sequence's
+/* The same with the token's new rows appended to C_f first, inside the streaming pass's kernel (no launch of
+ * its own; the result is that of rkv_append(ctx, k_new, v_new, full, NULL) followed by rkv_full_attention): every sequence's
  * cache grows by one row - inactive ones too, as in rkv_append - and the attention of the active ones
  * covers the new row.  max_len_hint bounds the lengths AFTER the append.  A cache already at capacity
- * sets RKV_DEV_APPEND_OVERFLOW and is attended as it is.  (Sec. 2.1: new KV pairs are appended to both
+ * sets RKV_DEV_APPEND_OVERFLOW and is attended as it is.  (Sec. 2.2: new KV pairs are appended to both
  * caches; the full step that follows rebuilds C_p, so only C_f needs the row here.) */
 rkv_status rkv_append_full_attention(rkv_ctx* ctx, const void* q, const void* k_new, const void* v_new,
                                      const rkv_cache* full /*host struct*/, const int32_t* active, void* out,
