@@ -24,8 +24,9 @@
  *  - Errors: every call returns an rkv_status.  Bad arguments are detected on
  *    the host before anything is launched.  Conditions only the device can
  *    see (append past capacity, a length above the configured maximum,
- *    a non-finite score) set bits in a sticky device status word and the
- *    offending access is skipped or clamped; nothing traps.
+ *    a non-finite score, a bounded wait that ran out) set bits in a sticky
+ *    device status word (RKV_DEV_*) and the offending access is skipped or
+ *    clamped; nothing traps.
  *
  * Cache layout (rkv_cache).  K and V are each ONE buffer of n_rows rows of 128
  * bf16 channels (256 bytes per row, base 16-byte aligned).  Sequence b,
@@ -61,6 +62,10 @@ typedef enum {
 #define RKV_DEV_LEN_CLAMPED 2     /* a seq_len exceeded cap or max_len and was clamped   */
 #define RKV_DEV_NONFINITE 4       /* a NaN/Inf attention logit was seen                  */
 #define RKV_DEV_BAD_INDEX 8       /* rkv_gather_small: index outside [0, len), row skipped*/
+#define RKV_DEV_TIMEOUT 16        /* a bounded wait inside an attention kernel (for a copy into shared memory,
+                                     or for a peer CTA's partial result) ran out: the out[] rows of that call
+                                     are not valid.  Never seen in a healthy run; the waits are bounded so that
+                                     a lost copy cannot hang the GPU                                          */
 
 /* score aggregation over the query heads of a group (Sec. 2.2 footnote; App. A.3, Table 6) */
 typedef enum { RKV_AGG_MAX = 0, RKV_AGG_MEAN = 1, RKV_AGG_FIRST = 2 } rkv_agg;
@@ -70,11 +75,11 @@ typedef struct {
   int32_t n_q_heads;     /* Hq                                                         */
   int32_t n_kv_heads;    /* Hkv; Hq % Hkv == 0, Hq / Hkv <= 8                          */
   int32_t head_dim;      /* must be 128                                                */
-  int32_t max_len;       /* largest full-cache length any call will see                */
+  int32_t max_len;       /* largest full-cache length any call will see (<= 327680)    */
   int32_t max_small;     /* largest small-cache length any call will see               */
   int32_t agg;           /* rkv_agg; RKV_AGG_MAX is the paper's rule                   */
   int32_t pool_kernel;   /* 1 = no pooling; odd w in 3..31 = the scores are max-pooled over w neighbouring
-                            positions before the top-K (App. A.1: 7); then max_len <= 163840          */
+                            positions before the top-K (App. A.1: 7)                                   */
   float softmax_scale;   /* 0 -> 1/sqrt(head_dim)                                      */
 } rkv_config;
 
@@ -283,8 +288,11 @@ rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_las
  * Of cfg only n_seq, n_q_heads, n_kv_heads, head_dim, max_small and softmax_scale are read.
  *
  * First call on a device: looks up the array's device address, sets the kernel's shared-memory
- * attribute and resolves the tensor-map encoder (host work, once per device, under a lock).  Make
- * that first call outside any stream capture.
+ * attribute and resolves the tensor-map encoder (host work, once per device, under a lock).  If the
+ * library's device code has not been loaded on that device yet, the CUDA runtime loads it during
+ * this first call, which is when the device memory for the code and for the array itself is taken;
+ * from the second call on, device memory use does not change.  Make that first call outside any
+ * stream capture.
  * Sharing: every call on a device uses the same array, which keeps the previous call's contents;
  * the call clears the tickets (and the built-in status word) on the stream before it launches.
  * Two calls that overlap on the GPU (different streams, no ordering) race on the array: order them.
@@ -346,13 +354,14 @@ rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
  *   total_us, launches   host arrays of RKV_KERNEL_KINDS entries
  */
 #define RKV_KERNEL_ATTN_FULL 0  /* full-cache attention + logit emission (rkv_full_step, 1st kernel) */
-#define RKV_KERNEL_SELECT 1     /* score finalisation + top-K            (rkv_full_step, 2nd kernel) */
+#define RKV_KERNEL_SELECT 1     /* top-K from the keys' histogram        (rkv_full_step, 3rd kernel) */
 #define RKV_KERNEL_ATTN_SMALL 2 /* small-cache attention                 (rkv_small_step)            */
 #define RKV_KERNEL_GATHER 3     /* rkv_gather_small                                                  */
 #define RKV_KERNEL_APPEND 4     /* rkv_append                                                        */
 #define RKV_KERNEL_TRIGGER 5    /* rkv_should_refresh                                                */
 #define RKV_KERNEL_FOLD 6       /* output from the split partials        (rkv_[append_]full_attention, 2nd kernel) */
-#define RKV_KERNEL_KINDS 7
+#define RKV_KERNEL_SCORE 7      /* logits -> scores, keys, histogram     (rkv_full_step, 2nd kernel) */
+#define RKV_KERNEL_KINDS 8
 rkv_status rkv_set_profiling(rkv_ctx* ctx, int32_t on);
 rkv_status rkv_get_profile(rkv_ctx* ctx, double* total_us /*host*/, int64_t* launches /*host*/);
 

@@ -12,6 +12,7 @@ namespace {
 
 using rkv::AttnParams;
 using rkv::CacheDev;
+using rkv::ScoreParams;
 using rkv::SelectParams;
 
 rkv::EncodeTiledFn g_encode = nullptr;
@@ -27,7 +28,6 @@ bool config_ok(const rkv_config* c, rkv_status* why) {
   if (c->head_dim != rkv::kHeadDim || c->n_q_heads / c->n_kv_heads > rkv::kMaxGroup ||
       c->agg < RKV_AGG_MAX || c->agg > RKV_AGG_FIRST || c->pool_kernel < 1 || c->pool_kernel > 31 ||
       c->pool_kernel % 2 == 0 ||
-      (c->pool_kernel > 1 && (int64_t)c->max_len > (int64_t)rkv::kSelectCluster * rkv::kSelectMaxKeysPerCtaPooled) ||
       (int64_t)c->max_len > (int64_t)rkv::kSelectCluster * rkv::kSelectMaxKeysPerCta ||
       (int64_t)c->n_seq * c->n_kv_heads > 65535 * 8) { *why = RKV_ERR_UNSUPPORTED; return false; }
   if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) { *why = RKV_ERR_INVALID_ARG; return false; }
@@ -39,7 +39,7 @@ int splits_for(const rkv_config* c) {
   return s < rkv::kMaxSplits ? (s < 1 ? 1 : s) : rkv::kMaxSplits;
 }
 
-struct WsLayout { size_t partials, ml_t, tickets, len_tickets, win_keys, logits, status, total; int64_t logit_stride; };
+struct WsLayout { size_t partials, ml_t, tickets, len_tickets, win_keys, keys, hist, logits, status, total; int64_t logit_stride; };
 
 WsLayout ws_layout(const rkv_config* c) {
   WsLayout w;
@@ -53,6 +53,8 @@ WsLayout ws_layout(const rkv_config* c) {
   w.tickets = off;  off = up(off + bg * sizeof(int32_t));
   w.len_tickets = off; off = up(off + (size_t)c->n_seq * sizeof(int32_t));
   w.win_keys = off; off = up(off + bg * (size_t)c->max_small * sizeof(uint32_t));
+  w.keys = off;     off = up(off + bg * (size_t)w.logit_stride * sizeof(uint32_t));
+  w.hist = off;     off = up(off + bg * (size_t)rkv::kSelectBins * sizeof(uint32_t));
   const int gp = group <= 4 ? 4 : 8;   // position-major logits, padded to a vector width
   w.logits = off;   off = up(off + bg * gp * (size_t)w.logit_stride * sizeof(float));
   w.status = off;   off = up(off + sizeof(int32_t));
@@ -335,6 +337,9 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.tickets);
   ctx->len_tickets = reinterpret_cast<int32_t*>(ctx->workspace + w.len_tickets);
   ctx->win_keys = reinterpret_cast<uint32_t*>(ctx->workspace + w.win_keys);
+  ctx->keys = reinterpret_cast<uint32_t*>(ctx->workspace + w.keys);
+  ctx->hist = reinterpret_cast<uint32_t*>(ctx->workspace + w.hist);   // zeroed with the rest of the workspace above
+  ctx->hist_dirty = false;
   ctx->logits = reinterpret_cast<float*>(ctx->workspace + w.logits);
   ctx->status = reinterpret_cast<int32_t*>(ctx->workspace + w.status);
   ctx->logit_stride = w.logit_stride;
@@ -390,45 +395,75 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   const int n_max = ctx->pending_full.n_max, chunk = ctx->pending_full.chunk, gx = ctx->pending_full.gx;
   if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
   ctx->pending_full.valid = false;
+  // two launches: the score pass over all positions (keys, scores, histogram; folds out[] when asked to), then
+  // the selection proper, one small cluster per (sequence, KV head)
+  const int bg = ctx->cfg.n_seq * ctx->cfg.n_kv_heads;
+  if (ctx->hist_dirty) {   // an earlier call launched its score pass but not its selection, which clears the histogram
+    cudaError_t e0 = cudaMemsetAsync(ctx->hist, 0, (size_t)bg * rkv::kSelectBins * sizeof(uint32_t), st);
+    if (e0 != cudaSuccess) return cuda_fail(ctx, e0, "histogram reset");
+    ctx->hist_dirty = false;
+  }
+  ScoreParams cp;
+  memset(&cp, 0, sizeof(cp));
+  cp.logits = ctx->logits;
+  cp.partials = ctx->partials;
+  cp.ml_t = ctx->ml_t;
+  cp.q = q;
+  cp.out = out;
+  cp.q_last_full = q_last_full;
+  cp.cap = full->cap;
+  cp.len = full->len;
+  cp.k_small = k_small;
+  cp.active = active;
+  cp.scores = scores;
+  cp.keys = ctx->keys;
+  cp.hist = ctx->hist;
+  cp.status = ctx->status;
+  cp.logit_stride = ctx->logit_stride;
+  cp.score_stride = score_stride;
+  cp.n_q_heads = ctx->cfg.n_q_heads;
+  cp.n_kv_heads = ctx->cfg.n_kv_heads;
+  cp.group = ctx->group;
+  cp.agg = ctx->cfg.agg;
+  cp.k_max = k_max;
+  cp.max_len = n_max;
+  cp.slice = rkv::score_slice_for(n_max, bg, ctx->sm_count);
+  cp.n_slices = (n_max + cp.slice - 1) / cp.slice;
+  cp.chunk = chunk;
+  cp.max_splits = ctx->max_splits;
+  cp.grid_splits = gx;
+  cp.pool_half = (ctx->cfg.pool_kernel - 1) / 2;
   SelectParams sp;
   memset(&sp, 0, sizeof(sp));
-  sp.logits = ctx->logits;
-  sp.partials = ctx->partials;
-  sp.ml_t = ctx->ml_t;
-  sp.q = q;
-  sp.out = out;
-  sp.q_last_full = q_last_full;
+  sp.keys = ctx->keys;
+  sp.hist = ctx->hist;
   sp.cap = full->cap;
-  sp.chunk = chunk;
-  sp.max_splits = ctx->max_splits;
   sp.len = full->len;
   sp.k_small = k_small;
   sp.active = active;
-  sp.scores = scores;
   sp.topk_idx = topk_idx;
   sp.win_keys = ctx->win_keys;
   sp.win_stride = ctx->cfg.max_small;
-  sp.status = ctx->status;
   sp.logit_stride = ctx->logit_stride;
-  sp.score_stride = score_stride;
-  sp.n_q_heads = ctx->cfg.n_q_heads;
   sp.n_kv_heads = ctx->cfg.n_kv_heads;
-  sp.group = ctx->group;
-  sp.agg = ctx->cfg.agg;
   sp.k_max = k_max;
   sp.max_len = n_max;
-  const int per = (n_max + rkv::kSelectCluster - 1) / rkv::kSelectCluster;
-  sp.per_cta = (per + 3) & ~3;
-  sp.grid_splits = gx;
-  sp.per_fixed = ctx->cfg.n_seq == 1 ? 1 : 0;
-  sp.pool_half = (ctx->cfg.pool_kernel - 1) / 2;
-  sp.keys_cap = rkv::select_keys_cap(sp.per_cta);
+  const int cluster = rkv::select_cluster_for(n_max);
+  sp.keys_per_thread = rkv::select_keys_per_thread(n_max, cluster);
   cudaError_t e;
+  ctx->hist_dirty = true;
+  {
+    LaunchScope scope(ctx, st, RKV_KERNEL_SCORE);
+    e = rkv::launch_score(cp, ctx->cfg.n_seq, st);
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "score launch");
+  ctx->launches += 1;
   {
     LaunchScope scope(ctx, st, RKV_KERNEL_SELECT);
-    e = rkv::launch_select(sp, ctx->cfg.n_seq, ctx->sm_count, st);
+    e = rkv::launch_select(sp, ctx->cfg.n_seq, cluster, st);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
+  ctx->hist_dirty = false;
   ctx->launches += 1;
   rkv::note_launch(st, nullptr, nullptr);
   return RKV_OK;

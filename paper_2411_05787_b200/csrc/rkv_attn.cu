@@ -413,7 +413,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       for (int t = n_spec; t < n_tiles; ++t) {
         const int s = t % kStg, use = t / kStg;
         if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1)) {
-          atomicOr(p.status, kDevTimeoutBit);
+          atomicOr(p.status, RKV_DEV_TIMEOUT);
           break;
         }
         issue_tile(t, row0, policy);
@@ -445,7 +445,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   for (int t = grp; t < n_wait; t += kGroups) {
     const int s = t % kStg;
     if (!mbar_wait(bar_full + 8 * s, (t / kStg) & 1)) {
-      if (lane == 0) atomicOr(p.status, kDevTimeoutBit);
+      if (lane == 0) atomicOr(p.status, RKV_DEV_TIMEOUT);
       ok = false;
       break;
     }
@@ -694,7 +694,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       st_async_f32x2(map_rank(recv_ml_u32 + 4u * ((split * kMaxGroup + h) * 2), peer), Md, Ld, map_rank(bar_recv, peer));
     }
     if (!mbar_wait(bar_recv, 0)) {   // every peer's slice is here (bounded: a lost peer cannot hang the GPU)
-      if (lane == 0) atomicOr(p.status, kDevTimeoutBit);
+      if (lane == 0) atomicOr(p.status, RKV_DEV_TIMEOUT);
       ok = false;
     }
     take_len_ticket();

@@ -22,8 +22,10 @@ constexpr int kAttnThreads = 160;      // 4 MMA warps + 1 copy warp
 constexpr int kSelectCluster = 8;      // CTAs that share one top-K problem
 constexpr int kAttnCluster = 8;        // most CTAs that share one (sequence, KV head) in the clustered partial step
 constexpr int kSelectThreads = 512;
-constexpr int kSelectMaxKeysPerCta = 40960;
-constexpr int kDevTimeoutBit = 16;     // internal: a bounded barrier wait ran out
+constexpr int kScoreThreads = 256;
+constexpr int kSelectMaxKeysPerCta = 40960;   // max_len <= kSelectCluster * this
+constexpr int kSelectBins = 4096;      // bins of the per-(sequence, KV head) score histogram in the workspace
+constexpr int kSelectMaxSlice = 8192;  // most positions one CTA of the score pass takes
 
 struct PartialLayout {                 // split-K partial of one (b, g, split)
   // o: [8 heads][128] fp32 unnormalised, then m[8], l[8]
@@ -67,31 +69,45 @@ struct AttnParams {
   int32_t max_evict;
 };
 
-struct SelectParams {
+// Score pass of the full step: logits -> keys (+ scores) and the histogram of the keys; optionally the fold of out[].
+struct ScoreParams {
   const float* logits;        // [B*Hkv][logit_stride][gp]
-  const float* partials;      // split partials written by the attention kernel
+  const float* partials;      // split partials written by the attention kernel (read when out != null)
   const float* ml_t;          // [B*Hkv][16][max_splits]: m of head j (j < 8) / l of head j - 8, contiguous over the splits
-  const void* q;              // bf16 [B][Hq][128]
-  void* out;                  // bf16 [B][Hq][128]
+  const void* q;              // bf16 [B][Hq][128] (read when q_last_full != null)
+  void* out;                  // bf16 [B][Hq][128], or null: the attention output has been folded already
   void* q_last_full;          // bf16 [B][Hq][128] or null
   const int32_t* cap;
   const int32_t* len;
   const int32_t* k_small;     // [B]
   const int32_t* active;
   float* scores;              // [B][Hkv][score_stride] or null
-  int32_t* topk_idx;          // [B][Hkv][k_max]
-  uint32_t* win_keys;         // [B*Hkv][win_stride]: key of every winner, in output order (for the eviction order)
-  int32_t win_stride;
+  uint32_t* keys;             // [B*Hkv][logit_stride]: key of every position
+  uint32_t* hist;             // [B*Hkv][kSelectBins]: all zero on entry
   int32_t* status;
   int64_t logit_stride, score_stride;
   int32_t n_q_heads, n_kv_heads, group, agg;
   int32_t k_max, max_len;
-  int32_t per_cta;            // positions per CTA of the cluster (from the host's length bound; multiple of 4)
+  int32_t slice, n_slices;    // positions per CTA; CTAs per (sequence, KV head)
   int32_t chunk, max_splits;  // split geometry of the attention launch that produced the partials
   int32_t grid_splits;        // CTAs per (sequence, KV head) that launch had
-  int32_t per_fixed;          // 1: slices are rank * per_cta (one sequence); 0: cut by each sequence's own length
   int32_t pool_half;          // (pool_kernel - 1) / 2
-  int32_t keys_cap;           // padded key capacity of a CTA (offset of the unpooled keys in shared memory)
+};
+
+struct SelectParams {
+  const uint32_t* keys;       // [B*Hkv][logit_stride]
+  uint32_t* hist;             // [B*Hkv][kSelectBins]: read, then cleared
+  const int32_t* cap;
+  const int32_t* len;
+  const int32_t* k_small;     // [B]
+  const int32_t* active;
+  int32_t* topk_idx;          // [B][Hkv][k_max]
+  uint32_t* win_keys;         // [B*Hkv][win_stride]: key of every winner, in output order (for the eviction order)
+  int32_t win_stride;
+  int64_t logit_stride;
+  int32_t n_kv_heads;
+  int32_t k_max, max_len;
+  int32_t keys_per_thread;    // keys per thread of a selection CTA (slices are fixed by the host's length bound)
 };
 
 struct CacheDev {
@@ -108,7 +124,11 @@ cudaError_t launch_attention_scores(const AttnParams& p, const CUtensorMap& tm_k
 cudaError_t launch_evict_order(const uint32_t* win_keys, int win_stride, const int32_t* k_small, int k_max,
                                const int32_t* full_len, const int32_t* active, int32_t* evict_order,
                                int32_t* evict_count, int max_evict, int n_seq, int n_kv_heads, cudaStream_t st);
-cudaError_t launch_select(const SelectParams& p, int n_seq, int sm_count, cudaStream_t st);
+cudaError_t launch_score(const ScoreParams& p, int n_seq, cudaStream_t st);
+cudaError_t launch_select(const SelectParams& p, int n_seq, int cluster, cudaStream_t st);
+int score_slice_for(int n_max, int problems, int sm_count);   // positions per CTA of the score pass
+int select_cluster_for(int n_max);                            // CTAs per (sequence, KV head) of the selection
+int select_keys_per_thread(int n_max, int cluster);           // keys per thread of a CTA of such a cluster
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
                           int32_t* status, cudaStream_t st);
@@ -173,9 +193,7 @@ bool early_read_safe(cudaStream_t st, const rkv_cache* c);
 cudaError_t prepare_attention();  // one-time function attributes (dynamic shared memory sizes)
 cudaError_t prepare_select();
 size_t attention_smem_bytes();
-size_t select_smem_bytes(int keys_per_cta, int pool_half);
-int select_keys_cap(int keys_per_cta);
-constexpr int kSelectMaxKeysPerCtaPooled = 20480;   // with pooling a CTA keeps two key arrays
+size_t select_smem_bytes(int keys_per_thread);
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -209,6 +227,9 @@ struct rkv_ctx {
   int32_t* tickets;
   int32_t* len_tickets;
   uint32_t* win_keys;
+  uint32_t* keys;      // key of every position of the last score pass
+  uint32_t* hist;      // per (sequence, KV head) histogram of those keys; all zero between selections
+  bool hist_dirty;     // a score pass was launched whose selection (which clears the histogram) was not
   float* logits;
   int32_t* status;
   int64_t launches;

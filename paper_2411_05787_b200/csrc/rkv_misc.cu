@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const int32_t* __restrict__
     uint4 kv[4], vv[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      if (j[u] >= n) {
+      if (j[u] >= n || j[u] < -1) {   // -1 is the padding of topk_idx; anything else outside [0, len) is flagged
         if (sub == 0) atomicOr(status, RKV_DEV_BAD_INDEX);
         j[u] = -1;
       }

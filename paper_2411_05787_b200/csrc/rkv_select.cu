@@ -1,34 +1,37 @@
-// Full-step epilogue: fold of the split-K partials, score finalisation and exact top-K selection.
-// One thread-block cluster (8 CTAs) per (sequence, KV head).
+// Full-step epilogue: score finalisation and exact top-K selection, as two kernels.
 //
 // RefreshKV (arXiv 2411.05787) Sec. 2.2: the partial cache is rebuilt from the
 // top-K positions of the current token's attention scores a_L; for grouped-query
 // attention the scores of the query heads of a group are aggregated by max
-// (footnote of Sec. 2.2; mean / first head are the ablation modes of App. A.3).
+// (footnote of Sec. 2.2; mean / first head are the ablation modes of App. A.3), and the
+// scores may be max-pooled over neighbouring positions first (App. A.1: kernel size 7).
 //
 // Input: the scaled logits s[j][h] (position-major, GP = 4 or 8 floats per position)
-// and the split partials the attention kernel wrote.  Every CTA derives the
-// log-sum-exp of all heads of the group from the partials and folds one eighth of
-// out[] of the group.  Then
+// and the softmax statistics (m, l) of the split partials the attention kernel wrote.
 //   ell[j] = agg_h (s[j][h] - LSE[h])            (log of the aggregated probability)
 // and the K largest scores are the K smallest keys  key = bits(max(-ell, 0)),  an
-// order-preserving 31-bit image of -ell (equal images are ties and go to the lower
-// position).  The kernel is a chain of latencies, so it is laid out to have few links:
-//   1  one round trip fetches the per-sequence sizes, the split weights, this CTA's
-//      slice of the partial outputs and its first logits, all at once;
-//   2  keys + a 2048-bin histogram (1/64 nat per bin) in shared memory (with neighbour max-pooling
-//      of the scores, App. A.1, the keys of a window are min-reduced first);
-//   3  cluster barrier; the eight histograms are merged through distributed shared
-//      memory and the bin T that holds the K-th key is located (while T holds more
-//      than 256 keys, a finer histogram over T's key range repeats this step);
-//   4  every CTA pushes its few keys of bin T into a flat array in all peers, plus
-//      its count of keys below T;
-//   5  cluster barrier; every CTA finds the threshold key by brute force over the
-//      <= 256 pushed keys and knows how many winners precede its slice;
-//   6  winners are written in ascending position order (deterministic, and the later
+// order-preserving 31-bit image of -ell (equal images are ties and go to the lower position).
+//
+// score_kernel   grid-wide and bandwidth-shaped: one CTA per slice of positions of one
+//                (sequence, KV head).  Every CTA derives the log-sum-exp of the group's
+//                heads from the split statistics, turns its logits into keys (written to
+//                the workspace, 4 bytes per position, and - optionally - as scores) and counts
+//                them in the (sequence, KV head)'s histogram of 4096 bins (1/128 nat each) in
+//                global memory, one reduction per warp and distinct bin.
+//                Optional extra CTAs fold out[] from the split partials (rkv_full_step).
+// select_kernel  one thread-block cluster (1..8 CTAs) per (sequence, KV head), a short chain:
+//   1  one round trip fetches the sizes, the histogram and this CTA's slice of the keys;
+//   2  a block scan of the histogram locates the bin T that holds the K-th key (when T holds
+//      more than 256 keys - long runs of near-equal scores - finer histograms over T's key
+//      range, merged through distributed shared memory, narrow it down);
+//   3  every thread counts its keys below T (a block scan turns the counts into output
+//      offsets) and pushes its few keys inside T, with their positions, to all peers;
+//   4  one cluster barrier; every CTA ranks the <= 256 pushed (key, position) pairs by brute
+//      force - the ones of rank below the K-th's rank inside T are selected - and knows how
+//      many winners precede its slice;
+//   5  winners are written in ascending position order (deterministic, and the later
 //      gather walks the cache monotonically).
-// No global store precedes the first barrier (a release would wait for it); the
-// score output is regenerated from the keys between arrive and wait of the second.
+//      The histogram is cleared again by the cluster that used it.
 #include <cuda_bf16.h>
 
 #include <cstddef>
@@ -38,36 +41,25 @@
 namespace rkv {
 namespace {
 
-constexpr int NT = kSelectThreads;
+constexpr int NT = kSelectThreads;        // threads of a selection CTA
 constexpr int NW = NT / 32;
-constexpr int kBins = 2048;
-constexpr int kHistWords = kBins / 2;     // two 16-bit counters per word (a CTA holds at most 40960 keys)
+constexpr int NTS = kScoreThreads;        // threads of a score-pass CTA
+constexpr int kBins = kSelectBins;        // level-1 histogram: bins of 1/128 nat over -log p, the last one open-ended
+constexpr float kBinsPerNat = 128.f;
+constexpr int kFineBins = 2048;           // refinement histograms of the selection
+constexpr int kFineWords = kFineBins / 2; // packed 16-bit counters (a CTA holds fewer than 65536 keys)
 constexpr int kCandMax = 256;             // keys of the final bin that are resolved by brute force
-constexpr int kMaxPasses = 5;             // pass 0 + refinements of 11 bits each cover the 31-bit key
-constexpr int kOPre = 10;                 // partial-output values per thread fetched in the first round trip
+constexpr int kMaxPasses = 5;             // refinements of 11 bits each cover the 31-bit key
+constexpr int kFoldU = 10;                // splits per warp in the fold's first batch of loads
 constexpr uint32_t kWorstKey = 0x7f800000u;   // bits of +inf: probability 0, or a NaN score
 constexpr uint32_t kPadKey = 0xffffffffu;     // filler behind a CTA's last key: never a winner, never in a bin
 constexpr float kLog2eF = 1.4426950408889634f;
 constexpr float kLn2F = 0.6931471805599453f;
-static_assert(kSelectMaxKeysPerCta < 65536, "packed 16-bit histogram counters");
-static_assert(kSelectCluster == 8 && NT == 512, "merge and finish assume 8 CTAs of 16 warps");
-static_assert(kMaxSplits <= 128, "four weight loads per lane cover every split");
-
-struct SelectShared {
-  alignas(16) uint32_t hist[2][kHistWords];   // double-buffered: peers may still read the previous pass
-  alignas(16) uint32_t flat[kCandMax];        // final-bin keys of the whole cluster, in CTA order (pushed by peers)
-  alignas(16) float w[kMaxSplits * 8];        // w[s][h]: weight of split s for head h
-  alignas(16) float red[4][kHeadDim];
-  float lse[kMaxGroup], linv[kMaxGroup];
-  uint32_t below[kSelectCluster];             // pushed by CTA r: its keys below the final bin
-  uint32_t inbin[kSelectCluster];             // per CTA: its keys inside the located bin (from the merge)
-  uint32_t warp_a[NW];
-  uint32_t sel_bin, sel_want, sel_count;
-  uint32_t own_below, own_in, cand_fill;
-  uint32_t tau, ties, less_pre, eq_pre;
-  uint32_t bad;
-};
-static_assert(offsetof(SelectShared, hist) % 16 == 0 && offsetof(SelectShared, flat) % 16 == 0, "vector access");
+static_assert(kSelectMaxKeysPerCta + NT < 65536, "packed 16-bit counters in the refinement histograms and the tie scan");
+static_assert(NT == 512 && kBins == 8 * NT, "the histogram scan gives every thread 8 bins");
+static_assert(kFineWords == 2 * NT, "the refinement merge gives every thread two words");
+static_assert(kCandMax <= NT, "one thread per candidate when the flat list is built");
+static_assert(kMaxSplits <= 128 && NTS / 32 == kMaxGroup, "score pass: one warp per head, four split statistics per lane");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -76,11 +68,6 @@ __device__ __forceinline__ uint32_t map_rank(uint32_t local_addr, int rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
-}
-__device__ __forceinline__ uint4 ld_cluster_v4(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared::cluster.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
 }
 __device__ __forceinline__ void st_cluster(uint32_t addr, uint32_t v) {
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
@@ -123,170 +110,234 @@ __device__ __forceinline__ float warp_max_f(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
-
-// After a cluster barrier: merge hist[buf] of the eight CTAs and locate the bin that holds the
-// want-th smallest key.  Leaves sel_bin / sel_want (rank inside the bin) / sel_count (bin size) and
-// inbin[r] (CTA r's share of the bin) in shared memory.
-__device__ __forceinline__ void merge_locate(SelectShared* sh, int buf, uint32_t want) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  uint32_t m[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-  uint4 v[kSelectCluster];
-  if (tid < kHistWords / 4) {
-    const uint32_t local = smem_u32(&sh->hist[buf][tid * 4]);
-#pragma unroll
-    for (int r = 0; r < kSelectCluster; ++r) v[r] = ld_cluster_v4(map_rank(local, r));
-#pragma unroll
-    for (int r = 0; r < kSelectCluster; ++r) {
-      m[0] += v[r].x & 0xffffu; m[1] += v[r].x >> 16;
-      m[2] += v[r].y & 0xffffu; m[3] += v[r].y >> 16;
-      m[4] += v[r].z & 0xffffu; m[5] += v[r].z >> 16;
-      m[6] += v[r].w & 0xffffu; m[7] += v[r].w >> 16;
-    }
-  }
-  uint32_t sum = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) sum += m[i];
-  uint32_t inc = sum;
+__device__ __forceinline__ uint32_t warp_scan_incl(uint32_t v, int lane) {
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
+    const uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += t;
   }
-  if (lane == 31) sh->warp_a[warp] = inc;
-  __syncthreads();
-  if (tid < kHistWords / 4) {
-    uint32_t base = 0;
-#pragma unroll
-    for (int w2 = 0; w2 < kHistWords / 128; ++w2)
-      if (w2 < warp) base += sh->warp_a[w2];
-    const uint32_t excl = base + inc - sum;
-    if (excl < want && want <= excl + sum) {   // exactly one thread
-      uint32_t run = excl;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (run < want && want <= run + m[i]) {
-          sh->sel_bin = tid * 8 + i;
-          sh->sel_want = want - run;
-          sh->sel_count = m[i];
-#pragma unroll
-          for (int r = 0; r < kSelectCluster; ++r) {
-            const uint32_t word = (i >> 1) == 0 ? v[r].x : (i >> 1) == 1 ? v[r].y : (i >> 1) == 2 ? v[r].z : v[r].w;
-            sh->inbin[r] = (i & 1) ? (word >> 16) : (word & 0xffffu);
-          }
-        }
-        run += m[i];
-      }
-    }
-  }
-  __syncthreads();
+  return v;
 }
 
-// GP: floats per position in the logit scratch, 4 (G <= 4) or 8.  kMinBlocks = 2 trades a few spilled
-// registers for two resident CTAs per SM: with more clusters than one wave holds, their latency chains overlap.
-template <int GP, int kMinBlocks>
-__global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectParams p) {
-  extern __shared__ __align__(16) uint8_t smem_raw[];
-  const int rank = (int)cluster_rank();
-  const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  SelectShared* sh = reinterpret_cast<SelectShared*>(smem_raw);
-  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + ((sizeof(SelectShared) + 15) & ~size_t(15)));
-  for (int i = tid; i < 2 * kHistWords; i += NT) (&sh->hist[0][0])[i] = 0u;
-  if (tid == 0) {
-    sh->cand_fill = 0u;
-    sh->own_below = 0u;
-    sh->own_in = 0u;
-    sh->bad = 0u;
+// The sizes both kernels work with: the length clamped as the attention pass clamped it, the number of
+// positions to select, and whether there is anything to choose (only then is the histogram used at all,
+// and both kernels must agree on that: the one adds to it, the other clears it).
+struct Sizes {
+  int n, kk;
+  bool choose;
+};
+__device__ __forceinline__ Sizes clamp_sizes(int len, int cap, int max_len, int k_small, int k_max) {
+  Sizes s;
+  const int lim = cap < max_len ? cap : max_len;
+  s.n = len > lim ? lim : len;
+  if (s.n < 0) s.n = 0;
+  s.kk = k_small > k_max ? k_max : k_small;
+  if (s.kk > s.n) s.kk = s.n;
+  if (s.kk < 0) s.kk = 0;
+  s.choose = s.kk > 0 && s.kk < s.n;
+  return s;
+}
+
+// key of a position from its GP logits (heads >= G carry LSE = +inf and drop out)
+template <int GP, int AGG>
+__device__ __forceinline__ uint32_t make_key(const float* x, const float* lse_r, float inv_g, bool* bad) {
+  float ell;
+  if (AGG == RKV_AGG_MAX) {
+    ell = x[0] - lse_r[0];
+#pragma unroll
+    for (int h = 1; h < GP; ++h) ell = max_nan(ell, x[h] - lse_r[h]);
+  } else if (AGG == RKV_AGG_MEAN) {
+    float acc = 0.f;
+#pragma unroll
+    for (int h = 0; h < GP; ++h) acc += ex2f((x[h] - lse_r[h]) * kLog2eF);   // ex2(-inf) = 0 for heads >= G
+    ell = lg2f(acc * inv_g) * kLn2F;
+  } else {
+    ell = x[0] - lse_r[0];
   }
+  if (ell != ell) {
+    *bad = true;
+    return kWorstKey;
+  }
+  return __float_as_uint(fmaxf(-ell, 0.f)) & 0x7fffffffu;
+}
+__device__ __forceinline__ uint32_t bin_of(uint32_t key) {   // bin T holds T/128 <= -ell < (T+1)/128
+  return __float2uint_rz(fminf(__uint_as_float(key) * kBinsPerNat, (float)(kBins - 1)));
+}
+
+// ------------------------------------------------------------------------------------------------ score_kernel
+// GP: floats per position in the logit scratch, 4 (G <= 4) or 8.  kPool: neighbour max-pooling of the scores.
+// The kernel is a chain of a few hundred instructions per warp, so it is written for few of them.  The slice's
+// keys are counted in a shared-memory histogram, which ONE bulk reduction (cp.reduce.async.bulk: the copy engine
+// adds 16 KiB of counters to the (sequence, KV head)'s histogram in global memory) sends on: with bins this fine
+// a slice hardly ever puts two keys into one, and a reduction instruction per key costs an SM about two cycles.
+template <int GP, int AGG, bool kPool>
+__global__ void __launch_bounds__(NTS) score_kernel(const ScoreParams p) {
+  extern __shared__ __align__(16) uint32_t raw[];     // pooling only: unpooled keys of the slice and its halo
+  __shared__ __align__(128) uint32_t s_hist[kBins];
+  __shared__ uint32_t s_bmin, s_bmax;                 // range of bins the slice's keys fall into
+  __shared__ float s_lse[kMaxGroup];
+  __shared__ float s_e[kMaxSplits];
+  __shared__ float s_red[NTS / 32][32];
+  __shared__ float s_L;
+  const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = p.group;
-  const int bg = b * p.n_kv_heads + g;
-  // Positions per CTA: with one sequence the host fixes the slices from its length bound, so the first logits
-  // can be requested before the length arrives; with a batch (ragged lengths) each sequence is cut in eight
-  // by its own length once that is known, so that short sequences still use the whole cluster.
-  const bool per_fixed = p.per_fixed != 0;
-  int per = p.per_cta;
-  int lo = rank * per;
-  const float* pbase = p.partials + (int64_t)bg * p.max_splits * PartialLayout::kFloats;
-  const int half = p.pool_half;               // neighbour max-pooling of the scores over 2*half+1 positions (0: none)
-  // keys are made for positions lo-half .. lo+per+half-1 (the pooling window reaches into the neighbours' slices)
-  const float* lg = p.logits + ((int64_t)bg * p.logit_stride + lo - half) * GP;   // re-based below if the slices move
-  uint32_t* raw = half > 0 ? keys + p.keys_cap : keys;   // unpooled keys; the same array when there is no pooling
-  constexpr int U = 32 / GP;                  // positions per thread per round: all their loads are in flight together
+  const int64_t bg = (int64_t)b * p.n_kv_heads + g;
   const int gx = p.grid_splits;               // splits the attention launch had room for (>= the sequence's own count)
-  // slice of out[] this CTA folds: 16*G consecutive (head, channel) pairs of the group
-  const int o_local = tid & 127, sgrp = tid >> 7;
-  const bool o_on = o_local < 16 * G;
-  const bool fold_on = o_on && p.out != nullptr;   // the score-only step has no attention output to fold
-  const int o_flat = rank * 16 * G + o_local;
+
+  if ((int)blockIdx.x >= p.n_slices) {
+    // ---------------------------------------------------------------- extra CTAs: out[] from the split partials
+    // (flash-decoding merge: M = max_s m_s, w_s = exp(m_s - M), out = sum_s w_s O_s / sum_s w_s l_s).  One CTA
+    // per (head of the group, half of the channels); warp w takes the splits s = w (mod 4) of one 32-channel
+    // quarter; every load is issued before the first is used.
+    const int fx = (int)blockIdx.x - p.n_slices;
+    const int h = fx >> 1, quarter = (fx & 1) * 2 + (warp >> 2), w4 = warp & 3;
+    const int c = quarter * 32 + lane;
+    pdl_wait();
+    pdl_launch();
+    const int act = p.active != nullptr ? __ldcg(p.active + b) : 1;
+    const int len = __ldcg(p.len + b);
+    const int cap = __ldg(p.cap + b);
+    const float* po = p.partials + bg * p.max_splits * PartialLayout::kFloats + h * kHeadDim + c;
+    float v[kFoldU];
+#pragma unroll
+    for (int k = 0; k < kFoldU; ++k) {
+      const int s = w4 + 4 * k;
+      v[k] = s < gx ? __ldcg(po + (int64_t)s * PartialLayout::kFloats) : 0.f;
+    }
+    float m[4], l[4];
+    if (warp == 0) {
+      const float* pm = p.ml_t + bg * 16 * p.max_splits + (int64_t)h * p.max_splits;
+      const float* pl = pm + (int64_t)kMaxGroup * p.max_splits;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int s = lane + 32 * i;
+        m[i] = s < gx ? __ldcg(pm + s) : -INFINITY;
+        l[i] = s < gx ? __ldcg(pl + s) : 0.f;
+      }
+    }
+    if (act == 0) return;
+    const Sizes sz = clamp_sizes(len, cap, p.max_len, 0, 0);
+    if (sz.n <= 0) return;                    // nothing cached: the attention pass has written zeros
+    int n_splits = (sz.n + p.chunk - 1) / p.chunk;
+    if (n_splits > gx) n_splits = gx;
+    if (warp == 0) {
+      float M = -INFINITY, L = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (lane + 32 * i >= n_splits) {
+          m[i] = -INFINITY;
+          l[i] = 0.f;
+        }
+        M = fmaxf(M, m[i]);
+      }
+      M = warp_max_f(M);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float e = (m[i] == -INFINITY) ? 0.f : ex2f((m[i] - M) * kLog2eF);
+        L = fmaf(l[i], e, L);
+        s_e[lane + 32 * i] = e;
+      }
+      L = warp_sum_f(L);
+      if (lane == 0) s_L = L;
+    }
+    __syncthreads();
+    float acc = 0.f;
+#pragma unroll
+    for (int k = 0; k < kFoldU; ++k) {
+      const int s = w4 + 4 * k;
+      if (s < n_splits) acc = fmaf(v[k], s_e[s], acc);
+    }
+    for (int s = w4 + 4 * kFoldU; s < n_splits; s += 4)
+      acc = fmaf(__ldcg(po + (int64_t)s * PartialLayout::kFloats), s_e[s], acc);
+    s_red[warp][lane] = acc;
+    __syncthreads();
+    if (w4 == 0) {
+      const float sum = (s_red[warp][lane] + s_red[warp + 1][lane]) + (s_red[warp + 2][lane] + s_red[warp + 3][lane]);
+      static_cast<__nv_bfloat16*>(p.out)[((int64_t)b * p.n_q_heads + (int64_t)g * G + h) * kHeadDim + c] =
+          __float2bfloat16(sum / s_L);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- a slice of positions of one (sequence, KV head)
+  const int lo = (int)blockIdx.x * p.slice;
+  const int half = kPool ? p.pool_half : 0;
+#pragma unroll
+  for (int k = 0; k < kBins / 4 / NTS; ++k)
+    reinterpret_cast<uint4*>(s_hist)[k * NTS + tid] = make_uint4(0u, 0u, 0u, 0u);
+  if (tid == 0) {
+    s_bmin = kBins - 1;
+    s_bmax = 0u;
+  }
+  constexpr int U = 4;                        // positions per thread per round: all their loads are in flight together
+  // positions lo - half .. lo + slice + half - 1 become keys (the pooling window reaches into the neighbours' slices)
+  const int n_pos = p.slice + 2 * half;
+  const float4* lg = reinterpret_cast<const float4*>(p.logits + (bg * p.logit_stride + lo - half + tid) * GP);
+  // Addresses and predicates of everything the CTA reads are worked out above the dependency wait, so that
+  // behind it only the loads themselves are left to issue.
+  const int32_t* a_act = p.active != nullptr ? p.active + b : nullptr;
+  const int32_t* a_len = p.len + b;
+  const int32_t* a_cap = p.cap + b;
+  const int32_t* a_ks = p.k_small + b;
+  const float* a_ml = p.ml_t + (bg * 16 + warp) * p.max_splits + lane;   // warp h: (m, l) of head h, contiguous over the splits
+  const int ml_l = kMaxGroup * p.max_splits;
+  bool ml_on[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) ml_on[k] = lane + 32 * k < gx;
+  bool lg_on[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const int i = u * NTS + tid;
+    const int pos = lo - half + i;
+    lg_on[u] = i < n_pos && pos >= 0 && pos < p.logit_stride;
+  }
   const int64_t hrow0 = ((int64_t)b * p.n_q_heads + (int64_t)g * G) * kHeadDim;
+  const bool q_copy = blockIdx.x == 0 && p.q_last_full != nullptr && tid < G * 16;
+  const uint4* a_q = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.q) + hrow0) + tid;
   pdl_wait();
   pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
 
-  // ---------------------------------------------------------------- 1: everything the kernel reads, in one round trip
-  const int act = (p.active != nullptr) ? __ldcg(p.active + b) : 1;
-  int n = __ldcg(p.len + b);
-  const int cap = __ldcg(p.cap + b);
-  int kk = __ldcg(p.k_small + b);
-  float wm[4], wl[4];                          // warps 0..7: (m, l) of head `warp` for splits lane, lane+32, ...
+  // everything the CTA reads, in one round trip
+  const int act = (a_act != nullptr) ? __ldcg(a_act) : 1;
+  const int len = __ldcg(a_len);
+  const int cap = __ldg(a_cap);
+  const int k_small = __ldcg(a_ks);
+  float wm[4], wl[4];                          // (m, l) for splits lane, lane + 32, ...
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    const int s = lane + 32 * k;
-    const bool on = warp < kMaxGroup && s < gx;
-    const float* pt = p.ml_t + ((int64_t)bg * 16 + warp) * p.max_splits + s;   // contiguous over the splits
-    wm[k] = on ? __ldcg(pt) : -INFINITY;
-    wl[k] = on ? __ldcg(pt + (int64_t)kMaxGroup * p.max_splits) : 0.f;
+    wm[k] = ml_on[k] ? __ldcg(a_ml + 32 * k) : -INFINITY;
+    wl[k] = ml_on[k] ? __ldcg(a_ml + 32 * k + ml_l) : 0.f;
   }
-  float opre[kOPre];
+  float4 v[U][GP / 4];
 #pragma unroll
-  for (int k = 0; k < kOPre; ++k) {
-    const int s = sgrp + 4 * k;
-    opre[k] = (fold_on && s < gx) ? __ldcg(pbase + (int64_t)s * PartialLayout::kFloats + o_flat) : 0.f;
-  }
-  __nv_bfloat16 qv = __float2bfloat16(0.f);
-  if (p.q_last_full != nullptr && sgrp == 0 && o_on) qv = static_cast<const __nv_bfloat16*>(p.q)[hrow0 + o_flat];
-  float4 v[U][GP / 4], vnext[U][GP / 4];     // the round being turned into keys, and the one in flight behind it
-  auto load_round = [&](float4 (&dst)[U][GP / 4], int i0) {
+  for (int u = 0; u < U; ++u)
+#pragma unroll
+    for (int c = 0; c < GP / 4; ++c)
+      v[u][c] = lg_on[u] ? __ldcg(lg + (int64_t)(u * NTS) * (GP / 4) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  auto load_round = [&](int i0) {   // positions lo - half + i0 + u * NTS + tid (rounds after the first)
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * NT + tid;
+      const int i = i0 + u * NTS + tid;
       const int pos = lo - half + i;
-      const bool on = i < per + 2 * half && pos >= 0 && pos < p.logit_stride;
+      const bool on = i < n_pos && pos >= 0 && pos < p.logit_stride;
 #pragma unroll
       for (int c = 0; c < GP / 4; ++c)
-        dst[u][c] = on ? __ldcg(reinterpret_cast<const float4*>(lg + (int64_t)i * GP) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[u][c] = on ? __ldcg(lg + (int64_t)(i0 + u * NTS) * (GP / 4) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
-  if (per_fixed) load_round(v, 0);
+  uint4 qv = make_uint4(0u, 0u, 0u, 0u);
+  if (q_copy) qv = __ldcg(a_q);
 
-  if (act == 0) return;   // same decision in all CTAs of the cluster
-  {
-    const int lim = cap < p.max_len ? cap : p.max_len;
-    if (n > lim) n = lim;
-    if (n < 0) n = 0;
-  }
-  if (kk > p.k_max) kk = p.k_max;
-  if (kk > n) kk = n;
-  if (kk < 0) kk = 0;
-  int32_t* idx_out = p.topk_idx + (int64_t)bg * p.k_max;
-  if (n == 0) {   // the attention kernel has zeroed out[]
-    for (int i = rank * NT + tid; i < p.k_max; i += kSelectCluster * NT) idx_out[i] = -1;
-    return;
-  }
-  if (!per_fixed) {
-    per = (((n + kSelectCluster - 1) / kSelectCluster) + 3) & ~3;   // never above the host's per_cta (n <= its bound)
-    lo = rank * per;
-    lg = p.logits + ((int64_t)bg * p.logit_stride + lo - half) * GP;
-    load_round(v, 0);
-  }
-  const int cnt = (n - lo < 0) ? 0 : (n - lo < per ? n - lo : per);
-  const int R = (((cnt + NT - 1) / NT) + 3) & ~3;   // keys per thread in the ordered phases (multiple of 4)
-  const int cnt_pad = R * NT;
-  const bool all_selected = (kk == n);
-  const bool need_keys = (!all_selected && kk > 0) || p.scores != nullptr;
+  if (act == 0) return;
+  if (q_copy) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.q_last_full) + hrow0)[tid] = qv;
+  const Sizes sz = clamp_sizes(len, cap, p.max_len, k_small, p.k_max);
+  const int n = sz.n;
+  if (lo >= n) return;
   int n_splits = (n + p.chunk - 1) / p.chunk;
   if (n_splits > gx) n_splits = gx;
 
-  // ---------------------------------------------------------------- log-sum-exp and split weights, one warp per head
-  if (warp < kMaxGroup) {
+  // log-sum-exp of every head of the group, one warp per head
+  {
     float M = -INFINITY;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -299,336 +350,582 @@ __global__ void __launch_bounds__(NT, kMinBlocks) select_kernel(const SelectPara
     for (int k = 0; k < 4; ++k) {
       const float e = (wm[k] == -INFINITY) ? 0.f : ex2f((wm[k] - M) * kLog2eF);
       L = fmaf(wl[k], e, L);
-      if (lane + 32 * k < kMaxSplits) sh->w[(lane + 32 * k) * 8 + warp] = e;
     }
     L = warp_sum_f(L);
+    if (lane == 0) s_lse[warp] = M + lg2f(L) * kLn2F;
+  }
+  __syncthreads();
+  float lse_r[GP];
+#pragma unroll
+  for (int h = 0; h < GP; ++h) lse_r[h] = (h < G) ? s_lse[h] : INFINITY;
+  const float inv_g = 1.f / (float)G;
+  bool bad = false;
+  uint32_t* keys_out = p.keys + bg * p.logit_stride;
+  float* sc_out = p.scores != nullptr ? p.scores + bg * p.score_stride : nullptr;
+  uint32_t bmin = kBins - 1, bmax = 0u;
+  // a key leaves the kernel: the workspace copy, the optional score, the histogram
+  auto emit = [&](int pos, uint32_t key) {
+    keys_out[pos] = key;
+    if (sc_out != nullptr) sc_out[pos] = ex2f(-__uint_as_float(key) * kLog2eF);   // a NaN score has been flagged and reads as 0
+    if (sz.choose) {
+      const uint32_t bin = bin_of(key);
+      atomicAdd(&s_hist[bin], 1u);
+      bmin = min(bmin, bin);
+      bmax = max(bmax, bin);
+    }
+  };
+  for (int i0 = 0; i0 < n_pos; i0 += U * NTS) {
+    if (i0 > 0) load_round(i0);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * NTS + tid;
+      const int pos = lo - half + i;
+      if (i0 + u * NTS >= n_pos) continue;     // uniform over the CTA
+      const bool on = i < n_pos && pos >= 0 && pos < n;
+      uint32_t key = kPadKey;
+      if (on) key = make_key<GP, AGG>(reinterpret_cast<const float*>(&v[u][0]), lse_r, inv_g, &bad);
+      if (kPool) {
+        if (i < n_pos) raw[i] = key;
+      } else if (on) {
+        emit(pos, key);
+      }
+    }
+  }
+  if (kPool) {
+    // pooled score = max over the window = smallest key of the window (positions outside the sequence do not count)
+    __syncthreads();
+    for (int i = tid; i < p.slice; i += NTS) {
+      const int pos = lo + i;
+      if (pos >= n) break;
+      uint32_t key = kPadKey;
+      for (int d = 0; d <= 2 * half; ++d) key = min(key, raw[i + d]);
+      emit(pos, key);
+    }
+  }
+  // The counters go from the generic proxy (the atomics above) to the copy engine: fence, then barrier, then one
+  // issue - of the occupied range of bins only (16-byte granules), which is a fraction of the histogram.
+  if (sz.choose) {
+    bmin = __reduce_min_sync(0xffffffffu, bmin);
+    bmax = __reduce_max_sync(0xffffffffu, bmax);
     if (lane == 0) {
-      sh->lse[warp] = M + logf(L);
-      sh->linv[warp] = 1.f / L;
+      atomicMin(&s_bmin, bmin);
+      atomicMax(&s_bmax, bmax);
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  const int any_bad = __syncthreads_or(bad);
+  if (tid == 0) {
+    if (sz.choose) {
+      const uint32_t b0 = s_bmin & ~3u, b1 = (s_bmax | 3u) + 1u;
+      if (b1 > b0) {
+        asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.u32 [%0], [%1], %2;" ::"l"(p.hist + bg * kBins + b0),
+                     "r"(smem_u32(s_hist + b0)), "r"((uint32_t)((b1 - b0) * sizeof(uint32_t)))
+                     : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+    }
+    if (any_bad) atomicOr(p.status, RKV_DEV_NONFINITE);
+    // the CTA's shared memory must outlive the engine's read of it
+    if (sz.choose) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ select_kernel
+struct SelectShared {
+  alignas(16) unsigned long long seg[kSelectCluster][kCandMax];   // (key << 32 | position) of the final-bin keys of CTA r
+  alignas(16) unsigned long long flat[kCandMax];                  // the same in one array, in CTA order
+  alignas(16) uint32_t fine[2][kFineWords];   // refinement histograms, double-buffered: peers may still read the previous pass
+  int32_t mywin[kCandMax];                    // positions of this CTA's final-bin keys that are selected
+  uint32_t below[kSelectCluster];             // pushed by CTA r: its keys below the final bin
+  uint32_t candn[kSelectCluster];             // pushed by CTA r: its keys inside the final bin
+  uint32_t warp_a[NW];
+  uint32_t sel_bin, sel_want, sel_count;
+  uint32_t cand_fill, own_in, n_mywin, win_before;
+};
+
+// Merge fine[buf] of the C CTAs and locate the bin that holds the want-th smallest key.  Leaves sel_bin /
+// sel_want (rank inside the bin) / sel_count (bin size) in shared memory.  Called behind a cluster barrier.
+__device__ __noinline__ void merge_locate(SelectShared* sh, int buf, uint32_t want, int C) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t m[4] = {0u, 0u, 0u, 0u};
+  const uint32_t local = smem_u32(&sh->fine[buf][tid * 2]);
+  for (int r = 0; r < C; ++r) {
+    uint2 v;
+    if (C == 1) {
+      v = *reinterpret_cast<const uint2*>(&sh->fine[buf][tid * 2]);
+    } else {
+      asm volatile("ld.shared::cluster.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(map_rank(local, r)));
+    }
+    m[0] += v.x & 0xffffu; m[1] += v.x >> 16;
+    m[2] += v.y & 0xffffu; m[3] += v.y >> 16;
+  }
+  const uint32_t sum = (m[0] + m[1]) + (m[2] + m[3]);
+  const uint32_t inc = warp_scan_incl(sum, lane);
+  if (lane == 31) sh->warp_a[warp] = inc;
+  __syncthreads();
+  uint32_t base = 0;
+#pragma unroll
+  for (int w2 = 0; w2 < NW; ++w2)
+    if (w2 < warp) base += sh->warp_a[w2];
+  const uint32_t excl = base + inc - sum;
+  if (excl < want && want <= excl + sum) {   // exactly one thread
+    uint32_t run = excl;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (run < want && want <= run + m[i]) {
+        sh->sel_bin = tid * 4 + i;
+        sh->sel_want = want - run;
+        sh->sel_count = m[i];
+      }
+      run += m[i];
     }
   }
   __syncthreads();
+}
 
-  // this CTA's slice of out[] (and of the trigger's reference query); run where it hides a cluster barrier
-  auto fold_slice = [&] {
-    const int h = o_flat >> 7;
-    float acc = 0.f;
-    if (fold_on) {
-#pragma unroll
-      for (int k = 0; k < kOPre; ++k) {
-        const int s = sgrp + 4 * k;
-        if (s < n_splits) acc = fmaf(opre[k], sh->w[s * 8 + h], acc);
-      }
-      for (int s = sgrp + 4 * kOPre; s < n_splits; s += 4)
-        acc = fmaf(__ldcg(pbase + (int64_t)s * PartialLayout::kFloats + o_flat), sh->w[s * 8 + h], acc);
-    }
-    sh->red[sgrp][o_local] = acc;
-    __syncthreads();
-    if (sgrp == 0 && o_on) {
-      const float o = (sh->red[0][o_local] + sh->red[1][o_local]) + (sh->red[2][o_local] + sh->red[3][o_local]);
-      if (fold_on) static_cast<__nv_bfloat16*>(p.out)[hrow0 + o_flat] = __float2bfloat16(o * sh->linv[h]);
-      if (p.q_last_full != nullptr) static_cast<__nv_bfloat16*>(p.q_last_full)[hrow0 + o_flat] = qv;
-    }
-    for (int i = kk + rank * NT + tid; i < p.k_max; i += kSelectCluster * NT) idx_out[i] = -1;   // padding
-  };
-  // score[j] = exp(ell[j]) regenerated from the keys (a NaN score has been flagged and reads as 0)
-  auto write_scores = [&] {
-    if (p.scores != nullptr) {
-      float* sc = p.scores + (int64_t)bg * p.score_stride + lo;
-      for (int i = tid; i < cnt; i += NT) sc[i] = ex2f(-__uint_as_float(keys[i]) * kLog2eF);
-    }
-    if (tid == 0 && sh->bad != 0u) atomicOr(p.status, RKV_DEV_NONFINITE);
-  };
-
-  // ---------------------------------------------------------------- 2: keys and the pass-0 histogram
-  if (need_keys) {
-    float lse_r[GP];
-#pragma unroll
-    for (int h = 0; h < GP; ++h) lse_r[h] = (h < G) ? sh->lse[h] : INFINITY;
-    const int agg = p.agg;
-    const float inv_g = 1.f / (float)G;
-    bool bad = false;
-    const int n_raw = half > 0 ? (cnt > 0 ? cnt + 2 * half : 0) : cnt_pad;   // without pooling the padding is written here too
-    for (int i0 = 0; i0 < n_raw; i0 += U * NT) {
-      const bool more = i0 + U * NT < n_raw;
-      if (more) load_round(vnext, i0 + U * NT);   // overlaps the arithmetic below
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int i = i0 + u * NT + tid;
-        if (i >= n_raw) continue;
-        const float* x = reinterpret_cast<const float*>(&v[u][0]);
-        float ell;
-        if (agg == RKV_AGG_MAX) {   // heads >= G carry LSE = +inf and drop out of the max
-          ell = x[0] - lse_r[0];
-#pragma unroll
-          for (int h = 1; h < GP; ++h) ell = max_nan(ell, x[h] - lse_r[h]);
-        } else if (agg == RKV_AGG_MEAN) {
-          float acc = 0.f;
-#pragma unroll
-          for (int h = 0; h < GP; ++h) acc += ex2f((x[h] - lse_r[h]) * kLog2eF);   // ex2(-inf) = 0 for heads >= G
-          ell = lg2f(acc * inv_g) * kLn2F;
-        } else {
-          ell = x[0] - lse_r[0];
-        }
-        uint32_t key = kPadKey;
-        const int pos = lo - half + i;
-        if (i < cnt + 2 * half && pos >= 0 && pos < n) {
-          uint32_t bin;
-          if (ell != ell) {
-            bad = true;
-            key = kWorstKey;
-            bin = kBins - 1;
-          } else {
-            const float nl = fmaxf(-ell, 0.f);
-            key = __float_as_uint(nl) & 0x7fffffffu;
-            bin = __float2uint_rz(fminf(nl * 64.f, (float)(kBins - 1)));
-          }
-          if (!all_selected && half == 0) atomicAdd(&sh->hist[0][bin >> 1], 1u << ((bin & 1u) << 4));
-        }
-        raw[i] = key;
-      }
-      if (more) {
-#pragma unroll
-        for (int u = 0; u < U; ++u)
-#pragma unroll
-          for (int c = 0; c < GP / 4; ++c) v[u][c] = vnext[u][c];
-      }
-    }
-    if (bad) sh->bad = 1u;
-    if (half > 0) {
-      // pooled score = max over the window = smallest key of the window (App. A.1: kernel size 7 in the paper)
-      __syncthreads();
-      for (int i = tid; i < cnt_pad; i += NT) {
-        uint32_t key = kPadKey;
-        if (i < cnt) {
-          for (int d = 0; d <= 2 * half; ++d) key = min(key, raw[i + d]);
-          const uint32_t bin = __float2uint_rz(fminf(__uint_as_float(key) * 64.f, (float)(kBins - 1)));
-          if (!all_selected) atomicAdd(&sh->hist[0][bin >> 1], 1u << ((bin & 1u) << 4));
-        }
-        keys[i] = key;
-      }
-    }
-  }
-
-  if (all_selected || kk == 0) {   // uniform over the cluster: nothing to choose
-    __syncthreads();
-    fold_slice();
-    write_scores();
-    if (all_selected)
-      for (int i = tid; i < cnt; i += NT) {
-        idx_out[lo + i] = lo + i;
-        if (p.win_keys != nullptr && need_keys) p.win_keys[(int64_t)bg * p.win_stride + lo + i] = keys[i];
-      }
-    return;
-  }
-
-  // ---------------------------------------------------------------- 3: locate the bin of the kk-th smallest key
-  uint32_t lo_key = 0u, hi_key = kWorstKey, want = (uint32_t)kk, count = 0u;
-  int shb = 0;
+// Narrow [lo_key, hi_key] down with finer histograms until it holds at most kCandMax keys or a single key value.
+__device__ __noinline__ void refine(SelectShared* sh, const uint32_t* keys, int per, int C, uint32_t* lo_key_io,
+                                    uint32_t* hi_key_io, uint32_t* want_io, uint32_t* count_io) {
+  const int tid = threadIdx.x;
+  uint32_t lo_key = *lo_key_io, hi_key = *hi_key_io, want = *want_io, count = *count_io;
   for (int pass = 0; pass < kMaxPasses; ++pass) {
-    if (pass > 0) {   // refine inside [lo_key, hi_key]: bins of 2^shb key values
-      const uint32_t span = hi_key - lo_key;
-      shb = 32 - __clz(span) - 11;
-      if (shb < 0) shb = 0;
-      uint32_t* h = sh->hist[pass & 1];
-      for (int i = tid; i < kHistWords; i += NT) h[i] = 0u;
-      __syncthreads();
-      for (int i = tid; i < cnt; i += NT) {
-        const uint32_t key = keys[i];
-        if (key >= lo_key && key <= hi_key) {
-          const uint32_t bin = (key - lo_key) >> shb;
-          atomicAdd(&h[bin >> 1], 1u << ((bin & 1u) << 4));
-        }
+    const uint32_t span = hi_key - lo_key;
+    int shb = 32 - __clz(span) - 11;          // bins of 2^shb key values
+    if (shb < 0) shb = 0;
+    uint32_t* h = sh->fine[pass & 1];
+    for (int i = tid; i < kFineWords; i += NT) h[i] = 0u;
+    __syncthreads();
+    for (int i = tid; i < per; i += NT) {
+      const uint32_t key = keys[i];
+      if (key - lo_key <= span) {
+        const uint32_t bin = (key - lo_key) >> shb;
+        atomicAdd(&h[bin >> 1], 1u << ((bin & 1u) << 4));
       }
     }
-    cluster_arrive();
-    if (pass == 0) fold_slice();
-    cluster_wait();
-    merge_locate(sh, pass & 1, want);
+    if (C > 1) {
+      cluster_arrive();
+      cluster_wait();
+    } else {
+      __syncthreads();
+    }
+    merge_locate(sh, pass & 1, want, C);
     const uint32_t T = sh->sel_bin;
     want = sh->sel_want;
     count = sh->sel_count;
-    if (pass == 0) {   // bin T of pass 0 is  T/64 <= -ell < (T+1)/64  (the last bin is open-ended)
-      lo_key = __float_as_uint((float)T * (1.f / 64.f));
-      hi_key = (T == kBins - 1) ? kWorstKey : __float_as_uint((float)(T + 1) * (1.f / 64.f)) - 1u;
-    } else {
-      lo_key = lo_key + (T << shb);
-      const uint32_t top = lo_key + ((1u << shb) - 1u);
-      hi_key = top < hi_key ? top : hi_key;
-    }
+    lo_key = lo_key + (T << shb);
+    const uint32_t top = lo_key + ((1u << shb) - 1u);
+    hi_key = top < hi_key ? top : hi_key;
     if (count <= (uint32_t)kCandMax || lo_key == hi_key) break;
   }
-  // count > kCandMax here means the bin is a single key value shared by all its members
-  const bool ident = count > (uint32_t)kCandMax;
+  *lo_key_io = lo_key;
+  *hi_key_io = hi_key;
+  *want_io = want;
+  *count_io = count;
+}
 
-  // ---------------------------------------------------------------- 4: exchange the final bin
-  if (tid < kCandMax && tid >= (int)count) sh->flat[tid] = kPadKey;   // nobody pushes there: lets the search read vectors
-  uint32_t flat_base = 0;   // where this CTA's keys start in the flat array (CTA order)
-#pragma unroll
-  for (int r = 0; r < kSelectCluster; ++r)
-    if (r < rank) flat_base += sh->inbin[r];
-  const uint4* my_keys = reinterpret_cast<const uint4*>(keys + (size_t)tid * R);   // thread t owns keys [t*R, (t+1)*R)
-  {
-    uint32_t c_below = 0;
-    const uint32_t flat0 = smem_u32(&sh->flat[0]);
-    for (int j = 0; j < R / 4; ++j) {
-      const uint4 k4 = my_keys[j];
-      const uint32_t kv[4] = {k4.x, k4.y, k4.z, k4.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        c_below += (kv[e] < lo_key);
-        if (!ident && kv[e] >= lo_key && kv[e] <= hi_key) {   // rare: a handful per CTA
-          const uint32_t slot = flat_base + atomicAdd(&sh->cand_fill, 1u);
-          if (slot < (uint32_t)kCandMax) {
-#pragma unroll
-            for (int r = 0; r < kSelectCluster; ++r) st_cluster(map_rank(flat0 + 4u * slot, r), kv[e]);
-          }
-        }
-      }
-    }
-    c_below = warp_sum(c_below);
-    if (lane == 0 && c_below != 0u) atomicAdd(&sh->own_below, c_below);
-  }
-  __syncthreads();
-  if (tid < kSelectCluster) st_cluster(map_rank(smem_u32(&sh->below[rank]), tid), sh->own_below);
-  cluster_arrive();
-  write_scores();
-  cluster_wait();
-  // from here on nobody touches a peer's shared memory
-
-  // ---------------------------------------------------------------- 5: threshold key; winners before this slice
-  if (ident) {
-    if (tid == 0) {
-      sh->tau = lo_key;
-      sh->ties = want;
-      sh->less_pre = 0u;
-      sh->eq_pre = flat_base;
-    }
-  } else {
-    // P threads share one candidate (P a power of two, P * count <= 512): each counts over 1/P of the flat array
-    int lp = 0;                                   // log2(P)
-    while (lp < 5 && ((int)count << (lp + 1)) <= NT) ++lp;
-    const int ci = tid >> lp, part = tid & ((1 << lp) - 1);
-    if (ci < (int)count) {                        // whole groups of P lanes take this branch together
-      const int len = ((((int)count + (1 << lp) - 1) >> lp) + 3) & ~3;   // a multiple of four: 16-byte reads
-      const int j0 = part * len;
-      const uint32_t c = sh->flat[ci];
-      uint32_t less = 0, eq = 0, less_p = 0, eq_p = 0;
-      for (int j = j0; j < j0 + len && j < kCandMax; j += 4) {
-        const uint4 x4 = *reinterpret_cast<const uint4*>(&sh->flat[j]);
-        const uint32_t xs[4] = {x4.x, x4.y, x4.z, x4.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const bool pre = j + e < (int)flat_base;
-          less += (xs[e] < c);
-          eq += (xs[e] == c);
-          less_p += (pre && xs[e] < c);
-          eq_p += (pre && xs[e] == c);
-        }
-      }
-      const uint32_t gmask = __activemask();
-      for (int o = 1; o < (1 << lp); o <<= 1) {
-        less += __shfl_xor_sync(gmask, less, o);
-        eq += __shfl_xor_sync(gmask, eq, o);
-        less_p += __shfl_xor_sync(gmask, less_p, o);
-        eq_p += __shfl_xor_sync(gmask, eq_p, o);
-      }
-      if (part == 0 && less < want && want <= less + eq) {
-        // every thread that holds the threshold value writes the same four numbers
-        sh->tau = c;
-        sh->ties = want - less;
-        sh->less_pre = less_p;
-        sh->eq_pre = eq_p;
-      }
-    }
-  }
-  __syncthreads();
-  const uint32_t tau = sh->tau, ties_to_take = sh->ties;
-  uint32_t winners_before = sh->less_pre + (sh->eq_pre < ties_to_take ? sh->eq_pre : ties_to_take);
-#pragma unroll
-  for (int r = 0; r < kSelectCluster; ++r)
-    if (r < rank) winners_before += sh->below[r];
-  const uint32_t ties_before = sh->eq_pre;
-
-  // ---------------------------------------------------------------- 6: ordered output
+// Output when the final bin is one key value shared by more than kCandMax keys (long runs of equal scores): the
+// keys below it win, and of the equal ones the first ties_to_take in position order, cluster-wide.
+__device__ __noinline__ void write_ties(SelectShared* sh, const uint32_t* my, int R, int first, uint32_t tau,
+                                        uint32_t ties_to_take, uint32_t ties_before, uint32_t below_before, int kk,
+                                        int32_t* idx_out, uint32_t* win_out) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t c_less = 0, c_eq = 0;
-  for (int j = 0; j < R / 4; ++j) {
-    const uint4 k4 = my_keys[j];
-    c_less += (k4.x < tau) + (k4.y < tau) + (k4.z < tau) + (k4.w < tau);
-    c_eq += (k4.x == tau) + (k4.y == tau) + (k4.z == tau) + (k4.w == tau);
+  for (int j = 0; j < R; ++j) {
+    const uint32_t key = my[j];
+    c_less += key < tau;
+    c_eq += key == tau;
   }
   // exclusive block scan of both counts at once (each total fits 16 bits)
   const uint32_t packed = c_less | (c_eq << 16);
-  uint32_t inc = packed;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
+  const uint32_t inc = warp_scan_incl(packed, lane);
+  __syncthreads();   // warp_a may still be read by the scan before the exchange
   if (lane == 31) sh->warp_a[warp] = inc;
   __syncthreads();
   uint32_t wbase = (lane < warp) ? sh->warp_a[lane] : 0u;   // NW = 16 <= 32 lanes
   wbase = warp_sum(wbase);
   const uint32_t excl = wbase + inc - packed;
-  const uint32_t e_less = excl & 0xffffu;
   uint32_t eq_seen = ties_before + (excl >> 16);
-  // ties are kept in position order: the first ties_to_take of them (cluster-wide) win
-  uint32_t offs = winners_before + e_less +
-                  ((eq_seen < ties_to_take ? eq_seen : ties_to_take) - (ties_before < ties_to_take ? ties_before : ties_to_take));
-  const int i_base = tid * R;
-  for (int j = 0; j < R / 4; ++j) {
-    const uint4 k4 = my_keys[j];
-    const uint32_t kv[4] = {k4.x, k4.y, k4.z, k4.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      bool win = kv[e] < tau;
-      if (kv[e] == tau) {
-        win = eq_seen < ties_to_take;
-        ++eq_seen;
+  const uint32_t tb = ties_before < ties_to_take ? ties_before : ties_to_take;
+  uint32_t offs = below_before + tb + (excl & 0xffffu) + ((eq_seen < ties_to_take ? eq_seen : ties_to_take) - tb);
+  for (int j = 0; j < R; ++j) {
+    const uint32_t key = my[j];
+    bool win = key < tau;
+    if (key == tau) {
+      win = eq_seen < ties_to_take;
+      ++eq_seen;
+    }
+    if (win) {
+      if (offs < (uint32_t)kk) {
+        idx_out[offs] = first + j;
+        if (win_out != nullptr) win_out[offs] = key;
       }
-      if (win) {
-        if (offs < (uint32_t)kk) {
-          idx_out[offs] = lo + i_base + 4 * j + e;
-          if (p.win_keys != nullptr) p.win_keys[(int64_t)bg * p.win_stride + offs] = kv[e];
-        }
-        ++offs;
+      ++offs;
+    }
+  }
+}
+
+// Keys per thread of a CTA when n keys are cut over C CTAs of NT threads: a multiple of four (16-byte reads).
+__host__ __device__ __forceinline__ int keys_per_thread(int n, int C) {
+  int q = (n + 4 * C * NT - 1) / (4 * C * NT);
+  if (q < 1) q = 1;
+  return 4 * q;
+}
+
+__global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  const int C = (int)gridDim.x;               // CTAs per (sequence, KV head) = cluster size
+  const int rank = C > 1 ? (int)cluster_rank() : 0;
+  const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  SelectShared* sh = reinterpret_cast<SelectShared*>(smem_raw);
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + ((sizeof(SelectShared) + 15) & ~size_t(15)));
+  if (tid == 0) {
+    sh->cand_fill = 0u;
+    sh->own_in = 0u;
+    sh->n_mywin = 0u;
+    sh->win_before = 0u;
+    sh->sel_bin = kBins - 1;
+    sh->sel_want = 1u;
+    sh->sel_count = 0u;
+  }
+  const int64_t bg = (int64_t)b * p.n_kv_heads + g;
+  // slices are fixed by the host's length bound, so that the keys can be requested before the length is known
+  const int R = p.keys_per_thread;
+  const int per = R * NT;                     // a multiple of four
+  const int lo = rank * per;
+  const int n4 = per / 4;
+  const uint4* kg4 = reinterpret_cast<const uint4*>(p.keys + bg * p.logit_stride + lo);
+  const int lim4 = lo < p.logit_stride ? (int)((p.logit_stride - lo) / 4) : 0;   // vectors of this slice inside the buffer
+  // The one barrier that makes every peer's shared memory addressable sits above the dependency wait, where it is free.
+  if (C > 1) {
+    cluster_arrive();
+    cluster_wait();
+  } else {
+    __syncthreads();
+  }
+  // addresses and predicates are worked out above the dependency wait: behind it only the loads are left to issue
+  const int32_t* a_act = p.active != nullptr ? p.active + b : nullptr;
+  const int32_t* a_len = p.len + b;
+  const int32_t* a_cap = p.cap + b;
+  const int32_t* a_ks = p.k_small + b;
+  const uint4* hg = reinterpret_cast<const uint4*>(p.hist + bg * kBins) + tid * 2;
+  constexpr int KU = 4;
+  bool kq_on[KU];
+#pragma unroll
+  for (int u = 0; u < KU; ++u) kq_on[u] = u * NT + tid < n4 && u * NT + tid < lim4;
+  int32_t* idx_out = p.topk_idx + bg * p.k_max;
+  uint32_t* win_out = p.win_keys != nullptr ? p.win_keys + bg * p.win_stride : nullptr;
+  const int first = lo + tid * R;              // thread t owns keys [t R, (t + 1) R) of the slice
+  const uint32_t* my = keys + tid * R;
+  pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
+
+  // ---------------------------------------------------------------- 1: sizes, histogram and keys, one round trip
+  const int act = (a_act != nullptr) ? __ldcg(a_act) : 1;
+  const int len = __ldcg(a_len);
+  const int cap = __ldg(a_cap);
+  const int k_small = __ldcg(a_ks);
+  uint4 hv[2];                                 // thread t: bins 8 t .. 8 t + 7
+  hv[0] = __ldcg(hg);
+  hv[1] = __ldcg(hg + 1);
+  const uint4 pad4 = make_uint4(kPadKey, kPadKey, kPadKey, kPadKey);
+  uint4 kq[KU];
+#pragma unroll
+  for (int u = 0; u < KU; ++u) kq[u] = kq_on[u] ? __ldcg(kg4 + u * NT + tid) : pad4;
+  if (act == 0) return;   // same decision in all CTAs of the cluster
+  const Sizes sz = clamp_sizes(len, cap, p.max_len, k_small, p.k_max);
+  const int n = sz.n, kk = sz.kk;
+  for (int i = kk + rank * NT + tid; i < p.k_max; i += C * NT) idx_out[i] = -1;   // padding
+  if (n == 0) return;
+  {
+    uint4* keys4 = reinterpret_cast<uint4*>(keys);
+    const bool inside = lo + per <= n;        // the whole slice lies inside the sequence: nothing to pad
+    auto put = [&](int i4, uint4 k4) {        // keys at and beyond the length become padding
+      if (!inside) {
+        const int pos0 = lo + 4 * i4;
+        if (pos0 >= n) k4.x = kPadKey;
+        if (pos0 + 1 >= n) k4.y = kPadKey;
+        if (pos0 + 2 >= n) k4.z = kPadKey;
+        if (pos0 + 3 >= n) k4.w = kPadKey;
+      }
+      keys4[i4] = k4;
+    };
+#pragma unroll
+    for (int u = 0; u < KU; ++u) {
+      const int i4 = u * NT + tid;
+      if (i4 < n4) put(i4, kq[u]);
+    }
+    for (int base = KU * NT; base < n4; base += KU * NT) {
+#pragma unroll
+      for (int u = 0; u < KU; ++u) {
+        const int i4 = base + u * NT + tid;
+        kq[u] = (i4 < n4 && i4 < lim4 && lo + 4 * i4 < n) ? __ldcg(kg4 + i4) : pad4;
+      }
+#pragma unroll
+      for (int u = 0; u < KU; ++u) {
+        const int i4 = base + u * NT + tid;
+        if (i4 < n4) put(i4, kq[u]);
       }
     }
+  }
+  if (!sz.choose) {   // uniform over the cluster: nothing to choose (kk == 0, or every position is selected)
+    if (kk > 0) {
+      __syncthreads();
+      for (int j = 0; j < R; ++j)
+        if (first + j < n) {
+          idx_out[first + j] = first + j;
+          if (win_out != nullptr) win_out[first + j] = my[j];
+        }
+    }
+    return;
+  }
+
+  // ---------------------------------------------------------------- 2: the bin of the kk-th smallest key
+  uint32_t want = (uint32_t)kk, count;
+  {
+    const uint32_t hw[8] = {hv[0].x, hv[0].y, hv[0].z, hv[0].w, hv[1].x, hv[1].y, hv[1].z, hv[1].w};
+    uint32_t sum = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sum += hw[i];
+    const uint32_t inc = warp_scan_incl(sum, lane);
+    if (lane == 31) sh->warp_a[warp] = inc;
+    __syncthreads();   // also: the staged keys are visible
+    uint32_t wv = lane < NW ? sh->warp_a[lane] : 0u;
+    const uint32_t base = warp_sum(lane < warp ? wv : 0u);
+    const uint32_t excl = base + inc - sum;
+    if (excl < want && want <= excl + sum) {   // exactly one thread
+      uint32_t run = excl;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (run < want && want <= run + hw[i]) {
+          sh->sel_bin = tid * 8 + i;
+          sh->sel_want = want - run;
+          sh->sel_count = hw[i];
+        }
+        run += hw[i];
+      }
+    }
+    __syncthreads();
+  }
+  const uint32_t T = sh->sel_bin;
+  want = sh->sel_want;
+  count = sh->sel_count;
+  uint32_t lo_key = __float_as_uint((float)T * (1.f / kBinsPerNat));
+  uint32_t hi_key = (T == kBins - 1) ? kWorstKey : __float_as_uint((float)(T + 1) * (1.f / kBinsPerNat)) - 1u;
+  if (count > (uint32_t)kCandMax && lo_key != hi_key) refine(sh, keys, per, C, &lo_key, &hi_key, &want, &count);
+  // count > kCandMax here means the bin is a single key value shared by all its members
+  const bool ident = count > (uint32_t)kCandMax;
+
+  // ---------------------------------------------------------------- 3: count below the bin; exchange the bin's keys
+  const uint32_t span = hi_key - lo_key;
+  uint32_t c_below = 0, c_in = 0;
+  {
+    const uint32_t seg0 = smem_u32(&sh->seg[rank][0]);
+    const uint4* my4 = reinterpret_cast<const uint4*>(my);
+    for (int j4 = 0; j4 < R / 4; ++j4) {        // (R is the same for every thread: whole warps stay together)
+      const uint4 k4 = my4[j4];
+      const uint32_t kv[4] = {k4.x, k4.y, k4.z, k4.w};
+      c_below += (k4.x < lo_key) + (k4.y < lo_key) + (k4.z < lo_key) + (k4.w < lo_key);
+      // inside the bin (keys below it wrap around to huge values): rare
+      const bool any_in = k4.x - lo_key <= span || k4.y - lo_key <= span || k4.z - lo_key <= span || k4.w - lo_key <= span;
+      if (__any_sync(0xffffffffu, any_in)) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool in = kv[e] - lo_key <= span;
+          if (ident) {
+            c_in += in;
+            continue;
+          }
+          // the warp pushes its candidates together: each of them goes to peer `lane` from lane `lane`
+          uint32_t slot = 0;
+          if (in) slot = atomicAdd(&sh->cand_fill, 1u);
+          const unsigned long long kp = ((unsigned long long)kv[e] << 32) | (uint32_t)(first + 4 * j4 + e);
+          uint32_t todo = __ballot_sync(0xffffffffu, in && slot < (uint32_t)kCandMax);
+          while (todo != 0u) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1u;
+            const unsigned long long v = __shfl_sync(0xffffffffu, kp, src);
+            const uint32_t at = __shfl_sync(0xffffffffu, slot, src);
+            if (C == 1) {
+              if (lane == 0) sh->seg[0][at] = v;
+            } else if (lane < C) {
+              asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(map_rank(seg0 + 8u * at, lane)), "l"(v) : "memory");
+            }
+          }
+        }
+      }
+    }
+  }
+  // exclusive block scan of the counts below the bin: the thread's output offset inside the CTA, and the CTA's total
+  const uint32_t inc_b = warp_scan_incl(c_below, lane);
+  if (lane == 31) sh->warp_a[warp] = inc_b;
+  if (ident) {
+    c_in = warp_sum(c_in);
+    if (lane == 0 && c_in != 0u) atomicAdd(&sh->own_in, c_in);
+  }
+  __syncthreads();
+  uint32_t excl_below, own_below;
+  {
+    const uint32_t wv = lane < NW ? sh->warp_a[lane] : 0u;
+    const uint32_t wi = warp_scan_incl(wv, lane);                   // lane w: keys below the bin in warps 0..w
+    own_below = __shfl_sync(0xffffffffu, wi, NW - 1);
+    const uint32_t before = __shfl_sync(0xffffffffu, wi, warp > 0 ? warp - 1 : 0);
+    excl_below = (warp > 0 ? before : 0u) + inc_b - c_below;
+  }
+  {
+    uint32_t own_c = ident ? sh->own_in : sh->cand_fill;
+    if (!ident && own_c > (uint32_t)kCandMax) own_c = kCandMax;   // cannot happen: the bin holds at most kCandMax keys
+    if (C == 1) {
+      if (tid == 0) {
+        sh->below[0] = own_below;
+        sh->candn[0] = own_c;
+      }
+      __syncthreads();
+    } else {
+      if (tid < C) {
+        st_cluster(map_rank(smem_u32(&sh->below[rank]), tid), own_below);
+        st_cluster(map_rank(smem_u32(&sh->candn[rank]), tid), own_c);
+      }
+      cluster_arrive();
+      cluster_wait();
+    }
+  }
+  // From here on nobody touches a peer's shared memory, and every CTA of the cluster has read the histogram:
+  // clear it for the next selection on this workspace (each CTA its share).
+  {
+    uint4* hz = reinterpret_cast<uint4*>(p.hist + bg * kBins);
+    for (int i = rank * NT + tid; i < kBins / 4; i += C * NT) hz[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  uint32_t flat_base = 0, below_before = 0, total = 0;
+  int src = 0;                                // (threads below the candidate count) the CTA whose segment holds candidate tid
+  uint32_t pre = 0;                           // ... and the candidates of the CTAs before it
+#pragma unroll
+  for (int r = 0; r < kSelectCluster; ++r) {
+    const uint32_t c_r = r < C ? sh->candn[r] : 0u;
+    if (r < rank) {
+      flat_base += c_r;
+      below_before += sh->below[r];
+    }
+    total += c_r;
+    if (r < kSelectCluster - 1 && (uint32_t)tid >= total) {
+      src = r + 1;
+      pre = total;
+    }
+  }
+  if (ident) {
+    write_ties(sh, my, R, first, lo_key, want, flat_base, below_before, kk, idx_out, win_out);
+    return;
+  }
+
+  // ---------------------------------------------------------------- 4: which keys of the bin are selected
+  // (key, position) pairs are distinct, so the `want` smallest of them - ties to the lower position - are simply
+  // those of rank < want; P threads share one candidate (P a power of two, P * total <= NT).
+  if (total > (uint32_t)kCandMax) total = kCandMax;
+  if (tid < kCandMax) {
+    unsigned long long val = ~0ull;
+    if (tid < (int)total) val = sh->seg[src][tid - pre];
+    sh->flat[tid] = val;
+  }
+  __syncthreads();
+  {
+    int lp = 0;                                   // log2(P)
+    while (lp < 5 && ((int)total << (lp + 1)) <= NT) ++lp;
+    const int ci = tid >> lp, part = tid & ((1 << lp) - 1);
+    if (ci < (int)total) {                        // whole groups of P lanes take this branch together
+      const unsigned long long c = sh->flat[ci];
+      uint32_t less = 0;
+      for (int j = part; j < (int)total; j += (1 << lp)) less += sh->flat[j] < c;
+      const uint32_t gmask = __activemask();
+      for (int o = 1; o < (1 << lp); o <<= 1) less += __shfl_xor_sync(gmask, less, o);
+      if (part == 0 && less < want) {             // selected
+        if ((uint32_t)ci < flat_base) atomicAdd(&sh->win_before, 1u);
+        else if ((uint32_t)ci < flat_base + sh->candn[rank]) sh->mywin[atomicAdd(&sh->n_mywin, 1u)] = (int32_t)(uint32_t)c;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---------------------------------------------------------------- 5: ordered output
+  const int n_my = (int)sh->n_mywin;
+  uint32_t offs = below_before + sh->win_before + excl_below;
+  for (int i = 0; i < n_my; ++i) offs += sh->mywin[i] < first;   // selected keys of the bin that precede this thread's run
+  const uint4* my4 = reinterpret_cast<const uint4*>(my);
+  for (int j0 = 0; j0 < R; j0 += 32) {        // a mask of winners per 32 keys, then one store per winner
+    const int qn = (R - j0 < 32 ? R - j0 : 32) / 4;
+    uint32_t mask = 0;
+    for (int q = 0; q < qn; ++q) {
+      const uint4 k4 = my4[j0 / 4 + q];
+      uint32_t nib = (uint32_t)(k4.x < lo_key) | ((uint32_t)(k4.y < lo_key) << 1) | ((uint32_t)(k4.z < lo_key) << 2) |
+                     ((uint32_t)(k4.w < lo_key) << 3);
+      if (k4.x - lo_key <= span || k4.y - lo_key <= span || k4.z - lo_key <= span || k4.w - lo_key <= span) {
+        const uint32_t kv[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (kv[e] - lo_key <= span)
+            for (int i = 0; i < n_my; ++i) nib |= (uint32_t)(sh->mywin[i] == first + j0 + 4 * q + e) << e;
+      }
+      mask |= nib << (4 * q);
+    }
+    while (mask != 0u) {
+      const int j = __ffs(mask) - 1;
+      mask &= mask - 1u;
+      if (offs < (uint32_t)kk) {
+        idx_out[offs] = first + j0 + j;
+        if (win_out != nullptr) win_out[offs] = my[j0 + j];
+      }
+      ++offs;
+    }
+  }
+}
+
+template <int GP, bool kPool>
+cudaError_t launch_score_agg(const ScoreParams& p, dim3 grid, size_t smem, cudaStream_t st) {
+  switch (p.agg) {
+    case RKV_AGG_MEAN: return launch_ex(score_kernel<GP, RKV_AGG_MEAN, kPool>, grid, dim3(NTS), smem, st, 1, p);
+    case RKV_AGG_FIRST: return launch_ex(score_kernel<GP, RKV_AGG_FIRST, kPool>, grid, dim3(NTS), smem, st, 1, p);
+    default: return launch_ex(score_kernel<GP, RKV_AGG_MAX, kPool>, grid, dim3(NTS), smem, st, 1, p);
   }
 }
 
 }  // namespace
 
-int select_keys_cap(int keys_per_cta) {   // R * NT keys, R a multiple of 4
-  return (int)(((size_t)keys_per_cta + 4 * NT - 1) / (4 * NT) * (4 * NT));
+int select_cluster_for(int n_max) {   // CTAs per (sequence, KV head): about 4096 keys each, a power of two up to 8
+  int c = 1;
+  while (c < kSelectCluster && (int64_t)c * 4096 < n_max) c <<= 1;
+  return c;
 }
 
-size_t select_smem_bytes(int keys_per_cta, int pool_half) {
-  const size_t padded = (size_t)select_keys_cap(keys_per_cta);
-  const size_t raw = pool_half > 0 ? padded + 2 * (size_t)pool_half + 4 : 0;   // unpooled keys with their halo
-  return ((sizeof(SelectShared) + 15) & ~size_t(15)) + (padded + raw) * 4;
+int select_keys_per_thread(int n_max, int cluster) { return keys_per_thread(n_max, cluster); }
+
+size_t select_smem_bytes(int keys_per_thr) {
+  return ((sizeof(SelectShared) + 15) & ~size_t(15)) + (size_t)keys_per_thr * NT * 4;
 }
 
 cudaError_t prepare_select() {
-  const int bytes = (int)select_smem_bytes(kSelectMaxKeysPerCta, 0);
-  cudaError_t e = cudaFuncSetAttribute(select_kernel<4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  return e;
+  const int r_max = keys_per_thread(kSelectCluster * kSelectMaxKeysPerCta, kSelectCluster);
+  return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)select_smem_bytes(r_max));
 }
 
-cudaError_t launch_select(const SelectParams& p, int n_seq, int sm_count, cudaStream_t st) {
-  const dim3 grid(kSelectCluster, p.n_kv_heads, n_seq);
-  const size_t smem = select_smem_bytes(p.per_cta, p.pool_half);
-  // two CTAs per SM when one wave cannot hold every cluster and two CTAs' shared memory fits
-  const bool dense = (int64_t)kSelectCluster * p.n_kv_heads * n_seq > sm_count && 2 * (smem + 1024) <= 227 * 1024;
+// Positions per CTA of the score pass: the smallest slice that keeps the grid within about four CTAs per SM.
+int score_slice_for(int n_max, int problems, int sm_count) {
+  int slice = 1024;
+  while (slice < kSelectMaxSlice && (int64_t)problems * ((n_max + slice - 1) / slice) > 4 * (int64_t)sm_count) slice <<= 1;
+  return slice;
+}
+
+cudaError_t launch_score(const ScoreParams& p, int n_seq, cudaStream_t st) {
+  const dim3 grid(p.n_slices + (p.out != nullptr ? 2 * p.group : 0), p.n_kv_heads, n_seq);
+  const size_t smem = p.pool_half > 0 ? (size_t)(p.slice + 2 * p.pool_half) * 4 : 0;
   if (p.group <= 4) {
-    if (dense) return launch_ex(select_kernel<4, 2>, grid, dim3(NT), smem, st, kSelectCluster, p);
-    return launch_ex(select_kernel<4, 1>, grid, dim3(NT), smem, st, kSelectCluster, p);
+    if (p.pool_half > 0) return launch_score_agg<4, true>(p, grid, smem, st);
+    return launch_score_agg<4, false>(p, grid, smem, st);
   }
-  if (dense) return launch_ex(select_kernel<8, 2>, grid, dim3(NT), smem, st, kSelectCluster, p);
-  return launch_ex(select_kernel<8, 1>, grid, dim3(NT), smem, st, kSelectCluster, p);
+  if (p.pool_half > 0) return launch_score_agg<8, true>(p, grid, smem, st);
+  return launch_score_agg<8, false>(p, grid, smem, st);
+}
+
+cudaError_t launch_select(const SelectParams& p, int n_seq, int cluster, cudaStream_t st) {
+  const dim3 grid(cluster, p.n_kv_heads, n_seq);
+  return launch_ex(select_kernel, grid, dim3(NT), select_smem_bytes(p.keys_per_thread), st, cluster, p);
 }
 
 }  // namespace rkv

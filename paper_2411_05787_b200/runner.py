@@ -168,3 +168,99 @@ class OverlappedRefresh:
         for l in range(max(n - 2, 0), n):
             main.wait_event(self.ev_sel[l])
 
+
+
+class DeferredRefresh:
+    """Full-step token over a stack of layers with every layer's selection and rebuild AFTER the last attention pass.
+
+    The refreshed small cache of a layer is first read by the NEXT token's partial step, so nothing forces the
+    selection to run beside the following layers' attention, where its CTAs displace attention CTAs and unbalance
+    their single wave.  Here the attention passes of all layers follow each other undisturbed in the calling stream;
+    then the layers' selections and rebuilds run, spread over a few side streams so that several of these short,
+    latency-bound kernel chains are in flight at once.  Every layer needs a context of its own: its logits stay in
+    the context's workspace until its selection runs."""
+
+    def __init__(self, layers, n_side=8):
+        self.layers = layers
+        ctxs = [id(st.ctx) for st in layers]
+        if len(set(ctxs)) != len(ctxs):
+            raise ValueError("every layer needs its own context (the workspace holds its logits until the token's end)")
+        self.sides = [torch.cuda.Stream() for _ in range(max(1, min(n_side, len(layers))))]
+        self.ev_attn = torch.cuda.Event()
+        self.ev_done = [torch.cuda.Event() for _ in self.sides]
+
+    def run(self, q_of, k_new_of, v_new_of, max_len_hint=0):
+        """q_of(l), k_new_of(l), v_new_of(l): the layer's inputs.  Appends, attends; then selects and rebuilds."""
+        main = torch.cuda.current_stream()
+        for l, st in enumerate(self.layers):
+            st.append_refresh_attention(q_of(l), k_new_of(l), v_new_of(l), max_len_hint=max_len_hint)
+        self.ev_attn.record(main)
+        for i, side in enumerate(self.sides):
+            side.wait_event(self.ev_attn)
+            with torch.cuda.stream(side):
+                for l in range(i, len(self.layers), len(self.sides)):
+                    self.layers[l].refresh_select(q_of(l))
+                self.ev_done[i].record(side)
+        for ev in self.ev_done:
+            main.wait_event(ev)
+
+    def run_checked(self, q_of, k_new_of, v_new_of, threshold, small_hint=0, full_hint=0, after_trigger=None):
+        """Token of the dynamic schedule at a check position: per layer the trigger, then both branches under its
+        device masks (the partial step, which appends to both caches for every sequence, for the sequences that keep
+        their small cache; the full step's attention for those that refresh); the selections and rebuilds of the
+        refreshing sequences follow after the last layer, as in run()."""
+        main = torch.cuda.current_stream()
+        for l, st in enumerate(self.layers):
+            st.check_trigger(q_of(l), threshold)
+            if after_trigger is not None:
+                after_trigger(l, st)
+            st.append_partial(q_of(l), k_new_of(l), v_new_of(l), active=st.not_flag, max_len_hint=small_hint)
+            st.refresh_attention(q_of(l), active=st.flag, max_len_hint=full_hint)
+        self.ev_attn.record(main)
+        for i, side in enumerate(self.sides):
+            side.wait_event(self.ev_attn)
+            with torch.cuda.stream(side):
+                for l in range(i, len(self.layers), len(self.sides)):
+                    self.layers[l].refresh_select(q_of(l), active=self.layers[l].flag)
+                self.ev_done[i].record(side)
+        for ev in self.ev_done:
+            main.wait_event(ev)
+
+
+class LayerBatchedSmall:
+    """The partial step of ALL layers of a token as one call: the small caches of every (layer, sequence) live in one
+    K and one V buffer and one context sees them as layers x B sequences.
+
+    A decoder cannot run its layers' attention at once (layer l + 1's query depends on layer l's output); this form
+    exists to measure what the partial-step kernel streams when launch and dependency latencies are amortised over
+    all layers, which is legal for synthetic per-layer queries that do not depend on each other."""
+
+    def __init__(self, layers, max_len_hint: int):
+        first = layers[0]
+        dev = first.out.device
+        self.layers, self.n_layers, self.n_seq = layers, len(layers), first.n_seq
+        self.n_q, self.n_kv = first.n_q, first.n_kv
+        caps = []
+        for st in layers:
+            caps += st.small.cap.tolist()
+        self.cache = alloc_cache(caps, [0] * len(caps), self.n_kv, dev, fill=0.0)
+        self.cache_c = rkv.cache_struct(self.cache.k, self.cache.v, self.cache.row_offset, self.cache.cap, self.cache.len)
+        self.ctx = rkv.Context(len(caps), self.n_q, self.n_kv, max(max_len_hint, 1), max(max_len_hint, 1))
+        self.hint = max_len_hint
+
+    def sync_from_layers(self):
+        """Copy every layer's small cache (rows and lengths) into the combined buffers."""
+        offs = self.cache.row_offset.tolist()
+        for l, st in enumerate(self.layers):
+            base = offs[l * self.n_seq]
+            n = st.small.k.shape[0]
+            self.cache.k[base: base + n].copy_(st.small.k)
+            self.cache.v[base: base + n].copy_(st.small.v)
+            self.cache.len[l * self.n_seq: (l + 1) * self.n_seq].copy_(st.small.len)
+
+    def append_partial(self, q_all, k_all, v_all, out_all):
+        """q_all [layers, B, Hq, 128], k_all / v_all [layers, B, Hkv, 128], out_all [layers, B, Hq, 128]: one launch."""
+        n = self.n_layers * self.n_seq
+        self.ctx.append_small_step(q_all.view(n, self.n_q, HEAD_DIM), k_all.view(n, self.n_kv, HEAD_DIM),
+                                   v_all.view(n, self.n_kv, HEAD_DIM), None, self.cache_c,
+                                   out_all.view(n, self.n_q, HEAD_DIM), max_len_hint=self.hint)

@@ -66,16 +66,44 @@ def config1() -> Workload:
                     heavy_gain=4.0, heavy_noise=0.0, walk_sigma=0.1, seed=0)
 
 
-def config2(n_layers: int = 32, ctx: int = 32768, steps: int = 512) -> Workload:
-    """Llama-3.1-8B attention shape, batch 1, L=32768, K=2048, fixed stride 10."""
-    return Workload(f"cfg2_llama8b_L{ctx}_K{ctx // 16}_S10", n_layers, 32, 8, [ctx], [ctx // 16], steps,
-                    "fixed", 10, rho=[0.95], replant_every=64, seed=2)
+def config2(n_layers: int = 32, ctx: int = 32768, steps: int = 512, k_small: int = 0, stride: int = 10) -> Workload:
+    """Llama-3.1-8B attention shape, batch 1, L=32768, K=2048, fixed stride 10 (k_small = 0: ctx / 16)."""
+    k = k_small or ctx // 16
+    return Workload(f"cfg2_llama8b_L{ctx}_K{k}_S{stride}", n_layers, 32, 8, [ctx], [k], steps,
+                    "fixed", stride, rho=[0.95], replant_every=64, seed=2)
 
 
-def config3(n_layers: int = 28, ctx: int = 65536, steps: int = 1024, qc: int = 5) -> Workload:
-    """Qwen2-7B attention shape (G=7), batch 4, L=65536, K=4096, dynamic refresh at 0.9."""
-    return Workload(f"cfg3_qwen7b_L{ctx}_K{ctx // 16}_dyn{qc}", n_layers, 28, 4, [ctx] * 4, [ctx // 16] * 4,
-                    steps, "dynamic", qc, threshold=0.9, rho=[0.80, 0.90, 0.96, 0.99], seed=3)
+def config3(n_layers: int = 28, ctx: int = 65536, steps: int = 1024, qc: int = 5, k_small: int = 0,
+            threshold: float = 0.9) -> Workload:
+    """Qwen2-7B attention shape (G=7), batch 4, L=65536, K=4096, dynamic refresh at 0.9 (k_small = 0: ctx / 16)."""
+    k = k_small or ctx // 16
+    return Workload(f"cfg3_qwen7b_L{ctx}_K{k}_dyn{qc}", n_layers, 28, 4, [ctx] * 4, [k] * 4,
+                    steps, "dynamic", qc, threshold=threshold, rho=[0.80, 0.90, 0.96, 0.99], seed=3)
+
+
+# The paper's own operating points (Sec. 3 "Inference settings", Sec. 4.1 on strides, App. A.4 on thresholds):
+# K = L / 8 - 16K-token language-modelling inputs with K = 2048 and 256 generated tokens, 100K+-token inputs with
+# K = 4096 - fixed strides of 10 and 15, and the query-similarity trigger checked every 5 or 10 steps with
+# threshold 0.85 (Llama-3.1-8B) or 0.95 (Qwen2-7B), batch 1.  Shapes only: data and weights are synthetic.
+PAPER_POINTS = {
+    # name: (model shape, context, K, schedule, stride or QC, threshold, decode steps)
+    "lm16k_S10": ("llama", 16384, 2048, "fixed", 10, 0.0, 256),
+    "lm16k_S15": ("llama", 16384, 2048, "fixed", 15, 0.0, 256),
+    "lm16k_dyn085_qc5": ("llama", 16384, 2048, "dynamic", 5, 0.85, 256),
+    "lm16k_dyn085_qc10": ("llama", 16384, 2048, "dynamic", 10, 0.85, 256),
+    "novel128k_S10": ("llama", 131072, 4096, "fixed", 10, 0.0, 256),
+    "novel128k_dyn085_qc10": ("llama", 131072, 4096, "dynamic", 10, 0.85, 256),
+    "qwen16k_dyn095_qc5": ("qwen", 16384, 2048, "dynamic", 5, 0.95, 256),
+    "qwen16k_dyn095_qc10": ("qwen", 16384, 2048, "dynamic", 10, 0.95, 256),
+}
+
+
+def paper_point(name: str, n_layers: int = 0) -> Workload:
+    """One of the paper's operating points as a batch-1 workload (AR(1) queries with rho = 0.95, 1 % heavy keys)."""
+    model, ctx, k, schedule, stride, thr, steps = PAPER_POINTS[name]
+    n_q, n_kv, layers = (32, 8, 32) if model == "llama" else (28, 4, 28)
+    return Workload(f"paper_{name}", n_layers or layers, n_q, n_kv, [ctx], [k], steps, schedule, stride,
+                    threshold=thr, rho=[0.95], replant_every=64, seed=7)
 
 
 def config4(n_layers: int = 32, n_seq: int = 16, lo: int = 8192, hi: int = 131072, steps: int = 256) -> Workload:

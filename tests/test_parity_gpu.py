@@ -549,6 +549,46 @@ def test_ties_go_to_the_lower_position(mods):
     assert got == sorted(hot + [i for i in range(40) if i not in hot][:34])
 
 
+def test_many_near_equal_scores_take_the_refinement_path(mods):
+    """Thousands of distinct scores inside one histogram bin (keys that differ by a small perturbation): the
+    selection has to narrow the bin down with its finer histograms before it can resolve the threshold."""
+    rkv, runner, synth = mods
+    for lens, k_small, n_q, n_kv in (([3000], [700], 4, 1), ([9000, 5000], [1500, 4000], 8, 2), ([40000], [9000], 4, 1)):
+        ctx, st, cache, q = make_layer(mods, lens, k_small, n_q, n_kv, seed=23 + len(lens))
+        g = torch.Generator(device="cuda"); g.manual_seed(77)
+        base = torch.randn((1, 128), generator=g, device="cuda")
+        cache.k.copy_((base + 0.004 * torch.randn(cache.k.shape, generator=g, device="cuda")).to(torch.bfloat16))
+        st.refresh(q)
+        assert ctx.device_status() == 0
+        check_full_against_oracle(st, cache, q, lens, k_small, n_kv)
+        a = st.topk_idx.clone()
+        st.refresh(q)                       # the histogram was left clean: the same answer again
+        assert torch.equal(a, st.topk_idx)
+
+
+def test_gather_flags_indices_outside_the_cache(mods):
+    """rkv_gather_small: -1 is padding and is skipped silently; any other index outside [0, len) is skipped
+    and raises RKV_DEV_BAD_INDEX; the rows of valid indices are still copied."""
+    rkv, runner, synth = mods
+    lens, k_small = [200], [8]
+    ctx, st, cache, q = make_layer(mods, lens, k_small, 4, 2, seed=31)
+    for bad in (200, 10 ** 6, -2, -(2 ** 31)):
+        idx = torch.tensor([[[3, 5, bad, 9, 11, -1, 20, 21], [0, 1, 2, 3, 4, 5, 6, 7]]], dtype=torch.int32, device="cuda")
+        st.small.k.fill_(0.0); st.small.v.fill_(0.0)
+        ctx.gather_small(idx, st.k_small, 8, st.full_c, st.small_c)
+        assert ctx.device_status() == rkv.DEV_BAD_INDEX, bad
+        fk, sk = host_heads(cache, 0, 2, "k"), host_heads(st.small, 0, 2, "k")
+        for r, j in enumerate([3, 5, None, 9, 11, None, 20, 21]):
+            if j is None:
+                assert not sk[0, r].any()
+            else:
+                assert np.array_equal(sk[0, r], fk[0, j])
+        assert np.array_equal(sk[1, :8], fk[1, :8])
+    idx = torch.tensor([[[3, 5, -1, 9, 11, -1, 20, 21], [0, 1, 2, 3, 4, 5, 6, 7]]], dtype=torch.int32, device="cuda")
+    ctx.gather_small(idx, st.k_small, 8, st.full_c, st.small_c)
+    assert ctx.device_status() == 0
+
+
 def test_deterministic_bits(mods):
     lens, k_small = [5000, 3000], [256, 100]
     ctx, st, cache, q = make_layer(mods, lens, k_small, 32, 8, seed=15)
@@ -581,7 +621,7 @@ def test_host_side_argument_errors(mods):
     with pytest.raises(rkv.RkvError):
         rkv.Context(1, 8, 2, 100, 10, pool_kernel=33)
     with pytest.raises(rkv.RkvError):
-        rkv.Context(1, 8, 2, 200000, 10, pool_kernel=7)      # with pooling the length limit is 163840
+        rkv.Context(1, 8, 2, 8 * 40960 + 1, 10, pool_kernel=7)   # the length limit, with or without pooling
     # bf16 tensors start on a 16-byte boundary: a query (or output) view that begins 2 bytes in is refused
     skew = torch.zeros(q.numel() + 8, dtype=torch.bfloat16, device=q.device)
     q_off = skew[1: 1 + q.numel()].view_as(q)
@@ -859,6 +899,16 @@ def test_largest_supported_length(mods):
     rkv = mods[0]
     with pytest.raises(rkv.RkvError):
         rkv.Context(1, 2, 1, 8 * 40960 + 1, 64)            # beyond the limit: refused at creation
+
+
+@pytest.mark.parametrize("pool", [7, 31])
+def test_pooling_on_a_long_sequence(mods, pool):
+    """Neighbour max-pooling at a length where the selection runs with its largest slices (163840 positions)."""
+    lens, k_small = [163840], [4096]
+    ctx, st, cache, q = make_layer(mods, lens, k_small, 2, 1, seed=43 + pool, want_scores=True, pool=pool)
+    st.refresh(q)
+    assert ctx.device_status() == 0
+    check_full_against_oracle(st, cache, q, lens, k_small, 1, pool=pool)
 
 
 def test_bench_configuration_graph_replay_shared_context(mods):

@@ -5,13 +5,18 @@ owns the device heap, or an allocation's implicit synchronisation is not allowed
 they cannot create an rkv_ctx.  The context-free entry point keeps its scratch in a fixed array in
 the library image instead.  This test calls it through the C ABI twice in a row - the second call
 finds the array as the first one left it - and checks each result against rkv_small_step on the
-same inputs, with the tolerance of the other attention tests (the two may split the cache
-differently, so sums differ in order).  Collected last, so a run that stops at the first failure
-has already covered everything else.
+same inputs and against the fp64 CPU oracle, with the tolerance of the other attention tests (the
+context call merges its splits inside a thread-block cluster, the context-free one through the static
+array, so the two reach the answer by different routes and their sums differ in order).  The second
+call must also leave the amount of free device memory unchanged: the first call on a device may load
+the library's device code, later ones take nothing.  Collected last, so a run that stops at the first
+failure has already covered everything else.
 """
 import numpy as np
 import pytest
 import torch
+
+from oracle import rkv_oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -24,6 +29,17 @@ def _close(a, b, what):
     err = np.abs(a - b).max()
     rel = np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
     assert err <= OUT_MAX_ABS and rel <= OUT_REL_L2, f"{what}: max-abs {err:.3e}, rel-L2 {rel:.3e}"
+
+
+def _bits(t):
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def _oracle_out(q_b, cache, b, n, n_kv):
+    off, cap = int(cache.row_offset[b]), int(cache.cap[b])
+    k = O.bf16_bits_to_f64(_bits(cache.k[off: off + n_kv * cap]).reshape(n_kv, cap, 128)[:, :n])
+    v = O.bf16_bits_to_f64(_bits(cache.v[off: off + n_kv * cap]).reshape(n_kv, cap, 128)[:, :n])
+    return O.decode_attention(O.bf16_bits_to_f64(_bits(q_b)), k, v)[0]
 
 
 def test_noalloc_small_step_matches_the_context_call_twice_in_a_row():
@@ -48,10 +64,19 @@ def test_noalloc_small_step_matches_the_context_call_twice_in_a_row():
         want = torch.zeros((len(lens), n_q, 128), dtype=torch.bfloat16, device=dev)
         got = torch.full_like(want, 7.0)
         ctx.small_step(q, small_c, want)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         rkv.small_step_noalloc(cfg, q, small_c, got, active=active if call else None, device_status=status)
         torch.cuda.synchronize()
+        free_after = torch.cuda.mem_get_info()[0]
+        if call:          # the first call on a device may load the library's device code; later calls take nothing
+            assert free_after == free_before, (free_before, free_after)
         assert ctx.device_status() == 0 and int(status.item()) == 0
         _close(got, want, f"call {call}")
+        cur = small.len.tolist()
+        for b in range(len(lens)):      # and against the definition itself, sequence by sequence
+            ref = torch.from_numpy(_oracle_out(q[b], small, b, cur[b], n_kv))
+            _close(got[b], ref, f"call {call} seq {b} vs oracle")
         # grow the caches between the calls, as decoding does
         ctx.append(torch.randn((len(lens), n_kv, 128), generator=g, device=dev).to(torch.bfloat16),
                    torch.randn((len(lens), n_kv, 128), generator=g, device=dev).to(torch.bfloat16), None, small_c)
