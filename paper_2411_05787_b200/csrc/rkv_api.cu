@@ -39,7 +39,7 @@ int splits_for(const rkv_config* c) {
   return s < rkv::kMaxSplits ? (s < 1 ? 1 : s) : rkv::kMaxSplits;
 }
 
-struct WsLayout { size_t partials, ml_t, tickets, len_tickets, win_keys, keys, hist, logits, status, total; int64_t logit_stride; };
+struct WsLayout { size_t partials, ml_t, tickets, len_tickets, win_keys, keys, hist, anchor, logits, status, total; int64_t logit_stride; };
 
 WsLayout ws_layout(const rkv_config* c) {
   WsLayout w;
@@ -55,6 +55,7 @@ WsLayout ws_layout(const rkv_config* c) {
   w.win_keys = off; off = up(off + bg * (size_t)c->max_small * sizeof(uint32_t));
   w.keys = off;     off = up(off + bg * (size_t)w.logit_stride * sizeof(uint32_t));
   w.hist = off;     off = up(off + bg * (size_t)rkv::kSelectBins * sizeof(uint32_t));
+  w.anchor = off;   off = up(off + bg * sizeof(int32_t));
   const int gp = group <= 4 ? 4 : 8;   // position-major logits, padded to a vector width
   w.logits = off;   off = up(off + bg * gp * (size_t)w.logit_stride * sizeof(float));
   w.status = off;   off = up(off + sizeof(int32_t));
@@ -339,6 +340,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->win_keys = reinterpret_cast<uint32_t*>(ctx->workspace + w.win_keys);
   ctx->keys = reinterpret_cast<uint32_t*>(ctx->workspace + w.keys);
   ctx->hist = reinterpret_cast<uint32_t*>(ctx->workspace + w.hist);   // zeroed with the rest of the workspace above
+  ctx->anchor = reinterpret_cast<int32_t*>(ctx->workspace + w.anchor);
   ctx->hist_dirty = false;
   ctx->logits = reinterpret_cast<float*>(ctx->workspace + w.logits);
   ctx->status = reinterpret_cast<int32_t*>(ctx->workspace + w.status);
@@ -418,6 +420,7 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   cp.scores = scores;
   cp.keys = ctx->keys;
   cp.hist = ctx->hist;
+  cp.anchor = ctx->anchor;
   cp.status = ctx->status;
   cp.logit_stride = ctx->logit_stride;
   cp.score_stride = score_stride;
@@ -437,6 +440,7 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   memset(&sp, 0, sizeof(sp));
   sp.keys = ctx->keys;
   sp.hist = ctx->hist;
+  sp.anchor = ctx->anchor;
   sp.cap = full->cap;
   sp.len = full->len;
   sp.k_small = k_small;
@@ -450,6 +454,7 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   sp.max_len = n_max;
   const int cluster = rkv::select_cluster_for(n_max);
   sp.keys_per_thread = rkv::select_keys_per_thread(n_max, cluster);
+  sp.per_fixed = ctx->cfg.n_seq == 1 ? 1 : 0;
   cudaError_t e;
   ctx->hist_dirty = true;
   {

@@ -84,6 +84,7 @@ struct ScoreParams {
   float* scores;              // [B][Hkv][score_stride] or null
   uint32_t* keys;             // [B*Hkv][logit_stride]: key of every position
   uint32_t* hist;             // [B*Hkv][kSelectBins]: all zero on entry
+  int32_t* anchor;            // [B*Hkv]: where each histogram's window starts (whole nats of -log p)
   int32_t* status;
   int64_t logit_stride, score_stride;
   int32_t n_q_heads, n_kv_heads, group, agg;
@@ -97,6 +98,7 @@ struct ScoreParams {
 struct SelectParams {
   const uint32_t* keys;       // [B*Hkv][logit_stride]
   uint32_t* hist;             // [B*Hkv][kSelectBins]: read, then cleared
+  const int32_t* anchor;      // [B*Hkv]: written by the score pass
   const int32_t* cap;
   const int32_t* len;
   const int32_t* k_small;     // [B]
@@ -107,7 +109,8 @@ struct SelectParams {
   int64_t logit_stride;
   int32_t n_kv_heads;
   int32_t k_max, max_len;
-  int32_t keys_per_thread;    // keys per thread of a selection CTA (slices are fixed by the host's length bound)
+  int32_t keys_per_thread;    // keys per thread of a selection CTA at the host's length bound
+  int32_t per_fixed;          // 1: slices are rank * keys_per_thread * threads (one sequence); 0: cut by each sequence's own length
 };
 
 struct CacheDev {
@@ -229,6 +232,7 @@ struct rkv_ctx {
   uint32_t* win_keys;
   uint32_t* keys;      // key of every position of the last score pass
   uint32_t* hist;      // per (sequence, KV head) histogram of those keys; all zero between selections
+  int32_t* anchor;     // per (sequence, KV head): start of the histogram's window
   bool hist_dirty;     // a score pass was launched whose selection (which clears the histogram) was not
   float* logits;
   int32_t* status;

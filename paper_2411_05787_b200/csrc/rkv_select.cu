@@ -160,8 +160,19 @@ __device__ __forceinline__ uint32_t make_key(const float* x, const float* lse_r,
   }
   return __float_as_uint(fmaxf(-ell, 0.f)) & 0x7fffffffu;
 }
-__device__ __forceinline__ uint32_t bin_of(uint32_t key) {   // bin T holds T/128 <= -ell < (T+1)/128
-  return __float2uint_rz(fminf(__uint_as_float(key) * kBinsPerNat, (float)(kBins - 1)));
+// The histogram's window: bin T of a (sequence, KV head) holds  A + T/128 <= -ell < A + (T+1)/128,  bin 0 also
+// everything below A and the last bin everything above.  For logits of spread sigma the bulk of the keys sits
+// around the log-sum-exp of the group's heads (a position of average logit has -ell = LSE) and the K-th key a few
+// sigma below it, so the window starts kWindowBelow nats below the smallest LSE of the group: sharply peaked
+// attention, whose keys all lie dozens of nats up, is resolved as finely as flat attention.  A is an integer, which
+// keeps  -ell - A  and the bin edges exact in fp32: both kernels agree on every key's bin.
+constexpr float kWindowBelow = 26.f;
+__device__ __forceinline__ int window_anchor(float lse_min) {
+  const float a = floorf(lse_min - kWindowBelow);
+  return a > 0.f ? (a < 1024.f ? (int)a : 1024) : 0;   // (NaN compares false: 0)
+}
+__device__ __forceinline__ uint32_t bin_of(uint32_t key, float anchor) {
+  return __float2uint_rz(fminf(fmaxf((__uint_as_float(key) - anchor) * kBinsPerNat, 0.f), (float)(kBins - 1)));
 }
 
 // ------------------------------------------------------------------------------------------------ score_kernel
@@ -314,17 +325,20 @@ __global__ void __launch_bounds__(NTS) score_kernel(const ScoreParams p) {
 #pragma unroll
     for (int c = 0; c < GP / 4; ++c)
       v[u][c] = lg_on[u] ? __ldcg(lg + (int64_t)(u * NTS) * (GP / 4) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 vnext[U][GP / 4];                     // the round in flight behind the one being turned into keys
+  int n_hint = 0x7fffffff;                     // the sequence's length (+ halo), once known: nothing is loaded beyond it
   auto load_round = [&](int i0) {   // positions lo - half + i0 + u * NTS + tid (rounds after the first)
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int i = i0 + u * NTS + tid;
       const int pos = lo - half + i;
-      const bool on = i < n_pos && pos >= 0 && pos < p.logit_stride;
+      const bool on = i < n_pos && pos >= 0 && pos < p.logit_stride && pos < n_hint;
 #pragma unroll
       for (int c = 0; c < GP / 4; ++c)
-        v[u][c] = on ? __ldcg(lg + (int64_t)(i0 + u * NTS) * (GP / 4) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        vnext[u][c] = on ? __ldcg(lg + (int64_t)(i0 + u * NTS) * (GP / 4) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
+
   uint4 qv = make_uint4(0u, 0u, 0u, 0u);
   if (q_copy) qv = __ldcg(a_q);
 
@@ -356,8 +370,15 @@ __global__ void __launch_bounds__(NTS) score_kernel(const ScoreParams p) {
   }
   __syncthreads();
   float lse_r[GP];
+  float lse_min = INFINITY;
 #pragma unroll
-  for (int h = 0; h < GP; ++h) lse_r[h] = (h < G) ? s_lse[h] : INFINITY;
+  for (int h = 0; h < GP; ++h) {
+    lse_r[h] = (h < G) ? s_lse[h] : INFINITY;
+    lse_min = fminf(lse_min, lse_r[h]);
+  }
+  const int anchor_i = window_anchor(lse_min);
+  const float anchor = (float)anchor_i;
+  if (blockIdx.x == 0 && tid == 0) p.anchor[bg] = anchor_i;   // the selection kernel turns bins back into key ranges
   const float inv_g = 1.f / (float)G;
   bool bad = false;
   uint32_t* keys_out = p.keys + bg * p.logit_stride;
@@ -368,14 +389,17 @@ __global__ void __launch_bounds__(NTS) score_kernel(const ScoreParams p) {
     keys_out[pos] = key;
     if (sc_out != nullptr) sc_out[pos] = ex2f(-__uint_as_float(key) * kLog2eF);   // a NaN score has been flagged and reads as 0
     if (sz.choose) {
-      const uint32_t bin = bin_of(key);
+      const uint32_t bin = bin_of(key, anchor);
       atomicAdd(&s_hist[bin], 1u);
       bmin = min(bmin, bin);
       bmax = max(bmax, bin);
     }
   };
+  n_hint = n + half;
   for (int i0 = 0; i0 < n_pos; i0 += U * NTS) {
-    if (i0 > 0) load_round(i0);
+    const bool more = i0 + U * NTS < n_pos && lo - half + i0 + U * NTS < n + half;
+    if (more) load_round(i0 + U * NTS);        // overlaps the arithmetic below
+    if (lo - half + i0 >= n + half) break;     // uniform over the CTA: the rest of the slice lies beyond the sequence
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int i = i0 + u * NTS + tid;
@@ -389,6 +413,12 @@ __global__ void __launch_bounds__(NTS) score_kernel(const ScoreParams p) {
       } else if (on) {
         emit(pos, key);
       }
+    }
+    if (more) {
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int c = 0; c < GP / 4; ++c) v[u][c] = vnext[u][c];
     }
   }
   if (kPool) {
@@ -571,7 +601,7 @@ __host__ __device__ __forceinline__ int keys_per_thread(int n, int C) {
   return 4 * q;
 }
 
-__global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
+__global__ void __launch_bounds__(NT, 2) select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int C = (int)gridDim.x;               // CTAs per (sequence, KV head) = cluster size
   const int rank = C > 1 ? (int)cluster_rank() : 0;
@@ -588,13 +618,16 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
     sh->sel_count = 0u;
   }
   const int64_t bg = (int64_t)b * p.n_kv_heads + g;
-  // slices are fixed by the host's length bound, so that the keys can be requested before the length is known
-  const int R = p.keys_per_thread;
-  const int per = R * NT;                     // a multiple of four
-  const int lo = rank * per;
-  const int n4 = per / 4;
+  // One sequence: the slices are fixed by the host's length bound, so that the keys can be requested before the
+  // length is known.  A batch (ragged lengths): each sequence is cut in C by its own length once that is known, so
+  // that short sequences use the whole cluster too.
+  const bool per_fixed = p.per_fixed != 0;
+  int R = p.keys_per_thread;
+  int per = R * NT;                           // a multiple of four
+  int lo = rank * per;
+  int n4 = per / 4;
   const uint4* kg4 = reinterpret_cast<const uint4*>(p.keys + bg * p.logit_stride + lo);
-  const int lim4 = lo < p.logit_stride ? (int)((p.logit_stride - lo) / 4) : 0;   // vectors of this slice inside the buffer
+  int lim4 = lo < p.logit_stride ? (int)((p.logit_stride - lo) / 4) : 0;   // vectors of this slice inside the buffer
   // The one barrier that makes every peer's shared memory addressable sits above the dependency wait, where it is free.
   if (C > 1) {
     cluster_arrive();
@@ -607,15 +640,14 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   const int32_t* a_len = p.len + b;
   const int32_t* a_cap = p.cap + b;
   const int32_t* a_ks = p.k_small + b;
+  const int32_t* a_anchor = p.anchor + bg;
   const uint4* hg = reinterpret_cast<const uint4*>(p.hist + bg * kBins) + tid * 2;
   constexpr int KU = 4;
   bool kq_on[KU];
 #pragma unroll
-  for (int u = 0; u < KU; ++u) kq_on[u] = u * NT + tid < n4 && u * NT + tid < lim4;
+  for (int u = 0; u < KU; ++u) kq_on[u] = per_fixed && u * NT + tid < n4 && u * NT + tid < lim4;
   int32_t* idx_out = p.topk_idx + bg * p.k_max;
   uint32_t* win_out = p.win_keys != nullptr ? p.win_keys + bg * p.win_stride : nullptr;
-  const int first = lo + tid * R;              // thread t owns keys [t R, (t + 1) R) of the slice
-  const uint32_t* my = keys + tid * R;
   pdl_wait();
   pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
 
@@ -624,6 +656,7 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   const int len = __ldcg(a_len);
   const int cap = __ldg(a_cap);
   const int k_small = __ldcg(a_ks);
+  const float anchor = (float)__ldcg(a_anchor);
   uint4 hv[2];                                 // thread t: bins 8 t .. 8 t + 7
   hv[0] = __ldcg(hg);
   hv[1] = __ldcg(hg + 1);
@@ -636,6 +669,21 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   const int n = sz.n, kk = sz.kk;
   for (int i = kk + rank * NT + tid; i < p.k_max; i += C * NT) idx_out[i] = -1;   // padding
   if (n == 0) return;
+  if (!per_fixed) {
+    R = keys_per_thread(n, C);                // never above the host's bound (n <= its length bound)
+    per = R * NT;
+    lo = rank * per;
+    n4 = per / 4;
+    kg4 = reinterpret_cast<const uint4*>(p.keys + bg * p.logit_stride + lo);
+    lim4 = lo < p.logit_stride ? (int)((p.logit_stride - lo) / 4) : 0;
+#pragma unroll
+    for (int u = 0; u < KU; ++u) {
+      const int i4 = u * NT + tid;
+      kq[u] = (i4 < n4 && i4 < lim4 && lo + 4 * i4 < n) ? __ldcg(kg4 + i4) : pad4;
+    }
+  }
+  const int first = lo + tid * R;              // thread t owns keys [t R, (t + 1) R) of the slice
+  const uint32_t* my = keys + tid * R;
   {
     uint4* keys4 = reinterpret_cast<uint4*>(keys);
     const bool inside = lo + per <= n;        // the whole slice lies inside the sequence: nothing to pad
@@ -709,8 +757,9 @@ __global__ void __launch_bounds__(NT, 1) select_kernel(const SelectParams p) {
   const uint32_t T = sh->sel_bin;
   want = sh->sel_want;
   count = sh->sel_count;
-  uint32_t lo_key = __float_as_uint((float)T * (1.f / kBinsPerNat));
-  uint32_t hi_key = (T == kBins - 1) ? kWorstKey : __float_as_uint((float)(T + 1) * (1.f / kBinsPerNat)) - 1u;
+  // bin T back into its range of keys (exact: the anchor is a small integer, the edges multiples of 1/128)
+  uint32_t lo_key = (T == 0u) ? 0u : __float_as_uint(anchor + (float)T * (1.f / kBinsPerNat));
+  uint32_t hi_key = (T == kBins - 1) ? kWorstKey : __float_as_uint(anchor + (float)(T + 1) * (1.f / kBinsPerNat)) - 1u;
   if (count > (uint32_t)kCandMax && lo_key != hi_key) refine(sh, keys, per, C, &lo_key, &hi_key, &want, &count);
   // count > kCandMax here means the bin is a single key value shared by all its members
   const bool ident = count > (uint32_t)kCandMax;
