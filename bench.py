@@ -69,6 +69,8 @@ def parse_args():
                          "pass; 'overlap' = behind the layer's attention in a second stream, beside the next layers'; "
                          "'one_stream' = attention, selection and rebuild of a layer in stream order")
     ap.add_argument("--no-overlap", action="store_true", help="same as --full-schedule one_stream")
+    ap.add_argument("--regions", type=int, default=0,
+                    help="timed regions of K steps to take (0: as many as region_repeats() says; 1 keeps a profiler run short)")
     return ap.parse_args()
 
 
@@ -508,7 +510,7 @@ def measure_workload(args, w, dev, world, steps, warmup, level):
     def repeated(n, **kw):
         """Regions of n tokens each, every one from the same starting state; (median ms, all ms, token counts)."""
         ms0, cnt = timed(n, **kw)
-        reps = region_repeats(ms0)
+        reps = args.regions if args.regions > 0 else region_repeats(ms0)
         if world > 1:                            # every rank must take the same number of regions
             tt = torch.tensor([reps], dtype=torch.int32, device=dev)
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)

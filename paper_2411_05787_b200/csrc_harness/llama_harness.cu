@@ -1,6 +1,7 @@
 // Batch-1 decoder kernels around the attention calls (see include/rkv_harness.h).
 // All of them are bound by streaming bf16 weights once per token; the matrix-vector kernels keep
-// 64 bytes per lane in flight and reduce inside a warp.
+// two batches of 128 bytes per lane in flight, request the first one before their stream dependency
+// has resolved (weights are constants) and reduce inside a warp.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -26,32 +27,40 @@ __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
     f[2 * i + 1] = t.y;
   }
 }
-// <row, x> for one weight row: lane l takes 16-byte chunks l, l+32, ...; x sits in shared memory as fp32.
-// Eight chunks (128 bytes) per lane are in flight at once, so a 4096-wide row costs two memory round trips.
-__device__ __forceinline__ float row_dot(const uint4* __restrict__ row, const float* xs, int n_chunks, int lane) {
-  constexpr int kFly = 8;
-  float acc = 0.f;
-  for (int c0 = lane; c0 < n_chunks; c0 += 32 * kFly) {
-    uint4 u[kFly];
+// Programmatic dependent launch: a kernel may be scheduled while its predecessor on the stream still runs and
+// waits here before it touches anything the predecessor writes.  Weights are constants, so the matrix-vector
+// kernels request their first batch of weights BEFORE this wait: launch latency and the staging of x then hide
+// behind the first memory round trip.  Dependents are released only after the kernel's own wait, so at most one
+// earlier kernel is ever still running.  Both are no-ops for a launch without the attribute.
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+constexpr int kFly = 4;   // 16-byte chunks per lane in one batch: 2 KiB per warp, two batches in flight
+
+// One batch of a weight row: lane l takes chunks b * 256 + l, + 32, ...  (nothing is read past the row or the matrix)
+__device__ __forceinline__ void load_batch(uint4 (&u)[kFly], const uint4* __restrict__ w, int64_t row, bool row_ok,
+                                           int b, int n_chunks, int lane) {
 #pragma unroll
-    for (int k = 0; k < kFly; ++k) {
-      const int c = c0 + 32 * k;
-      u[k] = (c < n_chunks) ? __ldcs(row + c) : make_uint4(0u, 0u, 0u, 0u);
-    }
+  for (int k = 0; k < kFly; ++k) {
+    const int c = b * 32 * kFly + lane + 32 * k;
+    u[k] = (row_ok && c < n_chunks) ? __ldcs(w + row * n_chunks + c) : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+// <batch, x>: x sits in shared memory as fp32
+__device__ __forceinline__ float batch_dot(const uint4 (&u)[kFly], const float* xs, int b, int n_chunks, int lane, float acc) {
 #pragma unroll
-    for (int k = 0; k < kFly; ++k) {
-      const int c = c0 + 32 * k;
-      if (c < n_chunks) {
-        float f[8];
-        unpack8(u[k], f);
-        const float4 x0 = *reinterpret_cast<const float4*>(xs + 8 * c);
-        const float4 x1 = *reinterpret_cast<const float4*>(xs + 8 * c + 4);
-        acc = fmaf(f[0], x0.x, acc); acc = fmaf(f[1], x0.y, acc); acc = fmaf(f[2], x0.z, acc); acc = fmaf(f[3], x0.w, acc);
-        acc = fmaf(f[4], x1.x, acc); acc = fmaf(f[5], x1.y, acc); acc = fmaf(f[6], x1.z, acc); acc = fmaf(f[7], x1.w, acc);
-      }
+  for (int k = 0; k < kFly; ++k) {
+    const int c = b * 32 * kFly + lane + 32 * k;
+    if (c < n_chunks) {
+      float f[8];
+      unpack8(u[k], f);
+      const float4 x0 = *reinterpret_cast<const float4*>(xs + 8 * c);
+      const float4 x1 = *reinterpret_cast<const float4*>(xs + 8 * c + 4);
+      acc = fmaf(f[0], x0.x, acc); acc = fmaf(f[1], x0.y, acc); acc = fmaf(f[2], x0.z, acc); acc = fmaf(f[3], x0.w, acc);
+      acc = fmaf(f[4], x1.x, acc); acc = fmaf(f[5], x1.y, acc); acc = fmaf(f[6], x1.z, acc); acc = fmaf(f[7], x1.w, acc);
     }
   }
-  return warp_sum(acc);
+  return acc;
 }
 // Bring x into shared memory as fp32; with a norm weight, apply RMSNorm on the way (every block recomputes the
 // mean square of the few thousand inputs, which is cheaper than a separate launch).
@@ -86,30 +95,52 @@ __device__ __forceinline__ void stage_x(const void* x, int x_is_bf16, const __nv
   __syncthreads();
 }
 
+// y[o] = <W[o], x> (+ residual[o]); kSwiglu: y[f] = silu(<W[f], x>) * <W[f + n_out], x>.  A warp walks its rows
+// (o = first, first + stride, ...) as one stream of weight batches: the loads of the next batch - of the same row
+// or of the warp's next row - are issued before the current batch is multiplied.
+template <bool kSwiglu>
 __global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const uint4* __restrict__ w, const void* x, int x_is_bf16,
                                                             const __nv_bfloat16* norm_w, float eps, const float* residual,
                                                             float* y, int n_out, int n_in) {
   extern __shared__ float xs[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = kGemvThreads / 32;
+  const int n_chunks = n_in / 8;
+  const int bpr = (n_chunks + 32 * kFly - 1) / (32 * kFly);   // batches per weight row
+  const int stride = gridDim.x * wpb;
+  constexpr int kParts = kSwiglu ? 2 : 1;                      // weight rows per output
+  int o = blockIdx.x * wpb + warp, part = 0, b = 0;            // the batch being multiplied
+  // the warp's first batch is requested before the stream dependency has resolved
+  uint4 cur[kFly], nxt[kFly];
+  load_batch(cur, w, (int64_t)o + (int64_t)part * n_out, o < n_out, 0, n_chunks, lane);
+  dep_wait();
+  dep_launch();
   stage_x(x, x_is_bf16, norm_w, eps, xs, n_in);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = kGemvThreads / 32;
-  const int n_chunks = n_in / 8;
-  for (int o = blockIdx.x * wpb + warp; o < n_out; o += gridDim.x * wpb) {
-    const float d = row_dot(w + (int64_t)o * n_chunks, xs, n_chunks, lane);
-    if (lane == 0) y[o] = d + (residual != nullptr ? residual[o] : 0.f);
-  }
-}
-
-__global__ void __launch_bounds__(kGemvThreads) gemv_swiglu_kernel(const uint4* __restrict__ w, const float* x,
-                                                                   const __nv_bfloat16* norm_w, float eps, float* y,
-                                                                   int n_ff, int n_in) {
-  extern __shared__ float xs[];
-  stage_x(x, 0, norm_w, eps, xs, n_in);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = kGemvThreads / 32;
-  const int n_chunks = n_in / 8;
-  for (int f = blockIdx.x * wpb + warp; f < n_ff; f += gridDim.x * wpb) {
-    const float g = row_dot(w + (int64_t)f * n_chunks, xs, n_chunks, lane);
-    const float u = row_dot(w + (int64_t)(f + n_ff) * n_chunks, xs, n_chunks, lane);
-    if (lane == 0) y[f] = g / (1.f + __expf(-g)) * u;
+  float acc = 0.f, gate = 0.f;
+  while (o < n_out) {
+    int no = o, np = part, nb = b + 1;                         // the batch after this one
+    if (nb == bpr) {
+      nb = 0;
+      if (++np == kParts) {
+        np = 0;
+        no = o + stride;
+      }
+    }
+    load_batch(nxt, w, (int64_t)no + (int64_t)np * n_out, no < n_out, nb, n_chunks, lane);
+    acc = batch_dot(cur, xs, b, n_chunks, lane, acc);
+    if (b == bpr - 1) {                                        // a weight row is complete
+      acc = warp_sum(acc);
+      if (kSwiglu && part == 0) {
+        gate = acc;
+      } else if (lane == 0) {
+        y[o] = kSwiglu ? gate / (1.f + __expf(-gate)) * acc : acc + (residual != nullptr ? residual[o] : 0.f);
+      }
+      acc = 0.f;
+    }
+#pragma unroll
+    for (int k = 0; k < kFly; ++k) cur[k] = nxt[k];
+    o = no;
+    part = np;
+    b = nb;
   }
 }
 
@@ -131,6 +162,8 @@ __global__ void __launch_bounds__(256) rope_split_kernel(const float* qkv, const
                                                          __nv_bfloat16* k, __nv_bfloat16* v, int n_q, int n_kv) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   const int n_rot = (n_q + n_kv) * 64;
+  dep_wait();
+  dep_launch();
   if (t < n_rot) {
     const int head = t >> 6, c = t & 63;
     // the angle reaches tens of thousands of radians: form it and its sine / cosine in double
@@ -213,8 +246,8 @@ int sm_count() {
 int ensure_attrs() {
   const int dev = current_device();
   if (g_attr_set[dev]) return 0;
-  cudaError_t e = cudaFuncSetAttribute(gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_swiglu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
+  cudaError_t e = cudaFuncSetAttribute(gemv_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxIn * 4);
   if (e != cudaSuccess) return (int)e;
   g_attr_set[dev] = true;
   return 0;
@@ -224,6 +257,24 @@ int gemv_grid(int n_rows) {
   int blocks = (n_rows + per_block - 1) / per_block;
   const int cap = sm_count() * 2;   // two blocks of 16 warps per SM: few copies of x, many rows in flight
   return blocks < cap ? (blocks < 1 ? 1 : blocks) : cap;
+}
+
+// launch with programmatic stream serialisation (see dep_wait above)
+template <bool kSwiglu>
+int launch_gemv(const void* w, const void* x, int x_is_bf16, const void* norm_w, float eps, const float* residual, float* y,
+                int n_out, int n_in, void* stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(gemv_grid(n_out));
+  cfg.blockDim = dim3(kGemvThreads);
+  cfg.dynamicSmemBytes = (size_t)n_in * 4;
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return (int)cudaLaunchKernelEx(&cfg, gemv_kernel<kSwiglu>, static_cast<const uint4*>(w), x, x_is_bf16,
+                                 static_cast<const __nv_bfloat16*>(norm_w), eps, residual, y, n_out, n_in);
 }
 
 }  // namespace
@@ -240,28 +291,31 @@ int llh_gemv(const void* w, const void* x, int32_t x_is_bf16, const void* norm_w
              float* y, int32_t n_out, int32_t n_in, void* stream) {
   if (!w || !x || !y || n_out < 1 || n_in < 256 || n_in > kMaxIn || n_in % 256) return -1;
   if (int e = ensure_attrs()) return e;
-  gemv_kernel<<<gemv_grid(n_out), kGemvThreads, (size_t)n_in * 4, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const uint4*>(w), x, x_is_bf16, static_cast<const __nv_bfloat16*>(norm_w), eps, residual, y, n_out, n_in);
-  return (int)cudaGetLastError();
+  return launch_gemv<false>(w, x, x_is_bf16, norm_w, eps, residual, y, n_out, n_in, stream);
 }
 
 int llh_gemv_swiglu(const void* w_gate_up, const float* x, const void* norm_w, float eps, float* y, int32_t n_ff,
                     int32_t n_in, void* stream) {
   if (!w_gate_up || !x || !y || n_ff < 1 || n_in < 256 || n_in > kMaxIn || n_in % 256) return -1;
   if (int e = ensure_attrs()) return e;
-  gemv_swiglu_kernel<<<gemv_grid(n_ff), kGemvThreads, (size_t)n_in * 4, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const uint4*>(w_gate_up), x, static_cast<const __nv_bfloat16*>(norm_w), eps, y, n_ff, n_in);
-  return (int)cudaGetLastError();
+  return launch_gemv<true>(w_gate_up, x, 0, norm_w, eps, nullptr, y, n_ff, n_in, stream);
 }
 
 int llh_rope_split(const float* qkv, const int32_t* pos, float theta, void* q, void* k, void* v, int32_t n_q,
                    int32_t n_kv, void* stream) {
   if (!qkv || !pos || !q || !k || !v || n_q < 1 || n_kv < 1 || !(theta > 1.f)) return -1;
   const int n = (n_q + n_kv) * 64 + n_kv * 128;
-  rope_split_kernel<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      qkv, pos, theta, static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k), static_cast<__nv_bfloat16*>(v), n_q,
-      n_kv);
-  return (int)cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((n + 255) / 256);
+  cfg.blockDim = dim3(256);
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return (int)cudaLaunchKernelEx(&cfg, rope_split_kernel, qkv, pos, theta, static_cast<__nv_bfloat16*>(q),
+                                 static_cast<__nv_bfloat16*>(k), static_cast<__nv_bfloat16*>(v), (int)n_q, (int)n_kv);
 }
 
 int llh_embed(const void* table, const int32_t* token, float* x, int32_t hidden, int32_t vocab, void* stream) {
