@@ -69,6 +69,8 @@ def parse_args():
                          "pass; 'overlap' = behind the layer's attention in a second stream, beside the next layers'; "
                          "'one_stream' = attention, selection and rebuild of a layer in stream order")
     ap.add_argument("--no-overlap", action="store_true", help="same as --full-schedule one_stream")
+    ap.add_argument("--side-streams", type=int, default=8,
+                    help="deferred schedule: streams the layers' selections and rebuilds are spread over")
     ap.add_argument("--regions", type=int, default=0,
                     help="timed regions of K steps to take (0: as many as region_repeats() says; 1 keeps a profiler run short)")
     return ap.parse_args()
@@ -380,7 +382,7 @@ def measure_workload(args, w, dev, world, steps, warmup, level):
     launch_total = lambda: sum(c.launch_count for c in ctxs)
 
     overlapped = runner.OverlappedRefresh(layers) if schedule == "overlap" else None
-    deferred = runner.DeferredRefresh(layers) if schedule == "deferred" else None
+    deferred = runner.DeferredRefresh(layers, n_side=args.side_streams) if schedule == "deferred" else None
     qf, kf, vf = (lambda l: q_stage[l]), (lambda l: k_stage[l]), (lambda l: v_stage[l])
 
     def token(kind: str):
@@ -780,7 +782,7 @@ def run_ours(args):
             "fractions": fr,
             "in_graph_us_per_layer": g,
             "full_token_schedule": {"deferred": "the layers' attention passes follow each other; every layer's selection and "
-                                                "small-cache rebuild run after the last pass, spread over eight side streams "
+                                                "small-cache rebuild run after the last pass, spread over %d side streams " % args.side_streams +
                                                 "(one context per layer)",
                                     "overlap": "two streams: the layers' attention passes follow each other; a layer's "
                                                "selection and small-cache rebuild run behind its attention in a second stream",
