@@ -339,11 +339,17 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
  *                             other origin complete before a kernel of this library starts, unless
  *                             they themselves release their dependents early while still writing
  *                             the cache - turn the option off in that case); 0: never.
+ *   RKV_OPT_INTERLEAVE_TILES  1 (default): the full-cache pass deals the 64-position tiles of a (sequence,
+ *                             KV head) out to its CTAs in turn, so that every CTA walks the whole length and
+ *                             all carry the same number of tiles up to one; 0: each CTA takes one contiguous
+ *                             chunk.  Either way the assignment is fixed by the launch geometry, so results
+ *                             are reproducible bit for bit (the two settings differ in summation order).
  */
 #define RKV_OPT_SMALL_MIN_CHUNK 1
 #define RKV_OPT_DEPENDENT_LAUNCH 2
 #define RKV_OPT_SMALL_CLUSTER 3
 #define RKV_OPT_EARLY_CACHE_READ 4
+#define RKV_OPT_INTERLEAVE_TILES 5
 rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
 
 /*

@@ -180,7 +180,10 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   } else {
     p.chunk = choose_chunk(ctx, n_max, logits, &gx);
   }
-  if (chunk_out) *chunk_out = p.chunk;
+  // Streaming forms: the head's tiles are dealt out to the gx CTAs in turn; the partial slots in use are then
+  // min(tiles, gx), which is what the consumers of (chunk, gx) compute when they are told chunk = one tile.
+  p.interleave = (logits && ctx->interleave) ? 1 : 0;
+  if (chunk_out) *chunk_out = p.interleave ? rkv::kTile : p.chunk;
   if (gx_out) *gx_out = gx;
   p.q = q;
   p.row_offset = cache->row_offset;
@@ -312,6 +315,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->small_min_chunk = 256;
   ctx->small_cluster = 1;
   ctx->early_read = 1;
+  ctx->interleave = 1;
   ctx->gp = ctx->group <= 4 ? 4 : 8;
   ctx->workspace = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
@@ -686,6 +690,9 @@ rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value) {
       return RKV_OK;
     case RKV_OPT_EARLY_CACHE_READ:
       ctx->early_read = value != 0;
+      return RKV_OK;
+    case RKV_OPT_INTERLEAVE_TILES:
+      ctx->interleave = value != 0;
       return RKV_OK;
     default:
       return RKV_ERR_INVALID_ARG;

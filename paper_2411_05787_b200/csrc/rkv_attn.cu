@@ -240,11 +240,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     }
   }
 
+  // Which positions a CTA's t-th tile covers.  Contiguous: the CTA owns the chunk [split * chunk, (split + 1) * chunk).
+  // Interleaved (streaming forms, AttnParams::interleave): the tiles of a (sequence, KV head) are dealt out to its
+  // CTAs in turn - tile j goes to CTA j mod gridDim.x - so that every CTA walks the whole length, all CTAs carry the
+  // same number of tiles up to one, and which CTA sums which positions stays fixed by the launch geometry alone.
+  const bool il = kLogits && p.interleave != 0;
+  auto tile_pos = [&](int t) { return il ? (split + t * (int)gridDim.x) * kTile : split * p.chunk + t * kTile; };
   // One tile = K (and V) rows [y, y + 64) into stage t % kStg, completion on that stage's barrier.
   auto issue_tile = [&](int t, int64_t row_first, uint64_t policy) {
     const int s = t % kStg;
     const uint32_t dst = smem_base + s * kStageBytes, bar = bar_full + 8 * s;
-    const int y = (int)(row_first + (int64_t)t * kTile);
+    const int y = (int)(row_first + (int64_t)tile_pos(t));
     mbar_expect_tx(bar, kScoreOnly ? 2 * kHalfBytes : kStageBytes);
     tma_load_tile(dst, &tm_k, y, bar, policy);
     if (!kScoreOnly) tma_load_tile(dst + 2 * kHalfBytes, &tm_v, y, bar, policy);
@@ -259,12 +265,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     if (tid == 32 * kMW) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-      const int64_t row_s = roff + (int64_t)g * cap + (int64_t)split * p.chunk;
+      const int64_t row_s = roff + (int64_t)g * cap;
       for (int t = 0; t < n_tiles_spec; ++t) issue_tile(t, row_s, policy);
     }
   };
   int n_spec = 0;
-  if (p.spec != 0) n_spec = (p.chunk + kTile - 1) / kTile < kStg ? (p.chunk + kTile - 1) / kTile : kStg;
+  if (p.spec != 0) n_spec = (!il && (p.chunk + kTile - 1) / kTile < kStg) ? (p.chunk + kTile - 1) / kTile : kStg;
   if (kCluster && p.early != 0) issue_spec(n_spec);
   pdl_wait();
   pdl_launch();   // after the wait: at most one predecessor is ever in flight behind a kernel of this library
@@ -390,7 +396,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     take_len_ticket();
     return;
   }
-  const int start = split * p.chunk;
+  const int start = il ? split * kTile : split * p.chunk;   // the CTA's first position
   if (!kCluster && start >= n) {   // in a cluster an idle CTA still owns a slice of the output
     if (n_spec > 0) {
       if (tid == 0)
@@ -400,10 +406,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     take_len_ticket();
     return;
   }
-  const int end = (start + p.chunk < n) ? start + p.chunk : n;
-  const int n_tiles = (end > start) ? (end - start + kTile - 1) / kTile : 0;
+  const int end = (il || start + p.chunk >= n) ? n : start + p.chunk;
+  const int total_tiles = (n + kTile - 1) / kTile;
+  const int n_tiles = il ? (total_tiles > split ? (total_tiles - split + (int)gridDim.x - 1) / (int)gridDim.x : 0)
+                         : ((end > start) ? (end - start + kTile - 1) / kTile : 0);
   const int n_splits = (n + p.chunk - 1) / p.chunk;
-  const int64_t row0 = roff + (int64_t)g * cap + start;
+  const int64_t row0 = roff + (int64_t)g * cap;
 
   if (warp == kMW) {
     // ------------------------------------------------------------ copy warp
@@ -449,11 +457,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       ok = false;
       break;
     }
-    const int pos_base = start + t * kTile + band0;
+    const int pos_base = tile_pos(t) + band0;
     if (kAppend) {
       // The tile came from global memory, where the new row may not have landed yet: the warp that owns the
       // row writes it into the tile itself (same 128-byte swizzle as the copy engine uses).
-      const int rel = pos_new - (start + t * kTile);
+      const int rel = pos_new - tile_pos(t);
       if (rel >= 0 && rel < kTile && rel / kBand == wb) {
         const uint32_t at = smem_base + s * kStageBytes + (lane >> 4) * kHalfBytes + rel * 128 +
                             ((((lane & 15) >> 1) ^ (rel & 7)) << 4) + (lane & 1) * 8;

@@ -52,6 +52,7 @@ struct AttnParams {
   int32_t max_len;            // clamp for len[b]
   int32_t spec;               // 1: every CTA has work by construction, first tiles may be requested before len is read
   int32_t early;              // 1 (clustered step with spec): request them before the dependency wait as well
+  int32_t interleave;         // 1 (streaming forms): tile j of a (sequence, KV head) goes to CTA j mod gridDim.x
   float scale;
   // fused append (clustered partial step only): the new token's rows and where they go
   const void* k_new;          // bf16 [B][Hkv][128]
@@ -242,6 +243,7 @@ struct rkv_ctx {
   int small_min_chunk;
   int small_cluster;   // 1: the partial step merges its splits inside a thread-block cluster when the length allows
   int early_read;      // 1: the clustered partial step may request its cache rows before its dependency wait
+  int interleave;      // 1: the full-cache pass deals a head's tiles out to its CTAs in turn
   // geometry of the last rkv_full_attention, for the rkv_select_topk that completes it
   struct { bool valid; int chunk, gx, n_max; const void* full_k; const int32_t* active; } pending_full;
   int gp;              // floats per position in the logit scratch

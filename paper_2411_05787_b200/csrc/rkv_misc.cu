@@ -203,7 +203,8 @@ __global__ void __launch_bounds__(128) fold_kernel(const float* __restrict__ par
   if (act == 0) return;
   n = n < lim ? n : lim;            // the clamp of the streaming pass
   if (n <= 0) return;               // nothing cached: the streaming pass has written zeros
-  const int n_splits = (n + chunk - 1) / chunk;
+  int n_splits = (n + chunk - 1) / chunk;
+  if (n_splits > grid_splits) n_splits = grid_splits;   // (interleaved tiles: every CTA of the pass carries some)
   if (warp == 0) {   // weights of the splits in use, their sum of denominators
     float M = -INFINITY, L = 0.f;
 #pragma unroll
