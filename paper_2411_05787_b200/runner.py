@@ -264,3 +264,29 @@ class LayerBatchedSmall:
         self.ctx.append_small_step(q_all.view(n, self.n_q, HEAD_DIM), k_all.view(n, self.n_kv, HEAD_DIM),
                                    v_all.view(n, self.n_kv, HEAD_DIM), None, self.cache_c,
                                    out_all.view(n, self.n_q, HEAD_DIM), max_len_hint=self.hint)
+
+
+class LayerBatchedFull:
+    """rkv_full_step of ALL layers of a token as one call: the full caches of every (layer, sequence) live in one K
+    and one V buffer (synth.alloc_layer_stack) and one context sees them as layers x B sequences.
+
+    Like LayerBatchedSmall this is a measuring form, legal only for synthetic per-layer queries that do not depend on
+    each other: it shows what the attention pass, the score pass and the selection stream when launch and dependency
+    latencies are amortised over all layers."""
+
+    def __init__(self, stack: LayerCache, n_layers: int, k_small: list, n_q_heads: int, n_kv_heads: int, max_len_hint: int):
+        dev = stack.k.device
+        n = stack.row_offset.shape[0]
+        self.n, self.n_q, self.n_kv, self.hint = n, n_q_heads, n_kv_heads, max_len_hint
+        self.k_max = max(max(k_small), 1)
+        self.ctx = rkv.Context(n, n_q_heads, n_kv_heads, max_len_hint, self.k_max)
+        self.full_c = rkv.cache_struct(stack.k, stack.v, stack.row_offset, stack.cap, stack.len)
+        self.k_small = torch.tensor(list(k_small) * n_layers, dtype=torch.int32, device=dev)
+        self.topk_idx = torch.full((n, n_kv_heads, self.k_max), -2, dtype=torch.int32, device=dev)
+        self.out = torch.zeros((n, n_q_heads, HEAD_DIM), dtype=torch.bfloat16, device=dev)
+
+    def full_step(self, q_all):
+        """q_all [layers, B, Hq, 128]: attention over every cache, scores and top-K, one call (three launches)."""
+        self.ctx.full_step(q_all.view(self.n, self.n_q, HEAD_DIM), self.full_c, self.k_small, self.k_max, self.out,
+                           self.topk_idx, max_len_hint=self.hint)
+        return self.out

@@ -180,12 +180,37 @@ def heavy_positions(w: Workload, layer: int, b: int, epoch: int, n_ctx: int, dev
     return torch.stack(rows).to(device)
 
 
-def fill_layer(w: Workload, layer: int, device, extra_cap: int | None = None) -> LayerCache:
-    """Random K/V for all context positions of one layer (noise part only)."""
+def layer_view(stack: LayerCache, layer: int, batch: int) -> LayerCache:
+    """One layer's sequences of a cache that holds `batch` sequences per layer for several layers in one K and one V
+    buffer: the same buffers, the layer's slice of the index tensors (row offsets stay global)."""
+    sl = slice(layer * batch, (layer + 1) * batch)
+    return LayerCache(stack.k, stack.v, stack.row_offset[sl], stack.cap[sl], stack.len[sl])
+
+
+def alloc_layer_stack(w: Workload, device, extra_cap: int | None = None) -> LayerCache:
+    """All layers' full caches in ONE K and ONE V buffer: layers x batch sequences."""
+    extra = w.steps + 1 if extra_cap is None else extra_cap
+    caps = [l + extra for l in w.lens] * w.n_layers
+    return alloc_cache(caps, list(w.lens) * w.n_layers, w.n_kv_heads, device)
+
+
+def fill_layer(w: Workload, layer: int, device, extra_cap: int | None = None, into: LayerCache | None = None) -> LayerCache:
+    """Random K/V for all context positions of one layer (noise part only).  into: a layer_view() to fill in place."""
     extra = w.steps + 1 if extra_cap is None else extra_cap
     caps = [l + extra for l in w.lens]
-    cache = alloc_cache(caps, list(w.lens), w.n_kv_heads, device)
     g = _gen(w.seed * 7907 + layer * 31 + 1, device)
+    if into is not None:
+        r0 = int(into.row_offset[0])
+        r1 = r0 + w.n_kv_heads * sum(caps)
+        assert into.cap.tolist() == caps
+        step = 1 << 22
+        for t in (into.k, into.v):
+            for a in range(r0, r1, step):
+                b = min(r1, a + step)
+                t[a:b] = (torch.randn((b - a, HEAD_DIM), generator=g, device=device,
+                                      dtype=torch.float32) * w.kv_scale).to(torch.bfloat16)
+        return into
+    cache = alloc_cache(caps, list(w.lens), w.n_kv_heads, device)
     # chunked so that the fp32 temporaries stay small next to the bf16 result
     step = 1 << 22
     for t in (cache.k, cache.v):

@@ -974,6 +974,42 @@ def test_layer_batched_partial_step_every_layer_and_sequence(mods):
         assert torch.equal(lb.cache.k[offs[2 * l] + cap0: offs[2 * l] + cap0 + 200], st.small.k[cap0: cap0 + 200])
 
 
+def test_layer_batched_full_step_every_layer_and_sequence(mods):
+    """rkv_full_step of all layers in one call (bench.py's layer-batched measurement): the full caches of three
+    layers x two ragged sequences in one K and one V buffer, one context that sees six sequences; outputs and top-K
+    sets of every (layer, sequence) against the oracle (the per-layer calls on the layers' views of the same buffers
+    split the caches differently, so their log-sum-exps - and with them keys one ulp apart - may differ in the last
+    bit: both are held to the oracle, not to each other)."""
+    rkv, runner, synth = mods
+    dev = torch.device("cuda")
+    w = synth.Workload("stack", 3, 28, 4, [3000, 700], [300, 64], 4, "fixed", 10, rho=[0.9, 0.9], seed=11)
+    stack = synth.alloc_layer_stack(w, dev)
+    qs = []
+    per_layer = []
+    for l in range(w.n_layers):
+        view = synth.fill_layer(w, l, dev, into=synth.layer_view(stack, l, w.batch))
+        q = synth.query_trajectory(w, l)[0].to(dev)
+        synth.plant_heavy(w, view, l, q)
+        qs.append(q)
+        ctx = rkv.Context(w.batch, w.n_q_heads, w.n_kv_heads, max(w.lens) + 8, max(w.k_small) + 8)
+        st = runner.LayerState(ctx, view, list(w.k_small), 8, w.n_q_heads, w.n_kv_heads, want_scores=False)
+        st.refresh(q)
+        assert ctx.device_status() == 0
+        per_layer.append((ctx, st, view))
+    q_all = torch.stack(qs)                                       # [layers, B, Hq, 128]
+    lb = runner.LayerBatchedFull(stack, w.n_layers, list(w.k_small), w.n_q_heads, w.n_kv_heads, max(w.lens) + 8)
+    out = lb.full_step(q_all).view(w.n_layers, w.batch, w.n_q_heads, 128)
+    assert lb.ctx.device_status() == 0
+    idx = lb.topk_idx.view(w.n_layers, w.batch, w.n_kv_heads, -1)
+    for l, (ctx, st, view) in enumerate(per_layer):
+        for b, n in enumerate(w.lens):
+            o_out, o_score, o_idx, _ = oracle_full(view, b, n, q_all[l, b], w.n_kv_heads, w.k_small[b])
+            check_out(out[l, b], o_out, f"layer {l} seq {b}")
+            for g in range(w.n_kv_heads):
+                why = O.check_topk_set(o_score[g], w.k_small[b], idx[l, b, g, : w.k_small[b]].cpu().numpy())
+                assert why is None, f"layer {l} seq {b} head {g}: {why}"
+
+
 def test_config3_full_size_single_step(mods):
     rkv, runner, synth = mods
     w = synth.scaled(synth.config3(n_layers=1), steps=2, stride=1)
