@@ -70,6 +70,7 @@ def parse_args():
                          "'one_stream' = attention, selection and rebuild of a layer in stream order")
     ap.add_argument("--no-overlap", action="store_true", help="same as --full-schedule one_stream")
     ap.add_argument("--no-interleave", action="store_true", help="full-cache pass: one contiguous chunk per CTA")
+    ap.add_argument("--select-keys-per-cta", type=int, default=0, help="override RKV_OPT_SELECT_KEYS_PER_CTA (0: default)")
     ap.add_argument("--side-streams", type=int, default=8,
                     help="deferred schedule: streams the layers' selections and rebuilds are spread over")
     ap.add_argument("--regions", type=int, default=0,
@@ -349,6 +350,8 @@ def measure_workload(args, w, dev, world, steps, warmup, level):
             c.set_option(rkv.OPT_SMALL_CLUSTER, 0)
         if args.no_interleave:
             c.set_option(rkv.OPT_INTERLEAVE_TILES, 0)
+        if args.select_keys_per_cta:
+            c.set_option(rkv.OPT_SELECT_KEYS_PER_CTA, args.select_keys_per_cta)
 
     # per-token inputs: one contiguous block per token = all layers' q, then all k_new, then all v_new, so that
     # one copy stages a token and the calls get contiguous views.  Queries follow the workload's AR(1) process

@@ -344,12 +344,17 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
  *                             all carry the same number of tiles up to one; 0: each CTA takes one contiguous
  *                             chunk.  Either way the assignment is fixed by the launch geometry, so results
  *                             are reproducible bit for bit (the two settings differ in summation order).
+ *   RKV_OPT_SELECT_KEYS_PER_CTA  keys (positions) one CTA of a top-K cluster takes, 512..40960; default 4096.
+ *                             The cluster has 1, 2, 4 or 8 CTAs per (sequence, KV head): fewer keys per CTA give
+ *                             the shortest chain for a single selection, more keys per CTA occupy fewer SMs
+ *                             when many selections run side by side.  The selected set does not depend on it.
  */
 #define RKV_OPT_SMALL_MIN_CHUNK 1
 #define RKV_OPT_DEPENDENT_LAUNCH 2
 #define RKV_OPT_SMALL_CLUSTER 3
 #define RKV_OPT_EARLY_CACHE_READ 4
 #define RKV_OPT_INTERLEAVE_TILES 5
+#define RKV_OPT_SELECT_KEYS_PER_CTA 6
 rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
 
 /*

@@ -316,6 +316,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->small_cluster = 1;
   ctx->early_read = 1;
   ctx->interleave = 1;
+  ctx->select_keys_per_cta = 4096;
   ctx->gp = ctx->group <= 4 ? 4 : 8;
   ctx->workspace = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
@@ -456,7 +457,7 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   sp.n_kv_heads = ctx->cfg.n_kv_heads;
   sp.k_max = k_max;
   sp.max_len = n_max;
-  const int cluster = rkv::select_cluster_for(n_max);
+  const int cluster = rkv::select_cluster_for(n_max, ctx->select_keys_per_cta);
   sp.keys_per_thread = rkv::select_keys_per_thread(n_max, cluster);
   sp.per_fixed = ctx->cfg.n_seq == 1 ? 1 : 0;
   cudaError_t e;
@@ -693,6 +694,10 @@ rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value) {
       return RKV_OK;
     case RKV_OPT_INTERLEAVE_TILES:
       ctx->interleave = value != 0;
+      return RKV_OK;
+    case RKV_OPT_SELECT_KEYS_PER_CTA:
+      if (value < 512 || value > rkv::kSelectMaxKeysPerCta) return RKV_ERR_INVALID_ARG;
+      ctx->select_keys_per_cta = value;
       return RKV_OK;
     default:
       return RKV_ERR_INVALID_ARG;

@@ -131,7 +131,7 @@ cudaError_t launch_evict_order(const uint32_t* win_keys, int win_stride, const i
 cudaError_t launch_score(const ScoreParams& p, int n_seq, cudaStream_t st);
 cudaError_t launch_select(const SelectParams& p, int n_seq, int cluster, cudaStream_t st);
 int score_slice_for(int n_max, int problems, int sm_count);   // positions per CTA of the score pass
-int select_cluster_for(int n_max);                            // CTAs per (sequence, KV head) of the selection
+int select_cluster_for(int n_max, int keys_per_cta);          // CTAs per (sequence, KV head) of the selection
 int select_keys_per_thread(int n_max, int cluster);           // keys per thread of a CTA of such a cluster
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
@@ -244,6 +244,7 @@ struct rkv_ctx {
   int small_cluster;   // 1: the partial step merges its splits inside a thread-block cluster when the length allows
   int early_read;      // 1: the clustered partial step may request its cache rows before its dependency wait
   int interleave;      // 1: the full-cache pass deals a head's tiles out to its CTAs in turn
+  int select_keys_per_cta;   // keys one CTA of a selection cluster takes (about): fewer = shorter chain, more = fewer CTAs
   // geometry of the last rkv_full_attention, for the rkv_select_topk that completes it
   struct { bool valid; int chunk, gx, n_max; const void* full_k; const int32_t* active; } pending_full;
   int gp;              // floats per position in the logit scratch

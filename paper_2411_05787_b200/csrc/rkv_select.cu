@@ -937,9 +937,9 @@ cudaError_t launch_score_agg(const ScoreParams& p, dim3 grid, size_t smem, cudaS
 
 }  // namespace
 
-int select_cluster_for(int n_max) {   // CTAs per (sequence, KV head): about 4096 keys each, a power of two up to 8
+int select_cluster_for(int n_max, int keys_per_cta) {   // CTAs per (sequence, KV head): a power of two up to 8
   int c = 1;
-  while (c < kSelectCluster && (int64_t)c * 4096 < n_max) c <<= 1;
+  while (c < kSelectCluster && ((int64_t)c * keys_per_cta < n_max || (int64_t)c * kSelectMaxKeysPerCta < n_max)) c <<= 1;
   return c;
 }
 

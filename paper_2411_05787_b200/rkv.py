@@ -26,6 +26,7 @@ EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", 
            "rkv_append_full_attention"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER, OPT_EARLY_CACHE_READ, OPT_INTERLEAVE_TILES = 1, 2, 3, 4, 5
+OPT_SELECT_KEYS_PER_CTA = 6
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger", "fold", "score"]
 
 
