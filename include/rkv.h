@@ -332,13 +332,14 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
  *   RKV_OPT_DEPENDENT_LAUNCH  1 (default): kernels are launched with programmatic stream
  *                             serialisation so that a kernel's launch overlaps the tail of its
  *                             predecessor; 0: plain stream order.  Process-wide.
- *   RKV_OPT_EARLY_CACHE_READ  1 (default): the clustered partial step may request its share of the
- *                             attended cache before its stream dependency has resolved, when the
- *                             library's previous launch on the same stream wrote no row of that
- *                             cache (the library keeps a host-side record per stream; kernels of
- *                             other origin complete before a kernel of this library starts, unless
- *                             they themselves release their dependents early while still writing
- *                             the cache - turn the option off in that case); 0: never.
+ *   RKV_OPT_EARLY_CACHE_READ  1 (default): an attention kernel may request its first tiles of the attended cache
+ *                             before its stream dependency has resolved - the clustered partial step its whole
+ *                             share, the full-cache pass (one sequence, no mask) the first one to three tiles per
+ *                             CTA - when the library's previous launch on the same stream wrote no row of that
+ *                             cache (the library keeps a host-side record per stream; the row a call appends
+ *                             itself is patched in on chip; kernels of other origin complete before a kernel of
+ *                             this library starts, unless they themselves release their dependents early while
+ *                             still writing the cache - turn the option off in that case); 0: never.
  *   RKV_OPT_INTERLEAVE_TILES  1 (default): the full-cache pass deals the 64-position tiles of a (sequence,
  *                             KV head) out to its CTAs in turn, so that every CTA walks the whole length and
  *                             all carry the same number of tiles up to one; 0: each CTA takes one contiguous

@@ -209,6 +209,10 @@ rkv_status run_attention(rkv_ctx* ctx, const void* q, const rkv_cache* cache, co
   // Early cache read: only when the launch before this one on the stream leaves the attended cache alone (a
   // gather or an append into it forbids it; so does an unknown history).
   p.early = (cluster && p.spec != 0 && ctx->early_read && rkv::early_read_safe(st, cache)) ? 1 : 0;
+  // The streaming pass does the same with its first tiles: all stages of its ring, or - when the launch before it
+  // is the short merge kernel of the previous pass, whose few loads would queue behind them - one tile.
+  if (logits && p.spec != 0 && ctx->early_read && rkv::early_read_safe(st, cache))
+    p.early = rkv::last_launch_was_fold(st) ? 1 : rkv::kStages;
   if (app != nullptr) {   // the clustered partial step and the full step's attention pass can take the append with them
     if (!cluster && !(logits && !score_only)) return RKV_ERR_INVALID_ARG;
     p.k_new = app->k_new;
@@ -253,7 +257,7 @@ bool g_use_pdl = true;
 namespace {
 struct ByteRange { uintptr_t lo, hi; };
 std::mutex g_writes_mu;
-struct LastLaunch { std::vector<ByteRange> writes; };
+struct LastLaunch { std::vector<ByteRange> writes; bool fold = false; };
 std::map<cudaStream_t, LastLaunch> g_writes;   // per stream: the library's last launch
 bool g_writes_lost = false;   // the record was dropped once: a stream without an entry is then unknown, not clean
 constexpr size_t kMaxTrackedStreams = 1024;
@@ -265,16 +269,23 @@ void add_ranges(std::vector<ByteRange>* v, const rkv_cache* c) {
 }
 }  // namespace
 
-void note_launch(cudaStream_t st, const rkv_cache* a, const rkv_cache* b) {
+void note_launch(cudaStream_t st, const rkv_cache* a, const rkv_cache* b, bool fold) {
   std::lock_guard<std::mutex> lock(g_writes_mu);
   if (g_writes.size() >= kMaxTrackedStreams && g_writes.find(st) == g_writes.end()) {
     g_writes.clear();
     g_writes_lost = true;
   }
   LastLaunch& v = g_writes[st];
+  v.fold = fold;
   v.writes.clear();
   add_ranges(&v.writes, a);
   add_ranges(&v.writes, b);
+}
+
+bool last_launch_was_fold(cudaStream_t st) {
+  std::lock_guard<std::mutex> lock(g_writes_mu);
+  auto it = g_writes.find(st);
+  return it != g_writes.end() && it->second.fold;
 }
 
 bool early_read_safe(cudaStream_t st, const rkv_cache* c) {
@@ -385,7 +396,7 @@ static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cac
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "fold launch");
     ctx->launches += 1;
-    rkv::note_launch(st, nullptr, nullptr);
+    rkv::note_launch(st, nullptr, nullptr, true);
   }
   ctx->pending_full = {true, chunk, gx, n_max, full->k, active};
   return RKV_OK;

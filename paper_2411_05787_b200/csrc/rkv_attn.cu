@@ -259,22 +259,35 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // this one on the stream does not write this cache (p.early), they are requested even before the
   // dependency wait: a clustered step usually sits at that wait while its predecessor runs, and a CTA's
   // share of the cache takes longer to arrive (about 64 bytes per cycle per SM) than the rest of the step
-  // takes to get ready.  Every kernel of this library releases its dependents only after its own wait, so the
-  // predecessor is the only kernel that can still be running at that point.
-  auto issue_spec = [&](int n_tiles_spec) {
+  // takes to get ready; the streaming pass gains the latency of its first tiles (p.early says how many: a
+  // predecessor with memory traffic of its own is slowed by what is queued in front of it).  Every kernel of
+  // this library releases its dependents only after its own wait, so the predecessor is the only kernel that
+  // can still be running at that point.
+  auto issue_spec = [&](int t_first, int t_end) {
     if (tid == 32 * kMW) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
       const int64_t row_s = roff + (int64_t)g * cap;
-      for (int t = 0; t < n_tiles_spec; ++t) issue_tile(t, row_s, policy);
+      for (int t = t_first; t < t_end; ++t) issue_tile(t, row_s, policy);
     }
   };
   int n_spec = 0;
   if (p.spec != 0) n_spec = (!il && (p.chunk + kTile - 1) / kTile < kStg) ? (p.chunk + kTile - 1) / kTile : kStg;
-  if (kCluster && p.early != 0) issue_spec(n_spec);
+  // tiles requested above the dependency wait: all of them in the clustered step, p.early of them in the streaming forms
+  int n_early = 0;
+  if (kCluster) {
+    if (p.early != 0) issue_spec(0, n_spec);
+  } else if (kLogits && p.early != 0) {
+    n_early = p.early < n_spec ? p.early : n_spec;
+    issue_spec(0, n_early);
+  }
   pdl_wait();
   pdl_launch();   // after the wait: at most one predecessor is ever in flight behind a kernel of this library
-  if (!(kCluster && p.early != 0)) issue_spec(n_spec);
+  if (kCluster) {
+    if (p.early == 0) issue_spec(0, n_spec);
+  } else {
+    issue_spec(n_early, n_spec);
+  }
 
   // (When the host knows that every CTA of the grid has work - no mask; one sequence, or a cluster per head - the
   // chunk of this CTA follows from the launch geometry alone, so its first tiles have been requested above, before

@@ -51,7 +51,8 @@ struct AttnParams {
   int32_t max_splits;
   int32_t max_len;            // clamp for len[b]
   int32_t spec;               // 1: every CTA has work by construction, first tiles may be requested before len is read
-  int32_t early;              // 1 (clustered step with spec): request them before the dependency wait as well
+  int32_t early;              // > 0 (with spec): request them before the dependency wait as well - all of them in the
+                              // clustered step, this many in the streaming forms
   int32_t interleave;         // 1 (streaming forms): tile j of a (sequence, KV head) goes to CTA j mod gridDim.x
   float scale;
   // fused append (clustered partial step only): the new token's rows and where they go
@@ -191,8 +192,9 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // NULL).  early_read_safe: the launch before this one on the stream writes no row of cache c, or nothing of
 // this library was ever launched on the stream (kernels of other origin complete before a kernel of this
 // library starts).
-void note_launch(cudaStream_t st, const rkv_cache* a, const rkv_cache* b);
+void note_launch(cudaStream_t st, const rkv_cache* a, const rkv_cache* b, bool fold = false);
 bool early_read_safe(cudaStream_t st, const rkv_cache* c);
+bool last_launch_was_fold(cudaStream_t st);   // the library's last launch on the stream was the full step's merge kernel
 
 cudaError_t prepare_attention();  // one-time function attributes (dynamic shared memory sizes)
 cudaError_t prepare_select();
@@ -242,7 +244,7 @@ struct rkv_ctx {
   int sm_count;
   int small_min_chunk;
   int small_cluster;   // 1: the partial step merges its splits inside a thread-block cluster when the length allows
-  int early_read;      // 1: the clustered partial step may request its cache rows before its dependency wait
+  int early_read;      // 1: the attention kernels may request their first cache tiles before their dependency wait
   int interleave;      // 1: the full-cache pass deals a head's tiles out to its CTAs in turn
   int select_keys_per_cta;   // keys one CTA of a selection cluster takes (about): fewer = shorter chain, more = fewer CTAs
   // geometry of the last rkv_full_attention, for the rkv_select_topk that completes it
