@@ -71,7 +71,12 @@ def parse_args():
     ap.add_argument("--no-overlap", action="store_true", help="same as --full-schedule one_stream")
     ap.add_argument("--no-interleave", action="store_true", help="full-cache pass: one contiguous chunk per CTA")
     ap.add_argument("--select-keys-per-cta", type=int, default=0, help="override RKV_OPT_SELECT_KEYS_PER_CTA (0: default)")
-    ap.add_argument("--side-streams", type=int, default=8,
+    ap.add_argument("--score-slice", type=int, default=0, help="override RKV_OPT_SCORE_SLICE (0: default)")
+    ap.add_argument("--deferred-keys-per-cta", type=int, default=16384,
+                    help="deferred schedule with 8+ layers: RKV_OPT_SELECT_KEYS_PER_CTA of the tail's selections (0: the contexts')")
+    ap.add_argument("--deferred-score-slice", type=int, default=4096,
+                    help="deferred schedule with 8+ layers: RKV_OPT_SCORE_SLICE of the tail's score passes (0: the contexts')")
+    ap.add_argument("--side-streams", type=int, default=16,
                     help="deferred schedule: streams the layers' selections and rebuilds are spread over")
     ap.add_argument("--regions", type=int, default=0,
                     help="timed regions of K steps to take (0: as many as region_repeats() says; 1 keeps a profiler run short)")
@@ -352,6 +357,8 @@ def measure_workload(args, w, dev, world, steps, warmup, level):
             c.set_option(rkv.OPT_INTERLEAVE_TILES, 0)
         if args.select_keys_per_cta:
             c.set_option(rkv.OPT_SELECT_KEYS_PER_CTA, args.select_keys_per_cta)
+        if args.score_slice:
+            c.set_option(rkv.OPT_SCORE_SLICE, args.score_slice)
 
     # per-token inputs: one contiguous block per token = all layers' q, then all k_new, then all v_new, so that
     # one copy stages a token and the calls get contiguous views.  Queries follow the workload's AR(1) process
@@ -391,7 +398,8 @@ def measure_workload(args, w, dev, world, steps, warmup, level):
     launch_total = lambda: sum(c.launch_count for c in ctxs)
 
     overlapped = runner.OverlappedRefresh(layers) if schedule == "overlap" else None
-    deferred = runner.DeferredRefresh(layers, n_side=args.side_streams) if schedule == "deferred" else None
+    deferred = (runner.DeferredRefresh(layers, n_side=args.side_streams, select_keys_per_cta=args.deferred_keys_per_cta,
+                                       score_slice=args.deferred_score_slice) if schedule == "deferred" else None)
     qf, kf, vf = (lambda l: q_stage[l]), (lambda l: k_stage[l]), (lambda l: v_stage[l])
 
     def token(kind: str):

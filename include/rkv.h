@@ -349,6 +349,11 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
  *                             The cluster has 1, 2, 4 or 8 CTAs per (sequence, KV head): fewer keys per CTA give
  *                             the shortest chain for a single selection, more keys per CTA occupy fewer SMs
  *                             when many selections run side by side.  The selected set does not depend on it.
+ *   RKV_OPT_SCORE_SLICE       positions one CTA of the score pass takes: 0 (default) = chosen per launch (the
+ *                             smallest of 1024, 2048, 4096, 8192 that keeps the grid near four CTAs per SM), or
+ *                             one of those four values.  Longer slices mean fewer CTAs that each pay the
+ *                             log-sum-exp and the histogram flush once: slower for a single selection, cheaper
+ *                             when many run side by side.  Keys, scores and the selected set do not depend on it.
  */
 #define RKV_OPT_SMALL_MIN_CHUNK 1
 #define RKV_OPT_DEPENDENT_LAUNCH 2
@@ -356,7 +361,10 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
 #define RKV_OPT_EARLY_CACHE_READ 4
 #define RKV_OPT_INTERLEAVE_TILES 5
 #define RKV_OPT_SELECT_KEYS_PER_CTA 6
+#define RKV_OPT_SCORE_SLICE 7
 rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value);
+/* The option's current value (host memory); RKV_ERR_INVALID_ARG for an unknown option or a NULL pointer. */
+rkv_status rkv_get_option(const rkv_ctx* ctx, int32_t option, int32_t* value);
 
 /*
  * Optional per-kernel timing (no counterpart in the paper, which reports wall-clock decode time

@@ -328,6 +328,7 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->early_read = 1;
   ctx->interleave = 1;
   ctx->select_keys_per_cta = 4096;
+  ctx->score_slice = 0;
   ctx->gp = ctx->group <= 4 ? 4 : 8;
   ctx->workspace = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
@@ -446,7 +447,7 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   cp.agg = ctx->cfg.agg;
   cp.k_max = k_max;
   cp.max_len = n_max;
-  cp.slice = rkv::score_slice_for(n_max, bg, ctx->sm_count);
+  cp.slice = ctx->score_slice != 0 ? ctx->score_slice : rkv::score_slice_for(n_max, bg, ctx->sm_count);
   cp.n_slices = (n_max + cp.slice - 1) / cp.slice;
   cp.chunk = chunk;
   cp.max_splits = ctx->max_splits;
@@ -710,8 +711,27 @@ rkv_status rkv_set_option(rkv_ctx* ctx, int32_t option, int32_t value) {
       if (value < 512 || value > rkv::kSelectMaxKeysPerCta) return RKV_ERR_INVALID_ARG;
       ctx->select_keys_per_cta = value;
       return RKV_OK;
+    case RKV_OPT_SCORE_SLICE:
+      if (value != 0 && value != 1024 && value != 2048 && value != 4096 && value != rkv::kSelectMaxSlice)
+        return RKV_ERR_INVALID_ARG;
+      ctx->score_slice = value;
+      return RKV_OK;
     default:
       return RKV_ERR_INVALID_ARG;
+  }
+}
+
+rkv_status rkv_get_option(const rkv_ctx* ctx, int32_t option, int32_t* value) {
+  if (!ctx || !value) return RKV_ERR_INVALID_ARG;
+  switch (option) {
+    case RKV_OPT_SMALL_MIN_CHUNK: *value = ctx->small_min_chunk; return RKV_OK;
+    case RKV_OPT_SMALL_CLUSTER: *value = ctx->small_cluster; return RKV_OK;
+    case RKV_OPT_DEPENDENT_LAUNCH: *value = rkv::g_use_pdl ? 1 : 0; return RKV_OK;
+    case RKV_OPT_EARLY_CACHE_READ: *value = ctx->early_read; return RKV_OK;
+    case RKV_OPT_INTERLEAVE_TILES: *value = ctx->interleave; return RKV_OK;
+    case RKV_OPT_SELECT_KEYS_PER_CTA: *value = ctx->select_keys_per_cta; return RKV_OK;
+    case RKV_OPT_SCORE_SLICE: *value = ctx->score_slice; return RKV_OK;
+    default: return RKV_ERR_INVALID_ARG;
   }
 }
 

@@ -247,6 +247,7 @@ struct rkv_ctx {
   int early_read;      // 1: the attention kernels may request their first cache tiles before their dependency wait
   int interleave;      // 1: the full-cache pass deals a head's tiles out to its CTAs in turn
   int select_keys_per_cta;   // keys one CTA of a selection cluster takes (about): fewer = shorter chain, more = fewer CTAs
+  int score_slice;           // positions per CTA of the score pass; 0: chosen per launch
   // geometry of the last rkv_full_attention, for the rkv_select_topk that completes it
   struct { bool valid; int chunk, gx, n_max; const void* full_k; const int32_t* active; } pending_full;
   int gp;              // floats per position in the logit scratch

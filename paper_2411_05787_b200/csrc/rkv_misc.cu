@@ -7,65 +7,100 @@
 namespace rkv {
 namespace {
 
-// small.K[b][g][r] = full.K[b][g][idx[b][g][r]] (and V): 16 threads move one 256-byte row as uint4.
-__global__ void __launch_bounds__(256) gather_kernel(const int32_t* __restrict__ topk_idx,
-                                                     const int32_t* __restrict__ k_small, int k_max,
-                                                     CacheDev full, CacheDev small_cache,
-                                                     const int32_t* __restrict__ active, int n_kv_heads,
-                                                     int32_t* status) {
-  const int b = blockIdx.z, g = blockIdx.y;
-  pdl_wait();
-  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
-  if (active != nullptr && active[b] == 0) return;
-  const int n = full.len[b];
-  int m = k_small[b];
-  if (m > k_max) m = k_max;
-  if (m > n) m = n;
-  if (m < 0) m = 0;
-  const int cap_s = small_cache.cap[b];
-  if (m > cap_s) {
-    m = cap_s;
-    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(status, RKV_DEV_LEN_CLAMPED);
-  }
-  if (blockIdx.x == 0 && g == 0 && threadIdx.x == 0) small_cache.len[b] = m;
-  const int cap_f = full.cap[b];
+__device__ __forceinline__ uint32_t smem_u32(const void* ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
+
+// small.K[b][g][r] = full.K[b][g][idx[b][g][r]] (and V).  One CTA of 128 threads per tile of 64 output rows: the
+// rows come into shared memory with 16-byte asynchronous copies (no register holds data, so the 32 KB of a tile are
+// in flight at once and the CTA fits beside register-heavy kernels), and since the output rows of a tile are
+// contiguous they leave with ONE bulk copy per cache.  Indices are requested together with the sizes (every slot
+// below k_max is readable), so the kernel costs two memory round trips.
+constexpr int kGatherRows = 64;
+constexpr int kGatherThreads = 128;
+
+__global__ void __launch_bounds__(kGatherThreads, 16) gather_kernel(const int32_t* __restrict__ topk_idx,
+                                                                const int32_t* __restrict__ k_small, int k_max,
+                                                                CacheDev full, CacheDev small_cache,
+                                                                const int32_t* __restrict__ active, int n_kv_heads,
+                                                                int32_t* status) {
+  __shared__ __align__(128) uint4 tile_k[kGatherRows * 16];
+  __shared__ __align__(128) uint4 tile_v[kGatherRows * 16];
+  const int b = blockIdx.z, g = blockIdx.y, tid = threadIdx.x;
+  const int sub = tid & 15, slot = tid >> 4;   // thread: 16 bytes of rows slot, slot + 8, ..
+  const int r_base = blockIdx.x * kGatherRows;
+  constexpr int kPer = kGatherRows / (kGatherThreads / 16);   // rows per thread
+  // the caches' geometry is never written by a kernel: read above the dependency wait
+  const int cap_s = small_cache.cap[b], cap_f = full.cap[b];
   const int64_t src0 = full.row_offset[b] + (int64_t)g * cap_f;
   const int64_t dst0 = small_cache.row_offset[b] + (int64_t)g * cap_s;
   const int32_t* idx = topk_idx + (int64_t)(b * n_kv_heads + g) * k_max;
+  pdl_wait();
+  pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
+  const int act = active != nullptr ? __ldcg(active + b) : 1;
+  const int n = __ldcg(full.len + b);
+  int m = __ldcg(k_small + b);
+  int j[kPer];
+#pragma unroll
+  for (int u = 0; u < kPer; ++u) {
+    const int r = r_base + slot + u * (kGatherThreads / 16);
+    j[u] = r < k_max ? __ldcg(idx + r) : -1;
+  }
+  if (act == 0) return;
+  if (m > k_max) m = k_max;
+  if (m > n) m = n;
+  if (m < 0) m = 0;
+  if (m > cap_s) {
+    m = cap_s;
+    if (tid == 0 && blockIdx.x == 0) atomicOr(status, RKV_DEV_LEN_CLAMPED);
+  }
+  if (blockIdx.x == 0 && g == 0 && tid == 0) small_cache.len[b] = m;
+  if (r_base >= m) return;
   const uint4* fk = static_cast<const uint4*>(full.k);
   const uint4* fv = static_cast<const uint4*>(full.v);
-  uint4* sk = static_cast<uint4*>(small_cache.k);
-  uint4* sv = static_cast<uint4*>(small_cache.v);
-  const int sub = threadIdx.x & 15;
-  // four rows per thread and round: first all indices, then all eight 16-byte loads, then the stores, so that a
-  // round costs two memory round trips however many rows it moves
-  const int stride = gridDim.x * 16;
-  for (int r0 = blockIdx.x * 16 + (threadIdx.x >> 4); r0 < m; r0 += 4 * stride) {
-    int j[4];
+  int ok = 1;
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int r = r0 + u * stride;
-      j[u] = (r < m) ? idx[r] : -1;
+  for (int u = 0; u < kPer; ++u) {
+    const int rl = slot + u * (kGatherThreads / 16);
+    if (r_base + rl >= m) {
+      j[u] = -1;                                   // beyond the rows to rebuild: not part of the tile
+      continue;
     }
-    uint4 kv[4], vv[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (j[u] >= n || j[u] < -1) {   // -1 is the padding of topk_idx; anything else outside [0, len) is flagged
-        if (sub == 0) atomicOr(status, RKV_DEV_BAD_INDEX);
-        j[u] = -1;
-      }
-      if (j[u] >= 0) {
-        kv[u] = __ldcs(fk + (src0 + j[u]) * 16 + sub);
-        vv[u] = __ldcs(fv + (src0 + j[u]) * 16 + sub);
-      }
+    if (j[u] >= n || j[u] < -1) {                  // -1 is the padding of topk_idx; anything else outside [0, len) is flagged
+      if (sub == 0) atomicOr(status, RKV_DEV_BAD_INDEX);
+      j[u] = -1;
     }
+    if (j[u] < 0) {
+      ok = 0;                                      // a row of the tile stays as it is: no bulk store for this tile
+      continue;
+    }
+    const uint32_t dk = smem_u32(&tile_k[rl * 16 + sub]), dv = smem_u32(&tile_v[rl * 16 + sub]);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dk), "l"(fk + (src0 + j[u]) * 16 + sub) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dv), "l"(fv + (src0 + j[u]) * 16 + sub) : "memory");
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy below reads what the copies above wrote
+  const int all_ok = __syncthreads_and(ok);
+  uint4* sk = static_cast<uint4*>(small_cache.k) + (dst0 + r_base) * 16;
+  uint4* sv = static_cast<uint4*>(small_cache.v) + (dst0 + r_base) * 16;
+  if (all_ok) {
+    if (tid == 0) {
+      const int rows = m - r_base < kGatherRows ? m - r_base : kGatherRows;
+      const uint32_t bytes = (uint32_t)rows * 256u;
+      asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(sk), "r"(smem_u32(tile_k)), "r"(bytes)
+                   : "memory");
+      asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(sv), "r"(smem_u32(tile_v)), "r"(bytes)
+                   : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
+    return;
+  }
+  // a tile with skipped rows (bad or padding indices): row by row
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (j[u] >= 0) {
-        const int r = r0 + u * stride;
-        sk[(dst0 + r) * 16 + sub] = kv[u];
-        sv[(dst0 + r) * 16 + sub] = vv[u];
-      }
+  for (int u = 0; u < kPer; ++u) {
+    const int rl = slot + u * (kGatherThreads / 16);
+    if (j[u] >= 0) {
+      sk[rl * 16 + sub] = tile_k[rl * 16 + sub];
+      sv[rl * 16 + sub] = tile_v[rl * 16 + sub];
     }
   }
 }
@@ -303,11 +338,9 @@ cudaError_t launch_evict_order(const uint32_t* win_keys, int win_stride, const i
 cudaError_t launch_gather(const int32_t* topk_idx, const int32_t* k_small, int k_max, CacheDev full,
                           CacheDev small_cache, const int32_t* active, int n_seq, int n_kv_heads,
                           int32_t* status, cudaStream_t st) {
-  int gx = (k_max + 63) / 64;   // a thread moves up to four rows per round
-  if (gx > 64) gx = 64;
-  if (gx < 1) gx = 1;
-  dim3 grid(gx, n_kv_heads, n_seq);
-  return launch_ex(gather_kernel, grid, dim3(256), 0, st, 1, topk_idx, k_small, k_max, full, small_cache, active,
+  const int gx = (k_max + kGatherRows - 1) / kGatherRows;   // one CTA per tile of output rows
+  dim3 grid(gx < 1 ? 1 : gx, n_kv_heads, n_seq);
+  return launch_ex(gather_kernel, grid, dim3(kGatherThreads), 0, st, 1, topk_idx, k_small, k_max, full, small_cache, active,
                    n_kv_heads, status);
 }
 

@@ -23,10 +23,11 @@ EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", 
            "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
            "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step", "rkv_score_step",
            "rkv_gather_small_evict", "rkv_append_small_step_evict", "rkv_full_attention", "rkv_select_topk",
-           "rkv_append_full_attention"]
+           "rkv_append_full_attention", "rkv_get_option"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER, OPT_EARLY_CACHE_READ, OPT_INTERLEAVE_TILES = 1, 2, 3, 4, 5
 OPT_SELECT_KEYS_PER_CTA = 6
+OPT_SCORE_SLICE = 7
 KERNEL_NAMES = ["attn_full", "select", "attn_small", "gather", "append", "trigger", "fold", "score"]
 
 
@@ -80,6 +81,8 @@ def _load() -> ctypes.CDLL:
     lib.rkv_launch_count.restype = i64
     lib.rkv_set_option.argtypes = [vp, i32, i32]
     lib.rkv_set_option.restype = i32
+    lib.rkv_get_option.argtypes = [vp, i32, ctypes.POINTER(i32)]
+    lib.rkv_get_option.restype = i32
     lib.rkv_set_profiling.argtypes = [vp, i32]
     lib.rkv_set_profiling.restype = i32
     lib.rkv_get_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
@@ -240,6 +243,11 @@ class Context:
 
     def set_option(self, option: int, value: int):
         self._check(lib.rkv_set_option(self._h, option, value))
+
+    def get_option(self, option: int) -> int:
+        value = ctypes.c_int32(0)
+        self._check(lib.rkv_get_option(self._h, option, ctypes.byref(value)))
+        return value.value
 
     def set_profiling(self, on: bool):
         self._check(lib.rkv_set_profiling(self._h, 1 if on else 0))

@@ -180,7 +180,7 @@ class DeferredRefresh:
     latency-bound kernel chains are in flight at once.  Every layer needs a context of its own: its logits stay in
     the context's workspace until its selection runs."""
 
-    def __init__(self, layers, n_side=8):
+    def __init__(self, layers, n_side=16, select_keys_per_cta=16384, score_slice=4096):
         self.layers = layers
         ctxs = [id(st.ctx) for st in layers]
         if len(set(ctxs)) != len(ctxs):
@@ -188,21 +188,40 @@ class DeferredRefresh:
         self.sides = [torch.cuda.Stream() for _ in range(max(1, min(n_side, len(layers))))]
         self.ev_attn = torch.cuda.Event()
         self.ev_done = [torch.cuda.Event() for _ in self.sides]
+        # With many layers, many selections run side by side, and what counts is the SM time each takes, not the
+        # length of its own chain: few large CTAs per score pass and per top-K cluster (0: leave the contexts'
+        # settings alone, as is done for a handful of layers, whose selections are still latency-bound).
+        many = len(layers) >= 8
+        self.tuning = [(rkv.OPT_SELECT_KEYS_PER_CTA, select_keys_per_cta if many else 0),
+                       (rkv.OPT_SCORE_SLICE, score_slice if many else 0)]
+
+    def _tail(self, main, select_of):
+        """After the attention passes: every layer's selection and rebuild, dealt out to the side streams."""
+        self.ev_attn.record(main)
+        saved = {}
+        for st in self.layers:
+            saved[id(st.ctx)] = [(opt, st.ctx.get_option(opt)) for opt, val in self.tuning if val]
+            for opt, val in self.tuning:
+                if val:
+                    st.ctx.set_option(opt, val)
+        for i, side in enumerate(self.sides):
+            side.wait_event(self.ev_attn)
+            with torch.cuda.stream(side):
+                for l in range(i, len(self.layers), len(self.sides)):
+                    select_of(l, self.layers[l])
+                self.ev_done[i].record(side)
+        for ev in self.ev_done:
+            main.wait_event(ev)
+        for st in self.layers:
+            for opt, val in saved[id(st.ctx)]:
+                st.ctx.set_option(opt, val)
 
     def run(self, q_of, k_new_of, v_new_of, max_len_hint=0):
         """q_of(l), k_new_of(l), v_new_of(l): the layer's inputs.  Appends, attends; then selects and rebuilds."""
         main = torch.cuda.current_stream()
         for l, st in enumerate(self.layers):
             st.append_refresh_attention(q_of(l), k_new_of(l), v_new_of(l), max_len_hint=max_len_hint)
-        self.ev_attn.record(main)
-        for i, side in enumerate(self.sides):
-            side.wait_event(self.ev_attn)
-            with torch.cuda.stream(side):
-                for l in range(i, len(self.layers), len(self.sides)):
-                    self.layers[l].refresh_select(q_of(l))
-                self.ev_done[i].record(side)
-        for ev in self.ev_done:
-            main.wait_event(ev)
+        self._tail(main, lambda l, st: st.refresh_select(q_of(l)))
 
     def run_checked(self, q_of, k_new_of, v_new_of, threshold, small_hint=0, full_hint=0, after_trigger=None):
         """Token of the dynamic schedule at a check position: per layer the trigger, then both branches under its
@@ -216,15 +235,7 @@ class DeferredRefresh:
                 after_trigger(l, st)
             st.append_partial(q_of(l), k_new_of(l), v_new_of(l), active=st.not_flag, max_len_hint=small_hint)
             st.refresh_attention(q_of(l), active=st.flag, max_len_hint=full_hint)
-        self.ev_attn.record(main)
-        for i, side in enumerate(self.sides):
-            side.wait_event(self.ev_attn)
-            with torch.cuda.stream(side):
-                for l in range(i, len(self.layers), len(self.sides)):
-                    self.layers[l].refresh_select(q_of(l), active=self.layers[l].flag)
-                self.ev_done[i].record(side)
-        for ev in self.ev_done:
-            main.wait_event(ev)
+        self._tail(main, lambda l, st: st.refresh_select(q_of(l), active=st.flag))
 
 
 class LayerBatchedSmall:

@@ -612,6 +612,32 @@ def test_deterministic_bits(mods):
         assert torch.equal(a[2], st.scores) and torch.equal(a[3], st.small.k)
 
 
+def test_launch_shape_options_change_nothing(mods):
+    """RKV_OPT_SCORE_SLICE and RKV_OPT_SELECT_KEYS_PER_CTA only change how the score pass and the top-K are cut
+    into CTAs: scores, indices and the rebuilt small cache keep their bits, the output agrees with the oracle, and
+    rkv_get_option returns what was set."""
+    rkv, runner, synth = mods
+    lens, k_small = [20000, 7001], [2048, 300]
+    ctx, st, cache, q = make_layer(mods, lens, k_small, 16, 4, seed=23)
+    assert ctx.get_option(rkv.OPT_SCORE_SLICE) == 0 and ctx.get_option(rkv.OPT_SELECT_KEYS_PER_CTA) == 4096
+    st.refresh(q)
+    check_full_against_oracle(st, cache, q, lens, k_small, 4)
+    a = (st.out.clone(), st.topk_idx.clone(), st.scores.clone(), st.small.k.clone(), st.small.v.clone())
+    for slice_, per_cta in ((1024, 512), (2048, 16384), (4096, 40960), (8192, 4096), (0, 8192)):
+        ctx.set_option(rkv.OPT_SCORE_SLICE, slice_)
+        ctx.set_option(rkv.OPT_SELECT_KEYS_PER_CTA, per_cta)
+        assert ctx.get_option(rkv.OPT_SCORE_SLICE) == slice_ and ctx.get_option(rkv.OPT_SELECT_KEYS_PER_CTA) == per_cta
+        st.small.k.fill_(0.0); st.small.v.fill_(0.0)
+        st.refresh(q)
+        assert torch.equal(a[0], st.out) and torch.equal(a[1], st.topk_idx), (slice_, per_cta)
+        assert torch.equal(a[2], st.scores) and torch.equal(a[3], st.small.k) and torch.equal(a[4], st.small.v)
+    with pytest.raises(rkv.RkvError):
+        ctx.set_option(rkv.OPT_SCORE_SLICE, 3000)
+    with pytest.raises(rkv.RkvError):
+        ctx.get_option(99)
+    assert ctx.device_status() == 0
+
+
 def test_length_above_hint_is_clamped_and_flagged(mods):
     rkv, runner, synth = mods
     lens, k_small = [600], [16]
