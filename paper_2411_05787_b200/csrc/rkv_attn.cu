@@ -281,6 +281,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     n_early = p.early < n_spec ? p.early : n_spec;
     issue_spec(0, n_early);
   }
+  // The output accumulators are cleared up here (and pinned to registers), not on the path between the query's
+  // arrival and the first product, where every instruction of a warp is paid for in full.
+  float o[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    asm volatile("" : "+f"(o[i][0]), "+f"(o[i][1]), "+f"(o[i][2]), "+f"(o[i][3]));
+  }
   pdl_wait();
   pdl_launch();   // after the wait: at most one predecessor is ever in flight behind a kernel of this library
   if (kCluster) {
@@ -300,6 +308,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // sixteen 4-byte loads per lane (the memory pipe's request rate, not its latency, is what those cost).
   uint32_t* sm_q = reinterpret_cast<uint32_t*>(smem_gen + kStg * kStageBytes + 16 * kStg + 16 + kRecvFloats * 4);
   const bool q_lane = warp < kMW && tid < G * 16;
+  const bool q_row = warp < kMW && tid < kMaxGroup * 16;   // rows of heads beyond the group are stored as zeros
   uint4 qv = make_uint4(0u, 0u, 0u, 0u);
   if (q_lane) qv = __ldcg(reinterpret_cast<const uint4*>(qg) + tid);
   // fused append: this lane's 8 bytes of the new K and V rows, and the second cache's sizes
@@ -321,7 +330,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       vn = __ldcg(static_cast<const uint2*>(p.v_new) + nrow + lane);
     }
     // (the query's store to shared memory waits for its load; it comes after every other load has been issued)
-    if (q_lane) *reinterpret_cast<uint4*>(sm_q + (tid >> 4) * kQPad + (tid & 15) * 4) = qv;
+    if (q_row) *reinterpret_cast<uint4*>(sm_q + (tid >> 4) * kQPad + (tid & 15) * 4) = qv;
     // Where the new row goes in the attended cache: behind the last row (the cache grows), or - fixed-size small
     // cache that has reached its size - into the slot of the lowest-scoring survivor of the last refresh.
     int slot = n;
@@ -358,14 +367,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
       if (!evicting) n = n + 1;
     }
   }
-  if (!kAppend && q_lane) *reinterpret_cast<uint4*>(sm_q + (tid >> 4) * kQPad + (tid & 15) * 4) = qv;
+  if (!kAppend && q_row) *reinterpret_cast<uint4*>(sm_q + (tid >> 4) * kQPad + (tid & 15) * 4) = qv;
   uint32_t qb[8][2];              // B fragments of Q^T: [k = channel][n = head]
   if (warp < kMW) {
     consumer_bar();               // the query rows are in shared memory
+    // four 8x8 blocks [head][8 channels] per instruction: block m of load i is channels 32 i + 8 m .. + 7
+    const uint32_t q_at = smem_u32(sm_q) + (uint32_t)(lane & 7) * (kQPad * 4) + (uint32_t)(lane >> 3) * 16u;
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      qb[ks][0] = qd < G ? sm_q[qd * kQPad + 8 * ks + (lane & 3)] : 0u;
-      qb[ks][1] = qd < G ? sm_q[qd * kQPad + 8 * ks + 4 + (lane & 3)] : 0u;
+    for (int i = 0; i < 4; ++i) {
+      uint32_t r[4];
+      ldsm_x4(r, q_at + 64u * i);
+      qb[2 * i][0] = r[0];
+      qb[2 * i][1] = r[1];
+      qb[2 * i + 1][0] = r[2];
+      qb[2 * i + 1][1] = r[3];
     }
   }
   // Fused append: the lengths are bumped by the last ticket holder of the sequence.  A ticket is taken only
@@ -446,9 +461,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // ---------------------------------------------------------------- MMA warps
   const float ninf = -INFINITY;
   float m0 = ninf, m1 = ninf, l0 = 0.f, l1 = 0.f;
-  float o[8][4];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
 
   // logit scratch is position-major: [position][GP] floats, GP = 4 or 8; this lane holds heads qc, qc+1
   float* lg0 = nullptr;
@@ -601,10 +613,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // and writes its accumulators already scaled to it, so that the merge itself is a plain sum (few
   // instructions per thread: this phase is bound by instruction issue, not by memory).
   float* sm_wm = reinterpret_cast<float*>(sm_q + kMaxGroup * kQPad);   // [kMW][8]: per-warp maximum (own memory)
-  if (lane < 4) {
-    sm_wm[warp * 8 + qc] = m0;
-    sm_wm[warp * 8 + qc + 1] = m1;
-  }
+  if (lane < 4) *reinterpret_cast<float2*>(sm_wm + warp * 8 + qc) = make_float2(m0, m1);
   consumer_bar();   // (m) of every warp is visible, and the stage memory is free
   float* sm_o = reinterpret_cast<float*>(smem_gen);   // [kMW][8][kOPad] scaled accumulators
   float* sm_l = sm_o + kMW * 8 * kOPad;               // [kMW][8] scaled denominators
@@ -613,8 +622,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     float M0 = ninf, M1 = ninf;
 #pragma unroll
     for (int w = 0; w < kMW; ++w) {
-      M0 = fmaxf(M0, sm_wm[w * 8 + qc]);
-      M1 = fmaxf(M1, sm_wm[w * 8 + qc + 1]);
+      const float2 mw = *reinterpret_cast<const float2*>(sm_wm + w * 8 + qc);   // qc is even
+      M0 = fmaxf(M0, mw.x);
+      M1 = fmaxf(M1, mw.y);
     }
     const float e0 = (m0 == ninf) ? 0.f : ex2((m0 - M0) * kLog2e);
     const float e1 = (m1 == ninf) ? 0.f : ex2((m1 - M1) * kLog2e);
@@ -720,39 +730,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
     }
     take_len_ticket();
     if (!ok) return;
-    // This CTA finishes dchunk channels of every head: G * dchunk / 4 items of four channels, and C adjacent
-    // lanes per item, one per source CTA, that combine through shuffles (G * 32 lanes in all, as above).
+    // This CTA finishes dchunk channels of every head: G * dchunk / 4 items of four channels, one thread each, which
+    // reads the C sources' slices straight from the receive buffer (independent loads, no shuffles: with one or two
+    // warps per scheduler a chain of dependent shuffles costs more than the loads it saves; two lanes per item with
+    // one round of shuffles measured the same).
     const int ph_sh = 5 - c_sh;             // log2 of the items per head, dchunk / 4
+    if (tid < (n_items >> c_sh)) {
+      const int h = tid >> ph_sh, dd = (tid & ((1 << ph_sh) - 1)) * 4;
+      float2 ml[kAttnCluster];
+      float4 v[kAttnCluster];
+      float M = ninf;
 #pragma unroll
-    for (int it = 0; it < kIt; ++it) {
-      const int j = tid + it * kNT;
-      if (j >= n_items) continue;          // whole warps: n_items is a multiple of 32
-      const int item = j >> c_sh, r = j & (C - 1);
-      const int h = item >> ph_sh, dd = (item & ((1 << ph_sh) - 1)) * 4;
-      const float2 ml = *reinterpret_cast<const float2*>(recv_ml + (r * kMaxGroup + h) * 2);
-      float4 v = *reinterpret_cast<const float4*>(recv + (r * kMaxGroup + h) * dchunk + dd);
-      float M = ml.x;
-      for (int sh = 1; sh < C; sh <<= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
-      const float e = (ml.x == ninf) ? 0.f : ex2((ml.x - M) * kLog2e);
-      float L = ml.y * e;
-      v.x *= e;
-      v.y *= e;
-      v.z *= e;
-      v.w *= e;
-      for (int sh = 1; sh < C; sh <<= 1) {
-        L += __shfl_xor_sync(0xffffffffu, L, sh);
-        v.x += __shfl_xor_sync(0xffffffffu, v.x, sh);
-        v.y += __shfl_xor_sync(0xffffffffu, v.y, sh);
-        v.z += __shfl_xor_sync(0xffffffffu, v.z, sh);
-        v.w += __shfl_xor_sync(0xffffffffu, v.w, sh);
+      for (int r = 0; r < kAttnCluster; ++r) {
+        if (r < C) {
+          ml[r] = *reinterpret_cast<const float2*>(recv_ml + (r * kMaxGroup + h) * 2);
+          v[r] = *reinterpret_cast<const float4*>(recv + (r * kMaxGroup + h) * dchunk + dd);
+          M = fmaxf(M, ml[r].x);
+        }
       }
-      if (r == 0) {
-        const float inv = __fdividef(1.f, L);
-        uint2 o2;
-        o2.x = pack_bf16(v.x * inv, v.y * inv);
-        o2.y = pack_bf16(v.z * inv, v.w * inv);
-        *reinterpret_cast<uint2*>(out + h * kHeadDim + split * dchunk + dd) = o2;
+      float L = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int r = 0; r < kAttnCluster; ++r) {
+        if (r < C) {
+          const float e = (ml[r].x == ninf) ? 0.f : ex2((ml[r].x - M) * kLog2e);
+          L = fmaf(ml[r].y, e, L);
+          acc.x = fmaf(v[r].x, e, acc.x);
+          acc.y = fmaf(v[r].y, e, acc.y);
+          acc.z = fmaf(v[r].z, e, acc.z);
+          acc.w = fmaf(v[r].w, e, acc.w);
+        }
       }
+      const float inv = __fdividef(1.f, L);
+      uint2 o2;
+      o2.x = pack_bf16(acc.x * inv, acc.y * inv);
+      o2.y = pack_bf16(acc.z * inv, acc.w * inv);
+      *reinterpret_cast<uint2*>(out + h * kHeadDim + split * dchunk + dd) = o2;
     }
     return;
   }
