@@ -387,7 +387,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   // after the old lengths have been read by everyone it stands for - one per cluster, taken behind the cluster
   // barrier, or (streaming form, no barrier) one per CTA, taken when the CTA is done - so nobody can still see
   // them change.
-  bool ticket_due = kAppend && tid == 0 && (!kCluster || split == 0);
+  // (In a cluster the ticket goes to the last MMA thread, not to thread 0: the atomic's round trip would otherwise
+  // hold up warp 0, which finishes the CTA's share of the output right behind it.)
+  bool ticket_due = kAppend && tid == (kCluster ? 32 * kMW - 1 : 0) && (!kCluster || split == 0);
   auto take_len_ticket = [&] {
     if (ticket_due) {
       ticket_due = false;
