@@ -385,16 +385,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
   }
   // Fused append: the lengths are bumped by the last ticket holder of the sequence.  A ticket is taken only
   // after the old lengths have been read by everyone it stands for - one per cluster, taken behind the cluster
-  // barrier, or (streaming form, no barrier) one per CTA, taken when the CTA is done - so nobody can still see
-  // them change.
+  // barrier, or (streaming form, no barrier) one per CTA - so nobody can still see them change.
   // (In a cluster the ticket goes to the last MMA thread, not to thread 0: the atomic's round trip would otherwise
   // hold up warp 0, which finishes the CTA's share of the output right behind it.)
   bool ticket_due = kAppend && tid == (kCluster ? 32 * kMW - 1 : 0) && (!kCluster || split == 0);
+  // Streaming form: the CTA takes its ticket right here - it has read the old lengths above - and looks at the
+  // number it drew only when it is done, so that the atomic's round trip through L2 (about 900 cycles) is not spent
+  // at the end of every CTA, where it would hold the SM and, in the last CTA, the whole kernel.
+  int ticket_old = -1;
+  if (!kCluster && ticket_due) {
+    // (the increment is made to depend on the lengths just loaded, so that the atomic cannot be issued before
+    // those loads have returned: a ticket says "this CTA HAS read the old lengths")
+    int one;
+    asm volatile("{\n\t.reg .b32 t;\n\tand.b32 t, %1, 0;\n\tadd.s32 %0, t, 1;\n\t}" : "=r"(one) : "r"(n ^ new_len_f ^ new_len_s));
+    ticket_old = atomicAdd(p.len_tickets + b, one);
+  }
   auto take_len_ticket = [&] {
     if (ticket_due) {
       ticket_due = false;
       const int holders = kCluster ? p.n_kv_heads : p.n_kv_heads * (int)gridDim.x;
-      const int old = atomicAdd(p.len_tickets + b, 1);
+      const int old = kCluster ? atomicAdd(p.len_tickets + b, 1) : ticket_old;
       if (old == holders - 1) {
         if (new_len_s >= 0) p.small_len[b] = new_len_s;
         if (new_len_f >= 0) p.full_len[b] = new_len_f;
@@ -812,7 +822,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CU
         t[(int64_t)(kMaxGroup + d) * p.max_splits] = Ld;
       }
     }
-    take_len_ticket();     // streaming form with the append: at the very end, off the CTA's critical path
+    take_len_ticket();     // streaming form with the append: the ticket drawn at the start is looked at here
     if (kLogits) return;   // full step: the selection kernel (or the fold kernel) finishes out from the partials
     __threadfence();
     consumer_bar();
