@@ -63,24 +63,38 @@ __device__ __forceinline__ float batch_dot(const uint4 (&u)[kFly], const float* 
   return acc;
 }
 // Bring x into shared memory as fp32; with a norm weight, apply RMSNorm on the way (every block recomputes the
-// mean square of the few thousand inputs, which is cheaper than a separate launch).
+// mean square of the few thousand inputs, which is cheaper than a separate launch).  A thread requests four 16-byte
+// pieces of x (and of the norm weight) before it uses the first: a hidden-size input is one round trip to L2, the
+// FFN-size input of the down projection two - not one per piece.
+constexpr int kStagePieces = 4;
+__device__ __forceinline__ float4 bf16x4_to_float4(uint2 u) {
+  const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
+  const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
+  return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
 __device__ __forceinline__ void stage_x(const void* x, int x_is_bf16, const __nv_bfloat16* norm_w, float eps, float* xs,
                                         int n_in) {
   __shared__ float red[32];
+  const int n4 = n_in / 4;
+  float4* xs4 = reinterpret_cast<float4*>(xs);
+  const uint2* wn = reinterpret_cast<const uint2*>(norm_w);
+  uint2 nw[kStagePieces];          // norm weights of the first round (the only round for a hidden-size input)
   float ss = 0.f;
-  if (x_is_bf16) {
-    const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
-    for (int i = threadIdx.x; i < n_in; i += blockDim.x) {
-      const float v = __bfloat162float(xb[i]);
-      xs[i] = v;
-      ss = fmaf(v, v, ss);
+  for (int base = 0; base < n4; base += kStagePieces * kGemvThreads) {
+    float4 v[kStagePieces];
+#pragma unroll
+    for (int k = 0; k < kStagePieces; ++k) {
+      const int i = base + threadIdx.x + k * kGemvThreads;
+      v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < n4) v[k] = x_is_bf16 ? bf16x4_to_float4(__ldcg(static_cast<const uint2*>(x) + i))
+                                   : __ldcg(static_cast<const float4*>(x) + i);
+      if (norm_w != nullptr && base == 0) nw[k] = i < n4 ? __ldg(wn + i) : make_uint2(0u, 0u);
     }
-  } else {
-    const float* xf = static_cast<const float*>(x);
-    for (int i = threadIdx.x; i < n_in; i += blockDim.x) {
-      const float v = xf[i];
-      xs[i] = v;
-      ss = fmaf(v, v, ss);
+#pragma unroll
+    for (int k = 0; k < kStagePieces; ++k) {
+      const int i = base + threadIdx.x + k * kGemvThreads;
+      if (i < n4) xs4[i] = v[k];
+      ss += (v[k].x * v[k].x + v[k].y * v[k].y) + (v[k].z * v[k].z + v[k].w * v[k].w);
     }
   }
   if (norm_w != nullptr) {
@@ -88,9 +102,20 @@ __device__ __forceinline__ void stage_x(const void* x, int x_is_bf16, const __nv
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
-    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) tot += red[i];
+#pragma unroll
+    for (int i = 0; i < kGemvThreads / 32; ++i) tot += red[i];
     const float r = rsqrtf(tot / (float)n_in + eps);
-    for (int i = threadIdx.x; i < n_in; i += blockDim.x) xs[i] = xs[i] * r * __bfloat162float(norm_w[i]);
+    for (int base = 0; base < n4; base += kStagePieces * kGemvThreads) {
+#pragma unroll
+      for (int k = 0; k < kStagePieces; ++k) {
+        const int i = base + threadIdx.x + k * kGemvThreads;
+        if (i < n4) {          // the thread's own pieces: no barrier needed in between
+          const float4 wv = bf16x4_to_float4(base == 0 ? nw[k] : __ldg(wn + i));
+          const float4 t = xs4[i];
+          xs4[i] = make_float4(t.x * r * wv.x, t.y * r * wv.y, t.z * r * wv.z, t.w * r * wv.w);
+        }
+      }
+    }
   }
   __syncthreads();
 }
