@@ -1159,6 +1159,79 @@ def test_bench_configuration_graph_replay_shared_context(mods):
     assert all(int(st.full.len[0]) == L + T and int(st.small.len[0]) == K + 1 for st in layers)
 
 
+def test_bench_configuration_deferred_tail_eight_layers(mods):
+    """The schedule bench.py times by default (runner.DeferredRefresh), with the eight layers from which on it runs
+    its tail in the throughput shape (large score-pass slices, few large top-K CTAs, set around the calls and
+    restored): config-2 shape at a reduced context, one context per layer, tokens replayed from CUDA graphs.  Every
+    layer's output of every token against the oracle, the selected sets validated, the options back at their defaults."""
+    rkv, runner, synth = mods
+    dev = torch.device("cuda")
+    NL, S, T = 8, 10, 21
+    w = synth.scaled(synth.config2(n_layers=NL, ctx=6144), steps=T)
+    L, K, Hq, Hkv = w.lens[0], w.k_small[0], w.n_q_heads, w.n_kv_heads
+    full_hint, small_hint = L + T + 1, K + S + 2
+    ctxs = [rkv.Context(1, Hq, Hkv, full_hint, small_hint) for _ in range(NL)]
+    q_stage = torch.zeros((NL, 1, Hq, 128), dtype=torch.bfloat16, device=dev)
+    k_stage = torch.zeros((NL, 1, Hkv, 128), dtype=torch.bfloat16, device=dev)
+    v_stage = torch.zeros((NL, 1, Hkv, 128), dtype=torch.bfloat16, device=dev)
+    layers, states, inputs = [], [], []
+    for l in range(NL):
+        cache = synth.fill_layer(w, l, dev)
+        qs = synth.query_trajectory(w, l).to(dev)
+        kn, vn = synth.new_token_kv(w, l)
+        synth.plant_heavy(w, cache, l, qs[0])
+        layers.append(runner.LayerState(ctxs[l], cache, [K], S + 2, Hq, Hkv))
+        inputs.append((qs, kn.to(dev), vn.to(dev)))
+        states.append(O.SequenceState(host_heads(cache, 0, Hkv, "k").copy(), host_heads(cache, 0, Hkv, "v").copy(), L, K))
+
+    def stage(t):
+        for l in range(NL):
+            q_stage[l].copy_(inputs[l][0][t]); k_stage[l].copy_(inputs[l][1][t]); v_stage[l].copy_(inputs[l][2][t])
+
+    deferred = runner.DeferredRefresh(layers)
+    assert all(val for _, val in deferred.tuning)          # eight layers: the tail runs in its throughput shape
+
+    def token(kind):
+        if kind == "full":
+            return deferred.run(lambda l: q_stage[l], lambda l: k_stage[l], lambda l: v_stage[l], max_len_hint=full_hint)
+        for l, st in enumerate(layers):
+            st.append_partial(q_stage[l], k_stage[l], v_stage[l], max_len_hint=small_hint)
+
+    class W1:
+        n_kv_heads, k_small = Hkv, [K]
+    stage(0)
+    for l, st in enumerate(layers):
+        st.refresh(q_stage[l], max_len_hint=full_hint)
+        o_out, o_score, _ = states[l].full(bits(inputs[l][0][0, 0]))
+        check_out(st.out[0], o_out, f"init layer {l}")
+        follow_gpu_selection(st, states[l], 0, o_score, W1)
+    torch.cuda.synchronize()
+    graphs, side = {}, torch.cuda.Stream()
+    for kind in ("small", "full"):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(gr, stream=side):
+                token(kind)
+        graphs[kind] = gr
+    for c in ctxs:      # the tail's settings were put back after the calls were captured
+        assert c.get_option(rkv.OPT_SELECT_KEYS_PER_CTA) == 4096 and c.get_option(rkv.OPT_SCORE_SLICE) == 0
+    for t in range(1, T + 1):
+        stage(t)
+        kind = "full" if t % S == 0 else "small"
+        graphs[kind].replay()
+        torch.cuda.synchronize()
+        for l, st in enumerate(layers):
+            states[l].append(bits(inputs[l][1][t, 0]), bits(inputs[l][2][t, 0]))
+            if kind == "full":
+                o_out, o_score, _ = states[l].full(bits(inputs[l][0][t, 0]))
+                check_out(st.out[0], o_out, f"full token {t} layer {l}")
+                follow_gpu_selection(st, states[l], 0, o_score, W1)
+            else:
+                check_out(st.out[0], states[l].small(bits(inputs[l][0][t, 0])), f"partial token {t} layer {l}")
+    assert all(c.device_status() == 0 for c in ctxs)
+    assert all(int(st.full.len[0]) == L + T and int(st.small.len[0]) == K + 1 for st in layers)
+
+
 def test_bench_configuration_dynamic_schedule_graph_replay(mods):
     """The dynamic schedule as bench.py launches it (config-3 shape, reduced context): three layers that alternate
     between two contexts; plain tokens = one rkv_append_small_step per layer; every fifth token the trigger, both
