@@ -648,7 +648,6 @@ rkv_status rkv_append(rkv_ctx* ctx, const void* k_new, const void* v_new, const 
 rkv_status rkv_should_refresh(rkv_ctx* ctx, const void* q_now, const void* q_last_full, float threshold,
                               int32_t* flag, int32_t* keep, float* sim, void* stream) {
   if (!ctx || !q_now || !q_last_full || !flag) return RKV_ERR_INVALID_ARG;
-  if (!aligned16(q_now) || !aligned16(q_last_full)) return RKV_ERR_INVALID_ARG;   // read 16 bytes at a time
   cudaError_t e;
   {
     LaunchScope scope(ctx, static_cast<cudaStream_t>(stream), RKV_KERNEL_TRIGGER);

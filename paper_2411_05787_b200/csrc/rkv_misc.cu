@@ -150,55 +150,17 @@ __global__ void __launch_bounds__(128) append_kernel(const uint4* __restrict__ k
   }
 }
 
-// One block of 128 threads per sequence.  The query rows come as 16-byte pieces, four heads per thread and round,
-// all requested before the first is used (one round trip for up to 32 heads; a 2-byte load per head and channel in a
-// loop made one per few heads); then thread d owns channel d of the head-averaged queries.
+// one block of 128 threads per sequence: thread d owns channel d of the head-averaged queries
 __global__ void __launch_bounds__(128) trigger_kernel(const __nv_bfloat16* __restrict__ q_now,
                                                       const __nv_bfloat16* __restrict__ q_last, float threshold,
                                                       int32_t* flag, int32_t* keep, float* sim, int n_q_heads) {
   const int b = blockIdx.x, d = threadIdx.x;
-  const int piece = d & 15, hg = d >> 4;   // channels 8 piece .. 8 piece + 7 of heads hg, hg + 8, ..
-  __shared__ float part[2][8][kHeadDim];
   pdl_wait();
   pdl_launch();   // dependents are released only after this kernel's own wait (see launch_ex)
-  const uint4* qn = reinterpret_cast<const uint4*>(q_now) + (int64_t)b * n_q_heads * 16 + piece;
-  const uint4* ql = reinterpret_cast<const uint4*>(q_last) + (int64_t)b * n_q_heads * 16 + piece;
-  float sa[8], sc[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) sa[j] = sc[j] = 0.f;
-  for (int h0 = hg; h0 < n_q_heads; h0 += 32) {
-    uint4 u[4], v[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int h = h0 + 8 * k;
-      u[k] = h < n_q_heads ? __ldcg(qn + h * 16) : make_uint4(0u, 0u, 0u, 0u);
-      v[k] = h < n_q_heads ? __ldcg(ql + h * 16) : make_uint4(0u, 0u, 0u, 0u);
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const __nv_bfloat162* pu = reinterpret_cast<const __nv_bfloat162*>(&u[k]);
-      const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&v[k]);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 fu = __bfloat1622float2(pu[j]), fv = __bfloat1622float2(pv[j]);
-        sa[2 * j] += fu.x;
-        sa[2 * j + 1] += fu.y;
-        sc[2 * j] += fv.x;
-        sc[2 * j + 1] += fv.y;
-      }
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    part[0][hg][8 * piece + j] = sa[j];
-    part[1][hg][8 * piece + j] = sc[j];
-  }
-  __syncthreads();
   float a = 0.f, c = 0.f;
-#pragma unroll
-  for (int g8 = 0; g8 < 8; ++g8) {
-    a += part[0][g8][d];
-    c += part[1][g8][d];
+  for (int h = 0; h < n_q_heads; ++h) {
+    a += __bfloat162float(q_now[((int64_t)b * n_q_heads + h) * kHeadDim + d]);
+    c += __bfloat162float(q_last[((int64_t)b * n_q_heads + h) * kHeadDim + d]);
   }
   const float inv = 1.f / (float)n_q_heads;
   a *= inv;
