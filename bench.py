@@ -76,6 +76,8 @@ def parse_args():
                     help="deferred schedule with 8+ layers: RKV_OPT_SELECT_KEYS_PER_CTA of the tail's selections (0: the contexts')")
     ap.add_argument("--deferred-score-slice", type=int, default=4096,
                     help="deferred schedule with 8+ layers: RKV_OPT_SCORE_SLICE of the tail's score passes (0: the contexts')")
+    ap.add_argument("--early-scores", action="store_true",
+                    help="deferred schedule: every layer's score pass right behind its attention pass, in a stream of its own")
     ap.add_argument("--side-streams", type=int, default=16,
                     help="deferred schedule: streams the layers' selections and rebuilds are spread over")
     ap.add_argument("--regions", type=int, default=0,
@@ -399,7 +401,8 @@ def measure_workload(args, w, dev, world, steps, warmup, level):
 
     overlapped = runner.OverlappedRefresh(layers) if schedule == "overlap" else None
     deferred = (runner.DeferredRefresh(layers, n_side=args.side_streams, select_keys_per_cta=args.deferred_keys_per_cta,
-                                       score_slice=args.deferred_score_slice) if schedule == "deferred" else None)
+                                       score_slice=args.deferred_score_slice, early_scores=args.early_scores)
+                if schedule == "deferred" else None)
     qf, kf, vf = (lambda l: q_stage[l]), (lambda l: k_stage[l]), (lambda l: v_stage[l])
 
     def token(kind: str):

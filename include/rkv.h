@@ -165,6 +165,16 @@ rkv_status rkv_append_full_attention(rkv_ctx* ctx, const void* q, const void* k_
 rkv_status rkv_select_topk(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/,
                            const int32_t* k_small, int32_t k_max, const int32_t* active, float* scores,
                            int64_t score_stride, int32_t* topk_idx, void* q_last_full, void* stream);
+/* The second half cut once more, for callers that want its first launch early: rkv_score_keys runs the score pass
+ * alone - the logits the attention pass left in the workspace become aggregated scores (written to scores[] when it
+ * is not NULL), their order-preserving keys and the per-(sequence, KV head) histogram, and q goes to q_last_full when
+ * that is not NULL - and the NEXT rkv_select_topk on the context (same cache, mask and k_max; scores and q_last_full
+ * NULL, they have been written) launches the selection alone.  Right behind the attention pass the logits are
+ * still in L2; the top-K and the rebuild can then follow whenever the caller likes (Sec. 2.2: the refreshed C_p is
+ * first needed by the next token).  Same indices and scores as rkv_full_step. */
+rkv_status rkv_score_keys(rkv_ctx* ctx, const void* q, const rkv_cache* full /*host struct*/, const int32_t* k_small,
+                          int32_t k_max, const int32_t* active, float* scores, int64_t score_stride,
+                          void* q_last_full, void* stream);
 
 /*
  * Score-only refresh step (Sec. 4.2 "Impact of full attention steps", the "w/o full attention" setting:

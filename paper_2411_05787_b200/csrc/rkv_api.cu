@@ -359,6 +359,8 @@ rkv_status rkv_create(const rkv_config* cfg, rkv_ctx** out) {
   ctx->hist = reinterpret_cast<uint32_t*>(ctx->workspace + w.hist);   // zeroed with the rest of the workspace above
   ctx->anchor = reinterpret_cast<int32_t*>(ctx->workspace + w.anchor);
   ctx->hist_dirty = false;
+  ctx->pending_keys.valid = false;
+  ctx->pending_full.valid = false;
   ctx->logits = reinterpret_cast<float*>(ctx->workspace + w.logits);
   ctx->status = reinterpret_cast<int32_t*>(ctx->workspace + w.status);
   ctx->logit_stride = w.logit_stride;
@@ -386,6 +388,7 @@ static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cac
   if (n_max < 1 || n_max > ctx->cfg.max_len) return RKV_ERR_INVALID_ARG;
   int chunk = 0, gx = 1;
   ctx->pending_full.valid = false;
+  ctx->pending_keys.valid = false;   // the logits those keys came from are about to be overwritten
   rkv_status s = run_attention(ctx, q, full, active, out, n_max, n_max, true, st, &chunk, &gx, app, score_only);
   if (s != RKV_OK) return s;
   if (fold_out && !score_only) {
@@ -404,20 +407,33 @@ static rkv_status full_attention_part(rkv_ctx* ctx, const void* q, const rkv_cac
 }
 
 // Second half: scores and top-K from what the first half left in the workspace; folds out unless it is NULL.
+// stage: both launches (the score pass, then the selection), or one of them - rkv_score_keys launches the score pass
+// alone and leaves a record for the rkv_select_topk that launches the selection alone.
+enum SelectStage { kStageBoth, kStageScore, kStageSelect };
 static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small,
                               int32_t k_max, const int32_t* active, void* out, float* scores, int64_t score_stride,
-                              int32_t* topk_idx, void* q_last_full, cudaStream_t st) {
-  if (!ctx || !cache_ok(full) || !k_small || !topk_idx || (q_last_full != nullptr && q == nullptr))
+                              int32_t* topk_idx, void* q_last_full, cudaStream_t st, SelectStage stage = kStageBoth) {
+  if (!ctx || !cache_ok(full) || !k_small || (!topk_idx && stage != kStageScore) ||
+      (q_last_full != nullptr && q == nullptr))
     return RKV_ERR_INVALID_ARG;
   if (k_max < 1 || k_max > ctx->cfg.max_small) return RKV_ERR_INVALID_ARG;
-  if (!ctx->pending_full.valid) return RKV_ERR_INVALID_ARG;   // no attention pass to take the logits from
-  const int n_max = ctx->pending_full.n_max, chunk = ctx->pending_full.chunk, gx = ctx->pending_full.gx;
-  if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
-  ctx->pending_full.valid = false;
+  int n_max, chunk, gx;
+  if (stage == kStageSelect) {
+    if (!ctx->pending_keys.valid || ctx->pending_keys.k_max != k_max) return RKV_ERR_INVALID_ARG;
+    n_max = ctx->pending_keys.n_max;
+    chunk = gx = 0;                 // (geometry of the attention pass: the score pass has used it)
+    ctx->pending_keys.valid = false;
+  } else {
+    if (!ctx->pending_full.valid) return RKV_ERR_INVALID_ARG;   // no attention pass to take the logits from
+    n_max = ctx->pending_full.n_max, chunk = ctx->pending_full.chunk, gx = ctx->pending_full.gx;
+    if (scores != nullptr && score_stride < n_max) return RKV_ERR_INVALID_ARG;
+    ctx->pending_full.valid = false;
+    ctx->pending_keys.valid = false;
+  }
   // two launches: the score pass over all positions (keys, scores, histogram; folds out[] when asked to), then
   // the selection proper, one small cluster per (sequence, KV head)
   const int bg = ctx->cfg.n_seq * ctx->cfg.n_kv_heads;
-  if (ctx->hist_dirty) {   // an earlier call launched its score pass but not its selection, which clears the histogram
+  if (ctx->hist_dirty && stage != kStageSelect) {   // an earlier score pass was never followed by its selection, which clears the histogram
     cudaError_t e0 = cudaMemsetAsync(ctx->hist, 0, (size_t)bg * rkv::kSelectBins * sizeof(uint32_t), st);
     if (e0 != cudaSuccess) return cuda_fail(ctx, e0, "histogram reset");
     ctx->hist_dirty = false;
@@ -473,13 +489,20 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   sp.keys_per_thread = rkv::select_keys_per_thread(n_max, cluster);
   sp.per_fixed = ctx->cfg.n_seq == 1 ? 1 : 0;
   cudaError_t e;
-  ctx->hist_dirty = true;
-  {
-    LaunchScope scope(ctx, st, RKV_KERNEL_SCORE);
-    e = rkv::launch_score(cp, ctx->cfg.n_seq, st);
+  if (stage != kStageSelect) {
+    ctx->hist_dirty = true;
+    {
+      LaunchScope scope(ctx, st, RKV_KERNEL_SCORE);
+      e = rkv::launch_score(cp, ctx->cfg.n_seq, st);
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "score launch");
+    ctx->launches += 1;
+    if (stage == kStageScore) {
+      ctx->pending_keys = {true, n_max, k_max, full->k, active};
+      rkv::note_launch(st, nullptr, nullptr);
+      return RKV_OK;
+    }
   }
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "score launch");
-  ctx->launches += 1;
   {
     LaunchScope scope(ctx, st, RKV_KERNEL_SELECT);
     e = rkv::launch_select(sp, ctx->cfg.n_seq, cluster, st);
@@ -538,11 +561,28 @@ rkv_status rkv_append_full_attention(rkv_ctx* ctx, const void* q, const void* k_
 rkv_status rkv_select_topk(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
                            const int32_t* active, float* scores, int64_t score_stride, int32_t* topk_idx,
                            void* q_last_full, void* stream) {
+  if (ctx != nullptr && ctx->pending_keys.valid) {   // rkv_score_keys has run: the selection alone is left
+    if (full == nullptr || ctx->pending_keys.full_k != full->k || ctx->pending_keys.active != active ||
+        scores != nullptr || q_last_full != nullptr)
+      return RKV_ERR_INVALID_ARG;   // (scores and q_last_full are outputs of the score pass)
+    return select_part(ctx, q, full, k_small, k_max, active, nullptr, nullptr, 0, topk_idx, nullptr,
+                       static_cast<cudaStream_t>(stream), kStageSelect);
+  }
   if (ctx != nullptr && ctx->pending_full.valid && full != nullptr &&
       (ctx->pending_full.full_k != full->k || ctx->pending_full.active != active))
     return RKV_ERR_INVALID_ARG;   // not the cache / mask of the attention pass it completes
   return select_part(ctx, q, full, k_small, k_max, active, nullptr, scores, score_stride, topk_idx, q_last_full,
                      static_cast<cudaStream_t>(stream));
+}
+
+rkv_status rkv_score_keys(rkv_ctx* ctx, const void* q, const rkv_cache* full, const int32_t* k_small, int32_t k_max,
+                          const int32_t* active, float* scores, int64_t score_stride, void* q_last_full,
+                          void* stream) {
+  if (ctx != nullptr && ctx->pending_full.valid && full != nullptr &&
+      (ctx->pending_full.full_k != full->k || ctx->pending_full.active != active))
+    return RKV_ERR_INVALID_ARG;   // not the cache / mask of the attention pass it completes
+  return select_part(ctx, q, full, k_small, k_max, active, nullptr, scores, score_stride, nullptr, q_last_full,
+                     static_cast<cudaStream_t>(stream), kStageScore);
 }
 
 rkv_status rkv_gather_small(rkv_ctx* ctx, const int32_t* topk_idx, const int32_t* k_small, int32_t k_max,

@@ -250,6 +250,8 @@ struct rkv_ctx {
   int score_slice;           // positions per CTA of the score pass; 0: chosen per launch
   // geometry of the last rkv_full_attention, for the rkv_select_topk that completes it
   struct { bool valid; int chunk, gx, n_max; const void* full_k; const int32_t* active; } pending_full;
+  // ... and of the last rkv_score_keys, for the rkv_select_topk that launches the selection alone
+  struct { bool valid; int n_max, k_max; const void* full_k; const int32_t* active; } pending_keys;
   int gp;              // floats per position in the logit scratch
   std::string last_error;
   std::map<std::pair<uint64_t, int64_t>, CUtensorMap> tmaps;   // (base address, rows) -> tensor map

@@ -23,7 +23,7 @@ EXPORTS = ["rkv_create", "rkv_destroy", "rkv_workspace_bytes", "rkv_full_step", 
            "rkv_status_string", "rkv_last_cuda_error", "rkv_launch_count", "rkv_set_profiling", "rkv_get_profile",
            "rkv_set_option", "rkv_small_step_noalloc", "rkv_append_small_step", "rkv_score_step",
            "rkv_gather_small_evict", "rkv_append_small_step_evict", "rkv_full_attention", "rkv_select_topk",
-           "rkv_append_full_attention", "rkv_get_option"]
+           "rkv_append_full_attention", "rkv_get_option", "rkv_score_keys"]
 NOALLOC_MAX_PROBLEMS, NOALLOC_MAX_LEN = 32, 65536
 OPT_SMALL_MIN_CHUNK, OPT_DEPENDENT_LAUNCH, OPT_SMALL_CLUSTER, OPT_EARLY_CACHE_READ, OPT_INTERLEAVE_TILES = 1, 2, 3, 4, 5
 OPT_SELECT_KEYS_PER_CTA = 6
@@ -66,6 +66,8 @@ def _load() -> ctypes.CDLL:
     lib.rkv_append_full_attention.restype = i32
     lib.rkv_select_topk.argtypes = [vp, vp, cachep, vp, i32, vp, vp, i64, vp, vp, vp]
     lib.rkv_select_topk.restype = i32
+    lib.rkv_score_keys.argtypes = [vp, vp, cachep, vp, i32, vp, vp, i64, vp, vp]
+    lib.rkv_score_keys.restype = i32
     lib.rkv_gather_small.argtypes = [vp, vp, vp, i32, cachep, cachep, vp, vp]
     lib.rkv_small_step.argtypes = [vp, vp, cachep, vp, vp, i32, vp]
     lib.rkv_append.argtypes = [vp, vp, vp, cachep, cachep, vp]
@@ -203,6 +205,12 @@ class Context:
         stride = scores.shape[-1] if scores is not None else 0
         self._check(lib.rkv_select_topk(self._h, _ptr(q), ctypes.byref(full), _ptr(k_small), k_max, _ptr(active),
                                         _ptr(scores), stride, _ptr(topk_idx), _ptr(q_last_full), _stream(stream)))
+
+    def score_keys(self, q, full: RkvCache, k_small, k_max, active=None, scores=None, q_last_full=None, stream=None):
+        """The score pass alone; the next select_topk (scores=None, q_last_full=None) launches the selection alone."""
+        stride = scores.shape[-1] if scores is not None else 0
+        self._check(lib.rkv_score_keys(self._h, _ptr(q), ctypes.byref(full), _ptr(k_small), k_max, _ptr(active),
+                                       _ptr(scores), stride, _ptr(q_last_full), _stream(stream)))
 
     def gather_small(self, topk_idx, k_small, k_max, full: RkvCache, small: RkvCache, active=None, stream=None):
         self._check(lib.rkv_gather_small(self._h, _ptr(topk_idx), _ptr(k_small), k_max, ctypes.byref(full),

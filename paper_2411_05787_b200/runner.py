@@ -81,6 +81,17 @@ class LayerState:
         self.ctx.gather_small(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c, active=active,
                               stream=stream)
 
+    def refresh_score_keys(self, q, active=None, stream=None):
+        """Second half, first launch: scores, keys and histogram (and q_last_full) from the logits of refresh_attention."""
+        self.ctx.score_keys(q, self.full_c, self.k_small, self.k_max, active=active, scores=self.scores,
+                            q_last_full=self.q_last_full, stream=stream)
+
+    def refresh_select_only(self, active=None, stream=None):
+        """Second half, second launch after refresh_score_keys: top-K, then the rebuild of the small cache."""
+        self.ctx.select_topk(None, self.full_c, self.k_small, self.k_max, self.topk_idx, active=active, stream=stream)
+        self.ctx.gather_small(self.topk_idx, self.k_small, self.k_max, self.full_c, self.small_c, active=active,
+                              stream=stream)
+
     def refresh_scores_only(self, q, active=None, max_len_hint=0, small_hint=0):
         """Score-only refresh: scores and top-K from K alone, rebuild of the small cache, attention over the new one."""
         self.ctx.score_step(q, self.full_c, self.k_small, self.k_max, self.topk_idx, active=active, scores=self.scores,
@@ -180,8 +191,14 @@ class DeferredRefresh:
     latency-bound kernel chains are in flight at once.  Every layer needs a context of its own: its logits stay in
     the context's workspace until its selection runs."""
 
-    def __init__(self, layers, n_side=16, select_keys_per_cta=16384, score_slice=4096):
+    def __init__(self, layers, n_side=16, select_keys_per_cta=16384, score_slice=4096, early_scores=False):
         self.layers = layers
+        # early_scores: every layer's score pass runs right behind its attention pass, in a stream of its own beside
+        # the next layer's attention (its logits are then still in L2); only top-K and rebuild wait for the tail
+        self.early_scores = early_scores
+        self.score_stream = torch.cuda.Stream() if early_scores else None
+        self.ev_layer = [torch.cuda.Event() for _ in layers] if early_scores else None
+        self.ev_scores = torch.cuda.Event() if early_scores else None
         ctxs = [id(st.ctx) for st in layers]
         if len(set(ctxs)) != len(ctxs):
             raise ValueError("every layer needs its own context (the workspace holds its logits until the token's end)")
@@ -195,33 +212,51 @@ class DeferredRefresh:
         self.tuning = [(rkv.OPT_SELECT_KEYS_PER_CTA, select_keys_per_cta if many else 0),
                        (rkv.OPT_SCORE_SLICE, score_slice if many else 0)]
 
-    def _tail(self, main, select_of):
-        """After the attention passes: every layer's selection and rebuild, dealt out to the side streams."""
-        self.ev_attn.record(main)
+    def _set_tuning(self):
         saved = {}
         for st in self.layers:
             saved[id(st.ctx)] = [(opt, st.ctx.get_option(opt)) for opt, val in self.tuning if val]
             for opt, val in self.tuning:
                 if val:
                     st.ctx.set_option(opt, val)
+        return saved
+
+    def _restore_tuning(self, saved):
+        for st in self.layers:
+            for opt, val in saved[id(st.ctx)]:
+                st.ctx.set_option(opt, val)
+
+    def _tail(self, main, select_of, wait_for=()):
+        """After the attention passes: every layer's selection and rebuild, dealt out to the side streams."""
+        self.ev_attn.record(main)
         for i, side in enumerate(self.sides):
             side.wait_event(self.ev_attn)
+            for ev in wait_for:
+                side.wait_event(ev)
             with torch.cuda.stream(side):
                 for l in range(i, len(self.layers), len(self.sides)):
                     select_of(l, self.layers[l])
                 self.ev_done[i].record(side)
         for ev in self.ev_done:
             main.wait_event(ev)
-        for st in self.layers:
-            for opt, val in saved[id(st.ctx)]:
-                st.ctx.set_option(opt, val)
 
     def run(self, q_of, k_new_of, v_new_of, max_len_hint=0):
         """q_of(l), k_new_of(l), v_new_of(l): the layer's inputs.  Appends, attends; then selects and rebuilds."""
         main = torch.cuda.current_stream()
-        for l, st in enumerate(self.layers):
-            st.append_refresh_attention(q_of(l), k_new_of(l), v_new_of(l), max_len_hint=max_len_hint)
-        self._tail(main, lambda l, st: st.refresh_select(q_of(l)))
+        saved = self._set_tuning()
+        if not self.early_scores:
+            for l, st in enumerate(self.layers):
+                st.append_refresh_attention(q_of(l), k_new_of(l), v_new_of(l), max_len_hint=max_len_hint)
+            self._tail(main, lambda l, st: st.refresh_select(q_of(l)))
+        else:
+            for l, st in enumerate(self.layers):
+                st.append_refresh_attention(q_of(l), k_new_of(l), v_new_of(l), max_len_hint=max_len_hint)
+                self.ev_layer[l].record(main)
+                self.score_stream.wait_event(self.ev_layer[l])
+                st.refresh_score_keys(q_of(l), stream=self.score_stream)
+            self.ev_scores.record(self.score_stream)
+            self._tail(main, lambda l, st: st.refresh_select_only(), wait_for=(self.ev_scores,))
+        self._restore_tuning(saved)
 
     def run_checked(self, q_of, k_new_of, v_new_of, threshold, small_hint=0, full_hint=0, after_trigger=None):
         """Token of the dynamic schedule at a check position: per layer the trigger, then both branches under its
@@ -235,7 +270,9 @@ class DeferredRefresh:
                 after_trigger(l, st)
             st.append_partial(q_of(l), k_new_of(l), v_new_of(l), active=st.not_flag, max_len_hint=small_hint)
             st.refresh_attention(q_of(l), active=st.flag, max_len_hint=full_hint)
+        saved = self._set_tuning()
         self._tail(main, lambda l, st: st.refresh_select(q_of(l), active=st.flag))
+        self._restore_tuning(saved)
 
 
 class LayerBatchedSmall:

@@ -212,6 +212,37 @@ def test_select_topk_needs_its_attention_pass(mods):
     assert ctx.device_status() == 0
 
 
+@pytest.mark.parametrize("lens,k_small,n_q,n_kv", [([5000, 3000], [256, 100], 32, 8), ([20000], [2048], 28, 4)])
+def test_full_step_in_three_launches_matches_oracle(mods, lens, k_small, n_q, n_kv):
+    """rkv_full_attention, rkv_score_keys, then rkv_select_topk for the selection alone (+ gather): same indices,
+    scores and q_last_full as the one call, everything against the oracle; and the order of the calls is enforced."""
+    rkv, runner, synth = mods
+    ctx, st, cache, q = make_layer(mods, lens, k_small, n_q, n_kv, seed=41)
+    with pytest.raises(rkv.RkvError):
+        st.refresh_score_keys(q)                      # no attention pass to take the logits from
+    st.refresh(q)
+    one = (st.topk_idx.clone(), st.scores.clone(), st.small.k.clone(), st.q_last_full.clone())
+    st.topk_idx.fill_(-7); st.scores.fill_(0.0); st.small.k.fill_(0.0); st.q_last_full.fill_(0.0)
+    st.refresh_attention(q)
+    st.refresh_score_keys(q)
+    assert torch.equal(one[1], st.scores) and torch.equal(one[3], st.q_last_full)
+    with pytest.raises(rkv.RkvError):                 # scores and q_last_full belong to the score pass
+        ctx.select_topk(q, st.full_c, st.k_small, st.k_max, st.topk_idx, scores=st.scores)
+    with pytest.raises(rkv.RkvError):                 # another k_max than the score pass was given
+        ctx.select_topk(None, st.full_c, st.k_small, st.k_max - 1, st.topk_idx)
+    st.refresh_select_only()
+    assert torch.equal(one[0], st.topk_idx) and torch.equal(one[2], st.small.k)
+    with pytest.raises(rkv.RkvError):
+        st.refresh_select_only()                      # used up
+    check_full_against_oracle(st, cache, q, lens, k_small, n_kv)
+    # a score pass whose selection never ran leaves its histogram behind: the next full step must not see it
+    st.refresh_attention(q)
+    st.refresh_score_keys(q)
+    st.refresh(q)
+    assert torch.equal(one[0], st.topk_idx) and torch.equal(one[1], st.scores)
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("agg,name", [(1, "mean"), (2, "first")])
 def test_aggregation_modes(mods, agg, name):
     lens, k_small = [500, 129], [50, 20]
@@ -1159,8 +1190,10 @@ def test_bench_configuration_graph_replay_shared_context(mods):
     assert all(int(st.full.len[0]) == L + T and int(st.small.len[0]) == K + 1 for st in layers)
 
 
-def test_bench_configuration_deferred_tail_eight_layers(mods):
-    """The schedule bench.py times by default (runner.DeferredRefresh), with the eight layers from which on it runs
+@pytest.mark.parametrize("early_scores", [False, True])
+def test_bench_configuration_deferred_tail_eight_layers(mods, early_scores):
+    """(early_scores: every layer's score pass right behind its attention pass in a stream of its own, rkv_score_keys.)
+    The schedule bench.py times by default (runner.DeferredRefresh), with the eight layers from which on it runs
     its tail in the throughput shape (large score-pass slices, few large top-K CTAs, set around the calls and
     restored): config-2 shape at a reduced context, one context per layer, tokens replayed from CUDA graphs.  Every
     layer's output of every token against the oracle, the selected sets validated, the options back at their defaults."""
@@ -1188,7 +1221,7 @@ def test_bench_configuration_deferred_tail_eight_layers(mods):
         for l in range(NL):
             q_stage[l].copy_(inputs[l][0][t]); k_stage[l].copy_(inputs[l][1][t]); v_stage[l].copy_(inputs[l][2][t])
 
-    deferred = runner.DeferredRefresh(layers)
+    deferred = runner.DeferredRefresh(layers, early_scores=early_scores)
     assert all(val for _, val in deferred.tuning)          # eight layers: the tail runs in its throughput shape
 
     def token(kind):
