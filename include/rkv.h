@@ -359,11 +359,12 @@ int64_t rkv_launch_count(const rkv_ctx* ctx);
  *                             The cluster has 1, 2, 4 or 8 CTAs per (sequence, KV head): fewer keys per CTA give
  *                             the shortest chain for a single selection, more keys per CTA occupy fewer SMs
  *                             when many selections run side by side.  The selected set does not depend on it.
- *   RKV_OPT_SCORE_SLICE       positions one CTA of the score pass takes: 0 (default) = chosen per launch (the
- *                             smallest of 1024, 2048, 4096, 8192 that keeps the grid near four CTAs per SM), or
- *                             one of those four values.  Longer slices mean fewer CTAs that each pay the
- *                             log-sum-exp and the histogram flush once: slower for a single selection, cheaper
- *                             when many run side by side.  Keys, scores and the selected set do not depend on it.
+ *   RKV_OPT_SCORE_SLICE       fewest positions one CTA of the score pass takes: 0 (default) = chosen per launch
+ *                             alone (the smallest of 1024, 2048, 4096, 8192 that keeps the grid near four CTAs per
+ *                             SM); 1024, 2048, 4096 or 8192 = that choice, but no less than this.  Longer slices mean
+ *                             fewer CTAs that each pay the log-sum-exp and the histogram flush once: slower for a
+ *                             single selection, cheaper when many run side by side.  Keys, scores and the selected
+ *                             set do not depend on it.
  */
 #define RKV_OPT_SMALL_MIN_CHUNK 1
 #define RKV_OPT_DEPENDENT_LAUNCH 2

@@ -463,7 +463,8 @@ static rkv_status select_part(rkv_ctx* ctx, const void* q, const rkv_cache* full
   cp.agg = ctx->cfg.agg;
   cp.k_max = k_max;
   cp.max_len = n_max;
-  cp.slice = ctx->score_slice != 0 ? ctx->score_slice : rkv::score_slice_for(n_max, bg, ctx->sm_count);
+  cp.slice = rkv::score_slice_for(n_max, bg, ctx->sm_count);
+  if (cp.slice < ctx->score_slice) cp.slice = ctx->score_slice;   // the option is a floor
   cp.n_slices = (n_max + cp.slice - 1) / cp.slice;
   cp.chunk = chunk;
   cp.max_splits = ctx->max_splits;
