@@ -510,18 +510,33 @@ def measure_workload(args, w, dev, world, steps, warmup, level):
             return "small"
         return "check" if dynamic else "full"
 
+    readback = torch.cuda.Stream()
+    ev_token, ev_read = torch.cuda.Event(), torch.cuda.Event()
+
     def run_tokens(n, e2e=False, always_full=False, force_small=False, force_kind=None):
-        """Enqueue n decode tokens; returns the count of each kind."""
+        """Enqueue n decode tokens; returns the count of each kind.  e2e: every token's inputs come from pinned host
+        memory and its outputs go back to the host.  The read-back runs in a stream of its own: the NEXT token's
+        inputs are copied in while it is under way (the two directions have their own copy engines), but the next
+        token's kernels start only when the read-back is complete (they overwrite what it reads)."""
         cnt = {k: 0 for k in graphs}
+        main = torch.cuda.current_stream()
         for _ in range(n):
             t = tok_counter[0]; tok_counter[0] += 1
             src = inputs_host if e2e else inputs_dev
             stage.copy_(src[t % n_in], non_blocking=True)
             kind = kind_of(t, always_full, force_small, force_kind)
+            if e2e:
+                main.wait_event(ev_read)          # (the first wait finds the event unrecorded and passes)
             graphs[kind].replay()
             if e2e:
-                outs_host.copy_(outs, non_blocking=True)
+                ev_token.record(main)
+                readback.wait_event(ev_token)
+                with torch.cuda.stream(readback):
+                    outs_host.copy_(outs, non_blocking=True)
+                    ev_read.record(readback)
             cnt[kind] += 1
+        if e2e:
+            main.wait_event(ev_read)              # the region ends when the last token has been read back
         return cnt
 
     def timed(n, fresh=True, **kw):
