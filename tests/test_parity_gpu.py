@@ -632,6 +632,43 @@ def test_gather_flags_indices_outside_the_cache(mods):
     assert ctx.device_status() == 0
 
 
+def test_gather_tiles_with_and_without_skipped_rows(mods):
+    """rkv_gather_small moves 64 output rows per CTA: whole tiles leave with one bulk store per cache, a tile with
+    a skipped row (padding or a flagged index) row by row, the last tile is ragged, rows at and beyond
+    min(k_small, len) stay untouched, inactive sequences too; both sequences and both heads bit for bit."""
+    rkv, runner, synth = mods
+    lens, k_small = [5000, 700], [200, 150]
+    ctx, st, cache, q = make_layer(mods, lens, k_small, 4, 2, seed=33)
+    g = torch.Generator().manual_seed(5)
+    k_max = 200
+    idx = torch.full((2, 2, k_max), -1, dtype=torch.int32)
+    for b in range(2):
+        for h in range(2):
+            idx[b, h, : k_small[b]] = torch.randperm(lens[b], generator=g)[: k_small[b]].to(torch.int32)
+    idx[0, 0, 70] = 5000          # flagged, tile 1 of (0, 0)
+    idx[0, 1, 130] = -1           # padding inside the range, tile 2 of (0, 1)
+    idx[1, 0, 149] = 10 ** 6      # flagged, in the ragged last tile of (1, 0)
+    idx = idx.cuda()
+    for active in (None, torch.tensor([1, 0], dtype=torch.int32, device="cuda")):
+        st.small.k.fill_(7.0); st.small.v.fill_(7.0); st.small.len.fill_(0)
+        ctx.gather_small(idx, st.k_small, k_max, st.full_c, st.small_c, active=active)
+        assert ctx.device_status() == rkv.DEV_BAD_INDEX
+        host_idx = idx.cpu().numpy()
+        for b in range(2):
+            fk, fv = host_heads(cache, b, 2, "k"), host_heads(cache, b, 2, "v")
+            sk, sv = host_heads(st.small, b, 2, "k"), host_heads(st.small, b, 2, "v")
+            on = active is None or int(active[b]) == 1
+            assert int(st.small.len[b]) == (k_small[b] if on else 0)
+            seven = bits(torch.tensor([7.0], dtype=torch.bfloat16))[0]
+            for h in range(2):
+                for r in range(st.small.cap[b].item()):
+                    j = host_idx[b, h, r] if r < k_small[b] else -1
+                    if on and 0 <= j < lens[b]:
+                        assert np.array_equal(sk[h, r], fk[h, j]) and np.array_equal(sv[h, r], fv[h, j]), (b, h, r)
+                    else:
+                        assert (sk[h, r] == seven).all() and (sv[h, r] == seven).all(), (b, h, r)
+
+
 def test_deterministic_bits(mods):
     lens, k_small = [5000, 3000], [256, 100]
     ctx, st, cache, q = make_layer(mods, lens, k_small, 32, 8, seed=15)
